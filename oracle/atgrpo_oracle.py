@@ -1,0 +1,270 @@
+"""Plain fp64 CPU oracle for the AT-GRPO policy-update hot path.
+
+TEST INFRASTRUCTURE ONLY.  This file is the slow, obviously-correct statement of
+what the CUDA library computes.  It shares no code with the CUDA path and must
+never be imported by the product package; only the tests, the smoke check and
+the benchmark's CPU-baseline leg call it.
+
+Everything is NumPy in float64.  Each function restates one definition of the
+paper (arXiv 2510.11062) in the paper's order and notation:
+
+  group_key            Algorithm 1, "define group key g <- hash(e, i, t)"
+  bucket_by_key        Algorithm 1 / Sec. 4.1 "Agent- and Turn-wise Grouping"
+  group_advantages     Eq. 1 (group-relative advantage)
+  route_tokens         Sec. 3 "Role-sharing vs. Role-specialized", B_m = U_{sigma(i)=m} D_i
+  token_logprobs       pi_theta in Eq. 2: log-softmax of the LM-head logits at the sampled token
+  clipped_objective    Eq. 2, per token (token-level credit, Sec. 4.1 "Reward Mask")
+  policy_loss          Eq. 2, one loss per policy m
+  policy_loss_grads    gradient of Eq. 2 w.r.t. the hidden states H and the head W_m
+
+Readings taken where the paper is silent (each is pinned by a test, none by the
+paper's own numbers -- the paper prints no worked example):
+  * F_norm of Eq. 1 is the standard deviation of the group's rewards;
+    population (ddof=0) by default, Bessel (ddof=1) on request.
+  * A = (R - mean) / (std + eps), eps added outside the square root.
+  * a group of one candidate has A = 0 (no comparison, no learning signal).
+  * the ratio of Eq. 2 is taken per response token and the expectation is the
+    mean over all response tokens of policy m's batch.
+  * hash(e, i, t) is the collision-free mixed-radix index (e*N + i)*T + t.
+  * no KL, entropy or temperature term (entropy coefficient 0, T_sample 1).
+Parity status: every function below is pinned by tests/test_oracle_pins.py
+against closed forms, invariants, brute force, finite differences or an
+independent library routine.  The *readings* above (std convention, eps
+placement, token- vs sequence-level ratio, denominator) are "parity unpinned"
+by the paper itself.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+__all__ = [
+    "group_key", "bucket_by_key", "group_advantages", "route_tokens",
+    "token_logprobs", "clipped_objective", "policy_loss", "dloss_dlogp", "policy_loss_grads",
+    "policy_loss_grad_rows",
+]
+
+
+def _f64(x):
+    """Widen any array-like (NumPy array or CPU torch tensor, bf16 included) to float64."""
+    if hasattr(x, "detach"):                      # torch tensor, without importing torch here
+        x = x.detach().cpu().double().numpy()
+    return np.asarray(x, dtype=np.float64)
+
+
+def _i64(x):
+    if hasattr(x, "detach"):
+        x = x.detach().cpu().numpy()
+    return np.asarray(x, dtype=np.int64)
+
+
+# --------------------------------------------------------------------------- grouping
+def group_key(env_id, role_id, turn_id, n_env, n_role, n_turn):
+    """Group key of Algorithm 1: one key per (environment e, agent i, turn t).
+
+    The paper's hash(e, i, t) is read as the mixed-radix index g = (e*N + i)*T + t,
+    which cannot collide.  Ids outside their declared range are an error."""
+    e, i, t = _i64(env_id), _i64(role_id), _i64(turn_id)
+    if ((e < 0) | (e >= n_env) | (i < 0) | (i >= n_role) | (t < 0) | (t >= n_turn)).any():
+        raise ValueError("group id out of range")
+    return (e * n_role + i) * n_turn + t
+
+
+def bucket_by_key(key, n_slots):
+    """Collect the items that share a key (Sec. 4.1: data stored together under g).
+
+    Returns (offsets[n_slots+1], perm[n_items]): slot s owns perm[offsets[s]:offsets[s+1]],
+    listed in ascending item index (a stable counting sort).  Empty slots are allowed
+    (an environment that terminated early leaves its later turns empty)."""
+    key = _i64(key)
+    if key.size and (key.min() < 0 or key.max() >= n_slots):
+        raise ValueError("key out of range")
+    counts = np.zeros(n_slots, dtype=np.int64)
+    for k in key:                                   # histogram
+        counts[k] += 1
+    offsets = np.zeros(n_slots + 1, dtype=np.int64)
+    for s in range(n_slots):                        # exclusive scan
+        offsets[s + 1] = offsets[s] + counts[s]
+    cursor = offsets[:-1].copy()
+    perm = np.zeros(key.size, dtype=np.int64)
+    for c in range(key.size):                       # stable placement, ascending item index
+        perm[cursor[key[c]]] = c
+        cursor[key[c]] += 1
+    return offsets, perm
+
+
+def group_advantages(rewards, key, n_slots, std_eps=1e-6, ddof=0):
+    """Eq. 1: A(a^(c)) = (R(a^(c)) - mean_c R) / F_norm({R}) inside every group.
+
+    F_norm = std + std_eps with std the (ddof) standard deviation of the group's K
+    rewards, two-pass formula.  K = 1 gives A = 0.
+    Returns (adv[n_cand], mean[n_slots], std[n_slots]); empty slots report mean = std = 0."""
+    r = _f64(rewards)
+    offsets, perm = bucket_by_key(key, n_slots)
+    adv = np.zeros(r.size, dtype=np.float64)
+    mean = np.zeros(n_slots, dtype=np.float64)
+    std = np.zeros(n_slots, dtype=np.float64)
+    for s in range(n_slots):
+        members = perm[offsets[s]:offsets[s + 1]]
+        K = members.size
+        if K == 0:
+            continue
+        R = r[members]
+        mu = R.sum() / K
+        if K - ddof > 0:
+            sd = np.sqrt(((R - mu) ** 2).sum() / (K - ddof))
+        else:
+            sd = 0.0
+        mean[s], std[s] = mu, sd
+        if K > 1:
+            adv[members] = (R - mu) / (sd + std_eps)
+    return adv, mean, std
+
+
+# --------------------------------------------------------------------------- routing
+def route_tokens(role_of_token, head_of_role, n_heads):
+    """Per-model batch B_m = union of D_i over the agents i with sigma(i) = m.
+
+    role_of_token[j] is the agent i that produced response token j, head_of_role is
+    sigma.  Returns (head_of_token, offsets[n_heads+1], perm[T]) with the tokens of
+    head m listed in ascending token index."""
+    role = _i64(role_of_token)
+    sigma = _i64(head_of_role)
+    if role.size and (role.min() < 0 or role.max() >= sigma.size):
+        raise ValueError("role out of range")
+    if sigma.size and (sigma.min() < 0 or sigma.max() >= n_heads):
+        raise ValueError("head out of range")
+    head = sigma[role] if role.size else np.zeros(0, dtype=np.int64)
+    offsets, perm = bucket_by_key(head, n_heads)
+    return head, offsets, perm
+
+
+# --------------------------------------------------------------------------- LM head
+def token_logprobs(H, W, target):
+    """log pi_theta(y_j | .) for every response token j under one LM head.
+
+    z_j = H_j W^T (all V logits), lse_j = log sum_v exp(z_jv),
+    logp_j = z_{j, y_j} - lse_j.  Sampling temperature 1, no other term.
+    Returns (lse[T], logp[T], z_target[T])."""
+    H, W, y = _f64(H), _f64(W), _i64(target)
+    if y.size and (y.min() < 0 or y.max() >= W.shape[0]):
+        raise ValueError("target out of range")
+    z = H @ W.T                                              # [T, V]
+    zmax = z.max(axis=1)
+    lse = zmax + np.log(np.exp(z - zmax[:, None]).sum(axis=1))
+    zt = z[np.arange(y.size), y]
+    return lse, zt - lse, zt
+
+
+# --------------------------------------------------------------------------- Eq. 2
+def clipped_objective(logp, old_logp, adv_of_token, eps_low=0.2, eps_high=0.2):
+    """Per-token term of Eq. 2 (without the sign and the mean).
+
+    r = pi_theta / pi_theta_old = exp(logp - old_logp);
+    term = min(r*A, clip(r, 1-eps_low, 1+eps_high)*A).
+    Also returns r and `active`, the indicator that d term / d r = A (the unclipped
+    branch attains the min; ties pass the gradient; A = 0 is inactive)."""
+    lp, lo, A = _f64(logp), _f64(old_logp), _f64(adv_of_token)
+    r = np.exp(lp - lo)
+    rc = np.minimum(np.maximum(r, 1.0 - eps_low), 1.0 + eps_high)
+    unclipped, clipped = r * A, rc * A
+    term = np.minimum(unclipped, clipped)
+    active = (unclipped <= clipped) & (A != 0.0)
+    return term, r, active
+
+
+def policy_loss(logp, old_logp, adv, resp_of_token, head_of_token, n_heads,
+                eps_low=0.2, eps_high=0.2):
+    """Eq. 2 for every policy m: L_m = -(1/T_m) sum_{j in B_m} term_j.
+
+    Token-level credit: token j carries the advantage of the response it belongs to,
+    A = adv[resp_of_token[j]].  A policy with no token has loss 0.
+    Returns (loss[n_heads], T_m[n_heads], clip_counts[n_heads, 2]) where clip_counts
+    counts the tokens whose ratio lies below 1-eps_low / above 1+eps_high."""
+    A = _f64(adv)[_i64(resp_of_token)]
+    head = _i64(head_of_token)
+    term, r, _ = clipped_objective(logp, old_logp, A, eps_low, eps_high)
+    loss = np.zeros(n_heads, dtype=np.float64)
+    count = np.zeros(n_heads, dtype=np.int64)
+    clip_counts = np.zeros((n_heads, 2), dtype=np.int64)
+    for m in range(n_heads):
+        sel = head == m
+        count[m] = sel.sum()
+        if count[m]:
+            loss[m] = -term[sel].sum() / count[m]
+            clip_counts[m, 0] = (r[sel] < 1.0 - eps_low).sum()
+            clip_counts[m, 1] = (r[sel] > 1.0 + eps_high).sum()
+    return loss, count, clip_counts
+
+
+def dloss_dlogp(logp, old_logp, adv, resp_of_token, head_of_token, n_heads, grad_loss=None,
+                eps_low=0.2, eps_high=0.2):
+    """c_j = d(sum_m grad_loss_m * L_m) / d logp_j = -grad_loss_m * A * r * active / T_m."""
+    A = _f64(adv)[_i64(resp_of_token)]
+    head = _i64(head_of_token)
+    _, r, active = clipped_objective(logp, old_logp, A, eps_low, eps_high)
+    count = np.bincount(head, minlength=n_heads).astype(np.float64)
+    g = np.ones(n_heads) if grad_loss is None else _f64(grad_loss)
+    denom = np.where(count > 0, count, 1.0)
+    return -(g[head] / denom[head]) * A * r * active
+
+
+def policy_loss_grads(H, W_list, target, old_logp, adv, resp_of_token, head_of_token,
+                      grad_loss=None, eps_low=0.2, eps_high=0.2):
+    """Gradient of sum_m grad_loss_m * L_m (Eq. 2) w.r.t. H and every head W_m.
+
+    With c_j = dL/dlogp_j and p_jv = softmax(z_j)_v:
+      dL/dz_jv = c_j * ([v = y_j] - p_jv)
+      dH_j     = sum_v dL/dz_jv * W_m[v, :]      (m = head of token j)
+      dW_m[v]  = sum_{j in B_m} dL/dz_jv * H_j
+    Returns (dH[T, d], [dW_m[V, d]])."""
+    Hd = _f64(H)
+    y = _i64(target)
+    head = _i64(head_of_token)
+    M = len(W_list)
+    logp = np.zeros(Hd.shape[0])
+    P = [None] * M
+    for m in range(M):
+        sel = np.nonzero(head == m)[0]
+        Wm = _f64(W_list[m])
+        z = Hd[sel] @ Wm.T
+        lse = np.log(np.exp(z - z.max(axis=1, keepdims=True)).sum(axis=1)) + z.max(axis=1)
+        P[m] = np.exp(z - lse[:, None])
+        logp[sel] = z[np.arange(sel.size), y[sel]] - lse
+    c = dloss_dlogp(logp, old_logp, adv, resp_of_token, head, M, grad_loss, eps_low, eps_high)
+    dH = np.zeros_like(Hd)
+    dW = []
+    for m in range(M):
+        sel = np.nonzero(head == m)[0]
+        Wm = _f64(W_list[m])
+        dz = -P[m] * c[sel][:, None]
+        dz[np.arange(sel.size), y[sel]] += c[sel]
+        dH[sel] = dz @ Wm
+        dW.append(dz.T @ Hd[sel])
+    return dH, dW
+
+
+def policy_loss_grad_rows(H, W, target, lse, coef, token_rows=None, vocab_rows=None):
+    """Selected rows of dH and dW for one head, from already-known lse and c_j = dL/dlogp_j.
+
+    Same formulas as policy_loss_grads; used where the full [T,V] softmax does not fit:
+    a dH row needs only that token's softmax, a dW row needs p_jv of one v for all j.
+    `coef` is c_j of policy_loss_grads (sign included).  H, W, target, lse, coef all refer
+    to the tokens of this head only."""
+    Hd, Wd = _f64(H), _f64(W)
+    y, lse, c = _i64(target), _f64(lse), _f64(coef)
+    out_h = out_w = None
+    if token_rows is not None:
+        rows = _i64(token_rows)
+        z = Hd[rows] @ Wd.T
+        p = np.exp(z - lse[rows][:, None])
+        dz = -p * c[rows][:, None]
+        dz[np.arange(rows.size), y[rows]] += c[rows]
+        out_h = dz @ Wd
+    if vocab_rows is not None:
+        vs = _i64(vocab_rows)
+        z = Hd @ Wd[vs].T                                   # [T, n_v]
+        p = np.exp(z - lse[:, None])
+        dz = -p * c[:, None]
+        dz += c[:, None] * (y[:, None] == vs[None, :])
+        out_w = dz.T @ Hd
+    return out_h, out_w
