@@ -1,0 +1,183 @@
+/*
+ * atgrpo.h -- C ABI of libatgrpo: the data-parallel hot path of the AT-GRPO policy update
+ * (arXiv 2510.11062) for NVIDIA B200 (sm_100a).
+ *
+ * Two operations of the paper are exported:
+ *   - the agent- and turn-wise group-relative advantage (Eq. 1 applied to the groups of
+ *     Algorithm 1, "define group key g <- hash(e, i, t)"), and
+ *   - the clipped-ratio policy loss (Eq. 2) through the LM head, forward and backward, for one
+ *     shared policy (M = 1) or one policy per role (M = N), Sec. 3 "Role-sharing vs.
+ *     Role-specialized Policy Optimization".
+ *
+ * Conventions common to every entry point
+ *   - Every pointer is a DEVICE pointer owned by the caller unless its comment says "host".
+ *     The library allocates no memory, keeps no state between calls, never synchronises the
+ *     device and enqueues all work on `stream` (a cudaStream_t passed as void*; NULL = the
+ *     legacy default stream).  Scratch comes from `workspace`, at least as many bytes as the
+ *     matching *_workspace_bytes() query returns, 256-byte aligned, private to the call
+ *     until the enqueued work has finished.
+ *   - Return value: ATGRPO_OK, or an error detected on the host, in which case nothing was
+ *     enqueued and no output was touched.
+ *   - Problems only the device can see (an index outside its range, a bounded wait that ran
+ *     out) are reported through `device_status`, one int32 in device memory that the caller
+ *     zeroes: the first error code is written there (first writer wins, later ones keep it),
+ *     the offending element is skipped without any out-of-bounds access and the kernels run to
+ *     completion.  No entry point traps, asserts or aborts.
+ *   - Arrays are dense and row-major.  int32 index arrays, fp32 statistics, bf16 operands.
+ *   - Calls may run concurrently on different streams if they use different workspaces and
+ *     different outputs.
+ */
+#ifndef ATGRPO_H_
+#define ATGRPO_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum atgrpo_status {
+  ATGRPO_OK = 0,
+  ATGRPO_ERR_INVALID_ARG = 1, /* NULL where data is required, negative size, bad enum       */
+  ATGRPO_ERR_UNSUPPORTED = 2, /* device is not sm_100, d not a multiple of 8, M too large ... */
+  ATGRPO_ERR_WORKSPACE = 3,   /* workspace NULL, misaligned or too small                      */
+  ATGRPO_ERR_BAD_INDEX = 4,   /* device-detected: an id / token / role outside its range      */
+  ATGRPO_ERR_TIMEOUT = 5,     /* device-detected: a bounded wait inside a kernel expired      */
+  ATGRPO_ERR_CUDA = 6         /* a CUDA runtime or driver call failed on the host             */
+} atgrpo_status;
+
+enum { ATGRPO_BF16 = 0, ATGRPO_F32 = 1 };
+
+/* Largest number of policies (LM heads) one call can route to. */
+#define ATGRPO_MAX_HEADS 8
+
+/* Scalars of Eq. 1 and Eq. 2.  The paper gives the symbols, not the values: epsilon of Eq. 2 is
+ * clip_eps_low / clip_eps_high (0.2 both in all shipped workloads); F_norm of Eq. 1 is
+ * std + std_eps with the population (ddof = 0) or Bessel (ddof = 1) standard deviation. */
+typedef struct atgrpo_params {
+  float clip_eps_low;
+  float clip_eps_high;
+  float std_eps;
+  int32_t ddof;
+  int32_t dH_dtype;      /* ATGRPO_BF16 (default) or ATGRPO_F32: element type of dH            */
+  int32_t dW_dtype;      /* ATGRPO_F32 (default) or ATGRPO_BF16: element type of every dW_m    */
+  int32_t accumulate_dW; /* 0: dW_m is overwritten; 1: dW_m += gradient (gradient accumulation)*/
+} atgrpo_params;
+
+/* Text for a status code (static storage, never NULL). */
+const char* atgrpo_status_string(int status);
+
+/* ------------------------------------------------------------------------------------------
+ * Grouped advantage -- Eq. 1 over the (environment, agent, turn) groups of Algorithm 1.
+ *
+ * Candidate c (one sampled response) carries reward rewards[c] and the ids env_id[c] in
+ * [0,n_env), role_id[c] in [0,n_role), turn_id[c] in [0,n_turn); candidates may come in any
+ * order.  Its group is g = (env*n_role + role)*n_turn + turn, a collision-free stand-in for the
+ * paper's hash(e,i,t); G = n_env*n_role*n_turn slots, empty slots allowed, G < 2^31.
+ * For each non-empty group of K members: mu = mean, sigma = std (params->ddof), and
+ *   adv[c] = (rewards[c] - mu) / (sigma + params->std_eps);   K = 1 gives adv = 0.
+ * Sums run in fp64 in ascending candidate order, so the result is bit-reproducible and a group
+ * of identical rewards yields exact zeros.
+ *
+ * Outputs: adv[n_cand] (required).  Optional (NULL to skip): group_of_cand[n_cand] = g;
+ * group_offsets[G+1] and group_perm[n_cand], the stable bucketing (slot s owns
+ * group_perm[group_offsets[s] .. group_offsets[s+1]) in ascending candidate index);
+ * group_mean[G], group_std[G] (0 for empty slots).
+ * A candidate with an id out of range raises ATGRPO_ERR_BAD_INDEX in *device_status, gets
+ * adv = 0 and belongs to no group.
+ * n_cand = 0 is valid (offsets are zero-filled).  n_cand < 2^31.
+ * ------------------------------------------------------------------------------------------ */
+size_t atgrpo_group_advantages_workspace_bytes(int64_t n_cand, int64_t n_groups);
+
+int atgrpo_group_advantages(
+    const float* rewards, const int32_t* env_id, const int32_t* role_id, const int32_t* turn_id,
+    int64_t n_cand, int32_t n_env, int32_t n_role, int32_t n_turn,
+    const atgrpo_params* params /* host */,
+    float* adv,
+    int32_t* group_of_cand, int32_t* group_offsets, int32_t* group_perm,
+    float* group_mean, float* group_std,
+    int32_t* device_status, void* workspace, size_t workspace_bytes, void* stream);
+
+/* ------------------------------------------------------------------------------------------
+ * Clipped-ratio loss from given log-probabilities -- Eq. 2 alone, one policy.
+ *
+ * For response token j: rho = exp(logp[j] - old_logp[j]), A = adv[resp_of_token[j]]
+ * (token-level credit: every response token carries its response's advantage, Sec. 4.1),
+ *   l_j = -min(rho*A, clip(rho, 1-eps_low, 1+eps_high)*A),   loss[0] = (1/T) sum_j l_j,
+ * summed in fp64 in a fixed order (bit-reproducible).  T = 0 gives loss = 0.
+ * Optional outputs: coef[T] = A*rho*[unclipped branch active]/T, the factor of
+ * d loss / d logit_jv = coef_j*(p_jv - [v = y_j]); clip_counts[2] (int64) = number of tokens with
+ * rho < 1-eps_low and with rho > 1+eps_high.
+ * resp_of_token[j] outside [0,n_resp) raises ATGRPO_ERR_BAD_INDEX; the token counts with A = 0.
+ * ------------------------------------------------------------------------------------------ */
+size_t atgrpo_clipped_loss_workspace_bytes(int64_t T);
+
+int atgrpo_clipped_loss(
+    const float* logp, const float* old_logp, const int32_t* resp_of_token, const float* adv,
+    int64_t T, int64_t n_resp, const atgrpo_params* params /* host */,
+    float* loss, float* coef, int64_t* clip_counts,
+    int32_t* device_status, void* workspace, size_t workspace_bytes, void* stream);
+
+/* ------------------------------------------------------------------------------------------
+ * Policy loss through the LM head, forward -- Eq. 2 with pi_theta evaluated by the head.
+ *
+ * H[T, d] (bf16, row stride ldH elements, ldH >= d, ldH % 8 == 0, 16-byte aligned base) holds,
+ * for every packed response token j, the hidden state that predicts it.  W is a HOST array of
+ * M device pointers, W[m] = bf16 [V, d] contiguous (16-byte aligned): the head of policy m.
+ * target[j] in [0,V) is the sampled token.  Policy of token j: m = head_of_role[role_of_token[j]]
+ * (sigma of the paper) when M > 1; with M == 1 both arrays may be NULL and every token uses W[0].
+ *   z_jv = <H_j, W_m[v]>  (bf16 x bf16, fp32 accumulation on tensor cores; never stored)
+ *   lse[j]  = log sum_v exp(z_jv)          logp[j] = z_{j,target[j]} - lse[j]
+ *   rho_j = exp(logp[j] - old_logp[j]),  A = adv[resp_of_token[j]]
+ *   loss[m] = (1/T_m) sum_{j of policy m} -min(rho_j*A, clip(rho_j)*A)   (0 if T_m = 0)
+ * Outputs: loss[M], logp[T], lse[T] (lse and logp are what the backward call needs).
+ * Optional: role_offsets[M+1], role_perm[T] = stable routing of tokens to policies (tokens of
+ * policy m in ascending token index); clip_counts[M*2] (int64) as in atgrpo_clipped_loss.
+ * Requirements: d % 8 == 0, d >= 64, V >= 1, 1 <= M <= ATGRPO_MAX_HEADS, T < 2^31 - 2^16.
+ * Out-of-range target / role / head / response index: ATGRPO_ERR_BAD_INDEX in *device_status;
+ * such a token gets logp = lse = 0 and contributes nothing.
+ * ------------------------------------------------------------------------------------------ */
+size_t atgrpo_policy_loss_workspace_bytes(int64_t T, int32_t d, int32_t V, int32_t M, int32_t is_bwd);
+
+int atgrpo_policy_loss_fwd(
+    const void* H, int64_t ldH, const void* const* W /* host array */, int32_t M,
+    const int32_t* target,
+    const int32_t* role_of_token, const int32_t* head_of_role, int32_t n_role,
+    const int32_t* resp_of_token, const float* adv, int64_t n_resp,
+    const float* old_logp,
+    int64_t T, int32_t d, int32_t V, const atgrpo_params* params /* host */,
+    float* loss, float* logp, float* lse,
+    int32_t* role_offsets, int32_t* role_perm, int64_t* clip_counts,
+    int32_t* device_status, void* workspace, size_t workspace_bytes, void* stream);
+
+/* ------------------------------------------------------------------------------------------
+ * Policy loss through the LM head, backward -- gradient of sum_m grad_loss[m]*loss[m] (Eq. 2)
+ * with respect to H and every W_m (the update theta_m <- theta_m - eta*grad L of Sec. 3).
+ *
+ * Inputs as in the forward call, plus logp[T] and lse[T] as the forward call wrote them and
+ * grad_loss[M] (device; NULL = all ones).  With
+ *   coef_j = grad_loss[m]*A*rho_j*[rho_j*A <= clip(rho_j)*A and A != 0]/T_m,
+ * the softmax is recomputed tile by tile, p_jv = exp(z_jv - lse[j]), and
+ *   dZ_jv = coef_j*(p_jv - [v = target[j]])   (rounded to bf16 for the contractions)
+ *   dH[j, :]   = sum_v dZ_jv * W_m[v, :]          -> dH [T, d], row stride d, params->dH_dtype
+ *   dW[m][v,:] = sum_{j of policy m} dZ_jv*H[j,:] -> dW[m] [V, d] contiguous, params->dW_dtype,
+ *                overwritten or accumulated into (params->accumulate_dW).
+ * dW is a HOST array of M device pointers.  A policy without tokens gets dW = 0 (or is left
+ * unchanged when accumulating).  The [T, V] logits and their gradient are never materialised:
+ * dZ lives in a bounded vocabulary-chunk buffer inside the workspace.
+ * ------------------------------------------------------------------------------------------ */
+int atgrpo_policy_loss_bwd(
+    const void* H, int64_t ldH, const void* const* W /* host array */, int32_t M,
+    const int32_t* target,
+    const int32_t* role_of_token, const int32_t* head_of_role, int32_t n_role,
+    const int32_t* resp_of_token, const float* adv, int64_t n_resp,
+    const float* old_logp, const float* logp, const float* lse, const float* grad_loss,
+    int64_t T, int32_t d, int32_t V, const atgrpo_params* params /* host */,
+    void* dH, void* const* dW /* host array */,
+    int32_t* device_status, void* workspace, size_t workspace_bytes, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ATGRPO_H_ */

@@ -1,0 +1,209 @@
+"""ctypes binding of libatgrpo.so: same names and arguments as include/atgrpo.h.
+
+Only argument marshalling happens here: torch tensors supply device pointers, the current
+CUDA stream and the workspace; every step of the computation runs inside the library's kernels.
+There is no CPU path: loading fails loudly when the library is missing, and every compute call
+requires CUDA tensors.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libatgrpo.so")
+
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_BAD_INDEX, ERR_TIMEOUT, ERR_CUDA = range(7)
+BF16, F32 = 0, 1
+MAX_HEADS = 8
+
+EXPORTS = (
+    "atgrpo_status_string",
+    "atgrpo_group_advantages_workspace_bytes", "atgrpo_group_advantages",
+    "atgrpo_clipped_loss_workspace_bytes", "atgrpo_clipped_loss",
+    "atgrpo_policy_loss_workspace_bytes", "atgrpo_policy_loss_fwd", "atgrpo_policy_loss_bwd",
+)
+
+
+class AtgrpoError(RuntimeError):
+    pass
+
+
+class _Params(ctypes.Structure):
+    _fields_ = [("clip_eps_low", ctypes.c_float), ("clip_eps_high", ctypes.c_float),
+                ("std_eps", ctypes.c_float), ("ddof", ctypes.c_int32),
+                ("dH_dtype", ctypes.c_int32), ("dW_dtype", ctypes.c_int32),
+                ("accumulate_dW", ctypes.c_int32)]
+
+
+@dataclass
+class Params:
+    clip_eps_low: float = 0.2
+    clip_eps_high: float = 0.2
+    std_eps: float = 1e-6
+    ddof: int = 0
+    dH_dtype: int = BF16
+    dW_dtype: int = F32
+    accumulate_dW: int = 0
+
+    def c(self) -> _Params:
+        return _Params(self.clip_eps_low, self.clip_eps_high, self.std_eps, self.ddof,
+                       self.dH_dtype, self.dW_dtype, self.accumulate_dW)
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Loads libatgrpo.so (built by paper_2510_11062_b200.build); raises if it is absent."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise AtgrpoError(f"{LIB_PATH} not found: run `python -m paper_2510_11062_b200.build`")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, i64, i32, sz = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int32, ctypes.c_size_t
+        pp = ctypes.POINTER(_Params)
+        L.atgrpo_status_string.restype = ctypes.c_char_p
+        L.atgrpo_status_string.argtypes = [ctypes.c_int]
+        L.atgrpo_group_advantages_workspace_bytes.restype = sz
+        L.atgrpo_group_advantages_workspace_bytes.argtypes = [i64, i64]
+        L.atgrpo_group_advantages.restype = ctypes.c_int
+        L.atgrpo_group_advantages.argtypes = [vp, vp, vp, vp, i64, i32, i32, i32, pp, vp, vp, vp, vp,
+                                              vp, vp, vp, vp, sz, vp]
+        L.atgrpo_clipped_loss_workspace_bytes.restype = sz
+        L.atgrpo_clipped_loss_workspace_bytes.argtypes = [i64]
+        L.atgrpo_clipped_loss.restype = ctypes.c_int
+        L.atgrpo_clipped_loss.argtypes = [vp, vp, vp, vp, i64, i64, pp, vp, vp, vp, vp, vp, sz, vp]
+        L.atgrpo_policy_loss_workspace_bytes.restype = sz
+        L.atgrpo_policy_loss_workspace_bytes.argtypes = [i64, i32, i32, i32, i32]
+        L.atgrpo_policy_loss_fwd.restype = ctypes.c_int
+        L.atgrpo_policy_loss_fwd.argtypes = [vp, i64, ctypes.POINTER(vp), i32, vp, vp, vp, i32, vp, vp,
+                                             i64, vp, i64, i32, i32, pp, vp, vp, vp, vp, vp, vp, vp,
+                                             vp, sz, vp]
+        L.atgrpo_policy_loss_bwd.restype = ctypes.c_int
+        L.atgrpo_policy_loss_bwd.argtypes = [vp, i64, ctypes.POINTER(vp), i32, vp, vp, vp, i32, vp, vp,
+                                             i64, vp, vp, vp, vp, i64, i32, i32, pp, vp,
+                                             ctypes.POINTER(vp), vp, vp, sz, vp]
+        _lib = L
+    return _lib
+
+
+def status_string(code: int) -> str:
+    return lib().atgrpo_status_string(int(code)).decode()
+
+
+def _check(rc: int, what: str) -> None:
+    if rc != OK:
+        raise AtgrpoError(f"{what}: {status_string(rc)} ({rc})")
+
+
+def _ptr(t, dtype=None):
+    if t is None:
+        return None
+    if not t.is_cuda:
+        raise AtgrpoError("libatgrpo takes device memory only (got a CPU tensor)")
+    if dtype is not None and t.dtype != dtype:
+        raise AtgrpoError(f"expected {dtype}, got {t.dtype}")
+    if not t.is_contiguous():
+        raise AtgrpoError("tensor must be contiguous")
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _ptr_array(tensors, dtype):
+    arr = (ctypes.c_void_p * len(tensors))()
+    for i, t in enumerate(tensors):
+        arr[i] = _ptr(t, dtype).value
+    return arr
+
+
+def new_status(device) -> torch.Tensor:
+    return torch.zeros(1, dtype=torch.int32, device=device)
+
+
+def workspace(nbytes: int, device) -> torch.Tensor:
+    return torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
+
+
+def atgrpo_group_advantages_workspace_bytes(n_cand: int, n_groups: int) -> int:
+    return int(lib().atgrpo_group_advantages_workspace_bytes(n_cand, n_groups))
+
+
+def atgrpo_group_advantages(rewards, env_id, role_id, turn_id, n_env, n_role, n_turn, params: Params,
+                            adv, group_of_cand=None, group_offsets=None, group_perm=None,
+                            group_mean=None, group_std=None, device_status=None, workspace=None):
+    """Eq. 1 over the (env, role, turn) groups; see include/atgrpo.h.  Enqueues on the current stream."""
+    i32, f32 = torch.int32, torch.float32
+    rc = lib().atgrpo_group_advantages(
+        _ptr(rewards, f32), _ptr(env_id, i32), _ptr(role_id, i32), _ptr(turn_id, i32),
+        rewards.numel(), n_env, n_role, n_turn, ctypes.byref(params.c()), _ptr(adv, f32),
+        _ptr(group_of_cand, i32), _ptr(group_offsets, i32), _ptr(group_perm, i32),
+        _ptr(group_mean, f32), _ptr(group_std, f32), _ptr(device_status, i32),
+        _ptr(workspace), workspace.numel(), _stream())
+    _check(rc, "atgrpo_group_advantages")
+
+
+def atgrpo_clipped_loss_workspace_bytes(T: int) -> int:
+    return int(lib().atgrpo_clipped_loss_workspace_bytes(T))
+
+
+def atgrpo_clipped_loss(logp, old_logp, resp_of_token, adv, params: Params, loss, coef=None,
+                        clip_counts=None, device_status=None, workspace=None):
+    """Eq. 2 from given log-probabilities (one policy); see include/atgrpo.h."""
+    i32, f32 = torch.int32, torch.float32
+    rc = lib().atgrpo_clipped_loss(
+        _ptr(logp, f32), _ptr(old_logp, f32), _ptr(resp_of_token, i32), _ptr(adv, f32),
+        logp.numel(), adv.numel(), ctypes.byref(params.c()), _ptr(loss, f32), _ptr(coef, f32),
+        _ptr(clip_counts, torch.int64), _ptr(device_status, i32), _ptr(workspace),
+        workspace.numel(), _stream())
+    _check(rc, "atgrpo_clipped_loss")
+
+
+def atgrpo_policy_loss_workspace_bytes(T: int, d: int, V: int, M: int, is_bwd: bool) -> int:
+    return int(lib().atgrpo_policy_loss_workspace_bytes(T, d, V, M, 1 if is_bwd else 0))
+
+
+def atgrpo_policy_loss_fwd(H, W, target, role_of_token, head_of_role, resp_of_token, adv, old_logp,
+                           params: Params, loss, logp, lse, role_offsets=None, role_perm=None,
+                           clip_counts=None, device_status=None, workspace=None):
+    """Eq. 2 through the LM head(s) W (list of [V,d] bf16 tensors), forward; see include/atgrpo.h."""
+    i32, f32, bf = torch.int32, torch.float32, torch.bfloat16
+    T, d = H.shape
+    V = W[0].shape[0]
+    if H.stride(1) != 1:
+        raise AtgrpoError("H must have unit stride along d")
+    n_role = 0 if head_of_role is None else head_of_role.numel()
+    rc = lib().atgrpo_policy_loss_fwd(
+        ctypes.c_void_p(H.data_ptr()), H.stride(0) if T > 1 else d, _ptr_array(W, bf), len(W),
+        _ptr(target, i32), _ptr(role_of_token, i32), _ptr(head_of_role, i32), n_role,
+        _ptr(resp_of_token, i32), _ptr(adv, f32), adv.numel(), _ptr(old_logp, f32), T, d, V,
+        ctypes.byref(params.c()), _ptr(loss, f32), _ptr(logp, f32), _ptr(lse, f32),
+        _ptr(role_offsets, i32), _ptr(role_perm, i32), _ptr(clip_counts, torch.int64),
+        _ptr(device_status, i32), _ptr(workspace), workspace.numel(), _stream())
+    _check(rc, "atgrpo_policy_loss_fwd")
+
+
+def atgrpo_policy_loss_bwd(H, W, target, role_of_token, head_of_role, resp_of_token, adv, old_logp,
+                           logp, lse, grad_loss, params: Params, dH, dW, device_status=None,
+                           workspace=None):
+    """Gradient of sum_m grad_loss[m]*loss[m] w.r.t. H and every W_m; see include/atgrpo.h."""
+    i32, f32, bf = torch.int32, torch.float32, torch.bfloat16
+    T, d = H.shape
+    V = W[0].shape[0]
+    n_role = 0 if head_of_role is None else head_of_role.numel()
+    dh_t = bf if params.dH_dtype == BF16 else f32
+    dw_t = bf if params.dW_dtype == BF16 else f32
+    rc = lib().atgrpo_policy_loss_bwd(
+        ctypes.c_void_p(H.data_ptr()), H.stride(0) if T > 1 else d, _ptr_array(W, bf), len(W),
+        _ptr(target, i32), _ptr(role_of_token, i32), _ptr(head_of_role, i32), n_role,
+        _ptr(resp_of_token, i32), _ptr(adv, f32), adv.numel(), _ptr(old_logp, f32),
+        _ptr(logp, f32), _ptr(lse, f32), _ptr(grad_loss, f32), T, d, V, ctypes.byref(params.c()),
+        _ptr(dH, dh_t), _ptr_array(dW, dw_t), _ptr(device_status, i32), _ptr(workspace),
+        workspace.numel(), _stream())
+    _check(rc, "atgrpo_policy_loss_bwd")

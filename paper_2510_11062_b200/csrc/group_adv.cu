@@ -1,0 +1,385 @@
+// Agent- and turn-wise grouped advantage (Eq. 1 over the groups of Algorithm 1).
+//
+// Pipeline, all on the caller's stream, no host synchronisation:
+//   key_count  : g = (e*n_role + i)*n_turn + t, per-group histogram; the atomic's return value is
+//                the candidate's (arbitrary) arrival slot inside its group
+//   scan       : exclusive scan of the histogram -> group_offsets        (two launches)
+//   scatter    : unordered bucket fill, perm_u[offsets[g] + slot] = c
+//   stats      : one thread per group sorts its few members by candidate index (which makes the
+//                permutation stable and the fp64 sums order-fixed), then mean / std / advantage.
+// Groups of the paper hold K = 4 .. 16 candidates, far fewer than a warp, so a thread per group
+// with block-cooperative coalesced staging keeps every lane busy; blocks that meet a large group
+// switch to a block-per-group path (shared-memory bitonic sort or an ordered rescan) with a
+// shuffle/shared-memory tree reduction.
+#include "internal.h"
+
+namespace atgrpo {
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kScanItems = 4;                        // counts per thread in the scan kernels
+constexpr int kScanBlock = kThreads * kScanItems;    // 1024 groups per scan block
+constexpr int kCap = 4096;                           // staged members per stats block
+constexpr int kSerialMaxK = 64;                      // largest group a single thread sorts
+
+__device__ __forceinline__ int group_of(int e, int i, int t, int n_env, int n_role, int n_turn) {
+  const bool ok = (unsigned)e < (unsigned)n_env && (unsigned)i < (unsigned)n_role &&
+                  (unsigned)t < (unsigned)n_turn;
+  return ok ? (e * n_role + i) * n_turn + t : -1;
+}
+
+template <bool kVec>
+__global__ void __launch_bounds__(kThreads)
+k_key_count(const int32_t* __restrict__ env, const int32_t* __restrict__ role,
+            const int32_t* __restrict__ turn, int n, int n_env, int n_role, int n_turn,
+            int32_t* __restrict__ count, int32_t* __restrict__ slot, int32_t* __restrict__ gid,
+            float* __restrict__ adv, int32_t* status) {
+  const int stride = gridDim.x * blockDim.x;
+  const int tid = blockIdx.x * blockDim.x + threadIdx.x;
+  if (kVec) {
+    const int n4 = n >> 2;
+    for (int q = tid; q < n4; q += stride) {
+      const int4 e = reinterpret_cast<const int4*>(env)[q];
+      const int4 r = reinterpret_cast<const int4*>(role)[q];
+      const int4 t = reinterpret_cast<const int4*>(turn)[q];
+      int4 g, s;
+      g.x = group_of(e.x, r.x, t.x, n_env, n_role, n_turn);
+      g.y = group_of(e.y, r.y, t.y, n_env, n_role, n_turn);
+      g.z = group_of(e.z, r.z, t.z, n_env, n_role, n_turn);
+      g.w = group_of(e.w, r.w, t.w, n_env, n_role, n_turn);
+      s.x = g.x >= 0 ? atomicAdd(&count[g.x], 1) : 0;
+      s.y = g.y >= 0 ? atomicAdd(&count[g.y], 1) : 0;
+      s.z = g.z >= 0 ? atomicAdd(&count[g.z], 1) : 0;
+      s.w = g.w >= 0 ? atomicAdd(&count[g.w], 1) : 0;
+      reinterpret_cast<int4*>(gid)[q] = g;
+      reinterpret_cast<int4*>(slot)[q] = s;
+      if ((g.x | g.y | g.z | g.w) < 0) {
+        raise_status(status, ATGRPO_ERR_BAD_INDEX);
+        if (g.x < 0) adv[4 * q + 0] = 0.f;
+        if (g.y < 0) adv[4 * q + 1] = 0.f;
+        if (g.z < 0) adv[4 * q + 2] = 0.f;
+        if (g.w < 0) adv[4 * q + 3] = 0.f;
+      }
+    }
+  }
+  const int first = kVec ? (n & ~3) : 0;
+  for (int c = first + tid; c < n; c += stride) {
+    const int g = group_of(env[c], role[c], turn[c], n_env, n_role, n_turn);
+    gid[c] = g;
+    if (g >= 0) {
+      slot[c] = atomicAdd(&count[g], 1);
+    } else {
+      slot[c] = 0;
+      adv[c] = 0.f;
+      raise_status(status, ATGRPO_ERR_BAD_INDEX);
+    }
+  }
+}
+
+// Inclusive scan of one int per thread across the block (shuffle inside warps, shared across).
+__device__ __forceinline__ int block_inclusive_scan(int v, int* warp_tot /* [kThreads/32] */) {
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int u = __shfl_up_sync(0xffffffffu, v, o);
+    if (lane >= o) v += u;
+  }
+  if (lane == 31) warp_tot[w] = v;
+  __syncthreads();
+  int add = 0;
+  for (int i = 0; i < w; ++i) add += warp_tot[i];
+  __syncthreads();
+  return v + add;
+}
+
+__global__ void __launch_bounds__(kThreads)
+k_block_sums(const int32_t* __restrict__ count, int G, int32_t* __restrict__ block_sum) {
+  __shared__ int warp_tot[kThreads / 32];
+  const int base = blockIdx.x * kScanBlock + threadIdx.x * kScanItems;
+  int v = 0;
+#pragma unroll
+  for (int i = 0; i < kScanItems; ++i)
+    if (base + i < G) v += count[base + i];
+  const int incl = block_inclusive_scan(v, warp_tot);
+  if (threadIdx.x == kThreads - 1) block_sum[blockIdx.x] = incl;
+}
+
+__global__ void __launch_bounds__(kThreads)
+k_scan_offsets(const int32_t* __restrict__ count, int G, const int32_t* __restrict__ block_sum,
+               int32_t* __restrict__ offsets) {
+  __shared__ int warp_tot[kThreads / 32];
+  __shared__ int red[kThreads];
+  // prefix of the blocks before this one, fixed-order tree
+  int pre = 0;
+  for (int b = threadIdx.x; b < (int)blockIdx.x; b += kThreads) pre += block_sum[b];
+  red[threadIdx.x] = pre;
+  __syncthreads();
+  for (int s = kThreads / 2; s > 0; s >>= 1) {
+    if ((int)threadIdx.x < s) red[threadIdx.x] += red[threadIdx.x + s];
+    __syncthreads();
+  }
+  const int block_pre = red[0];
+  const int base = blockIdx.x * kScanBlock + threadIdx.x * kScanItems;
+  int c[kScanItems];
+  int v = 0;
+#pragma unroll
+  for (int i = 0; i < kScanItems; ++i) {
+    c[i] = (base + i < G) ? count[base + i] : 0;
+    v += c[i];
+  }
+  const int incl = block_inclusive_scan(v, warp_tot);
+  int run = block_pre + incl - v;
+#pragma unroll
+  for (int i = 0; i < kScanItems; ++i) {
+    if (base + i < G) offsets[base + i] = run;
+    run += c[i];
+    if (base + i == G - 1) offsets[G] = run;
+  }
+}
+
+__global__ void __launch_bounds__(kThreads)
+k_scatter(const int32_t* __restrict__ gid, const int32_t* __restrict__ slot,
+          const int32_t* __restrict__ offsets, int n, int32_t* __restrict__ perm_u) {
+  const int stride = gridDim.x * blockDim.x;
+  for (int c = blockIdx.x * blockDim.x + threadIdx.x; c < n; c += stride) {
+    const int g = gid[c];
+    if (g >= 0) perm_u[offsets[g] + slot[c]] = c;
+  }
+}
+
+struct StatsArgs {
+  const float* rewards;
+  const int32_t* offsets;
+  const int32_t* gid;
+  int32_t* perm;          // in: unordered buckets, out: ordered
+  float* adv;
+  float* group_mean;
+  float* group_std;
+  int G, n;
+  float std_eps;
+  int ddof;
+};
+
+// Fixed-order block sum of one double per thread.
+__device__ __forceinline__ double block_sum_fixed(double v, double* red) {
+  red[threadIdx.x] = v;
+  __syncthreads();
+  for (int s = kThreads / 2; s > 0; s >>= 1) {
+    if ((int)threadIdx.x < s) red[threadIdx.x] += red[threadIdx.x + s];
+    __syncthreads();
+  }
+  const double r = red[0];
+  __syncthreads();
+  return r;
+}
+
+__global__ void __launch_bounds__(kThreads) k_group_stats(StatsArgs a) {
+  __shared__ int idx_s[kCap];
+  __shared__ __align__(16) float val_s[kCap];
+  __shared__ int warp_tot[kThreads / 32];
+  __shared__ int s_max;
+  __shared__ int s_tot;
+  double* red = reinterpret_cast<double*>(val_s);     // reused by the block-per-group path
+
+  const int g0 = blockIdx.x * kThreads;
+  const int g1 = min(g0 + kThreads, a.G);
+  const int g = g0 + threadIdx.x;
+  const int beg_blk = a.offsets[g0];
+  const int n_blk = a.offsets[g1] - beg_blk;
+  int beg = 0, K = 0;
+  if (g < a.G) {
+    beg = a.offsets[g];
+    K = a.offsets[g + 1] - beg;
+  }
+  if (threadIdx.x == 0) s_max = 0;
+  __syncthreads();
+  atomicMax(&s_max, K);
+  __syncthreads();
+  const int max_k = s_max;
+
+  if (n_blk <= kCap && max_k <= kSerialMaxK) {
+    // ---------------- thread-per-group path ----------------
+    for (int i = threadIdx.x; i < n_blk; i += kThreads) idx_s[i] = a.perm[beg_blk + i];
+    __syncthreads();
+    int* mine = idx_s + (beg - beg_blk);
+    for (int i = 1; i < K; ++i) {                       // insertion sort, ascending candidate index
+      const int x = mine[i];
+      int j = i - 1;
+      while (j >= 0 && mine[j] > x) {
+        mine[j + 1] = mine[j];
+        --j;
+      }
+      mine[j + 1] = x;
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < n_blk; i += kThreads) {
+      const int c = idx_s[i];
+      a.perm[beg_blk + i] = c;
+      val_s[i] = a.rewards[c];
+    }
+    __syncthreads();
+    if (g < a.G) {
+      float* r = val_s + (beg - beg_blk);
+      double mu = 0.0, sd = 0.0;
+      if (K > 0) {
+        double sum = 0.0;
+        for (int i = 0; i < K; ++i) sum += (double)r[i];
+        mu = sum / (double)K;
+        double ss = 0.0;
+        for (int i = 0; i < K; ++i) {
+          const double dlt = (double)r[i] - mu;
+          ss += dlt * dlt;
+        }
+        const int dof = K - a.ddof;
+        sd = dof > 0 ? sqrt(ss / (double)dof) : 0.0;
+        const double den = sd + (double)a.std_eps;
+        for (int i = 0; i < K; ++i) r[i] = K > 1 ? (float)(((double)r[i] - mu) / den) : 0.f;
+      }
+      if (a.group_mean) a.group_mean[g] = (float)mu;
+      if (a.group_std) a.group_std[g] = (float)sd;
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < n_blk; i += kThreads) a.adv[idx_s[i]] = val_s[i];
+    return;
+  }
+
+  // ---------------- block-per-group path (a large group is present) ----------------
+  for (int gg = g0; gg < g1; ++gg) {
+    const int b = a.offsets[gg];
+    const int Kg = a.offsets[gg + 1] - b;
+    double mu = 0.0, sd = 0.0;
+    if (Kg > 0) {
+      int* p = a.perm + b;
+      if (Kg <= kCap) {
+        int n2 = 1;
+        while (n2 < Kg) n2 <<= 1;
+        for (int i = threadIdx.x; i < n2; i += kThreads) idx_s[i] = i < Kg ? p[i] : 0x7fffffff;
+        __syncthreads();
+        for (int k = 2; k <= n2; k <<= 1) {
+          for (int j = k >> 1; j > 0; j >>= 1) {
+            for (int i = threadIdx.x; i < n2; i += kThreads) {
+              const int ixj = i ^ j;
+              if (ixj > i) {
+                const int x = idx_s[i], y = idx_s[ixj];
+                const bool up = (i & k) == 0;
+                if ((x > y) == up) {
+                  idx_s[i] = y;
+                  idx_s[ixj] = x;
+                }
+              }
+            }
+            __syncthreads();
+          }
+        }
+        for (int i = threadIdx.x; i < Kg; i += kThreads) p[i] = idx_s[i];
+        __syncthreads();
+      } else {
+        // ordered rescan of all candidates: members appear in ascending index by construction
+        int run = 0;
+        for (int base = 0; base < a.n; base += kThreads) {
+          const int c = base + threadIdx.x;
+          const int f = (c < a.n && a.gid[c] == gg) ? 1 : 0;
+          const int incl = block_inclusive_scan(f, warp_tot);
+          if (f) p[run + incl - 1] = c;
+          if (threadIdx.x == kThreads - 1) s_tot = incl;
+          __syncthreads();
+          run += s_tot;
+          __syncthreads();
+        }
+      }
+      __threadfence_block();
+      __syncthreads();
+      // statistics: strided partial sums in a fixed order, fixed tree across threads
+      double part = 0.0;
+      for (int i = threadIdx.x; i < Kg; i += kThreads) part += (double)a.rewards[p[i]];
+      mu = block_sum_fixed(part, red) / (double)Kg;
+      part = 0.0;
+      for (int i = threadIdx.x; i < Kg; i += kThreads) {
+        const double dlt = (double)a.rewards[p[i]] - mu;
+        part += dlt * dlt;
+      }
+      const double ss = block_sum_fixed(part, red);
+      const int dof = Kg - a.ddof;
+      sd = dof > 0 ? sqrt(ss / (double)dof) : 0.0;
+      const double den = sd + (double)a.std_eps;
+      for (int i = threadIdx.x; i < Kg; i += kThreads) {
+        const int c = p[i];
+        a.adv[c] = Kg > 1 ? (float)(((double)a.rewards[c] - mu) / den) : 0.f;
+      }
+    }
+    if (threadIdx.x == 0) {
+      if (a.group_mean) a.group_mean[gg] = (float)mu;
+      if (a.group_std) a.group_std[gg] = (float)sd;
+    }
+    __syncthreads();
+  }
+}
+
+struct Plan {
+  size_t count, slot, gid, offsets, perm, block_sum, total;
+};
+Plan make_plan(int64_t n, int64_t G) {
+  Carver c(nullptr);
+  Plan p;
+  p.count = c.off; c.take<int32_t>((size_t)G);
+  p.slot = c.off; c.take<int32_t>((size_t)n);
+  p.gid = c.off; c.take<int32_t>((size_t)n);
+  p.offsets = c.off; c.take<int32_t>((size_t)G + 1);
+  p.perm = c.off; c.take<int32_t>((size_t)n);
+  p.block_sum = c.off; c.take<int32_t>((size_t)((G + kScanBlock - 1) / kScanBlock) + 1);
+  p.total = c.off;
+  return p;
+}
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+}  // namespace
+
+size_t group_adv_workspace_bytes(int64_t n_cand, int64_t n_groups) {
+  return make_plan(n_cand < 0 ? 0 : n_cand, n_groups < 0 ? 0 : n_groups).total;
+}
+
+int group_adv_launch(const float* rewards, const int32_t* env_id, const int32_t* role_id,
+                     const int32_t* turn_id, int64_t n_cand, int32_t n_env, int32_t n_role,
+                     int32_t n_turn, const atgrpo_params& prm, float* adv, int32_t* group_of_cand,
+                     int32_t* group_offsets, int32_t* group_perm, float* group_mean,
+                     float* group_std, int32_t* device_status, void* workspace, cudaStream_t st) {
+  const int64_t G = (int64_t)n_env * n_role * n_turn;
+  const int n = (int)n_cand;
+  const Plan pl = make_plan(n_cand, G);
+  char* ws = static_cast<char*>(workspace);
+  int32_t* count = reinterpret_cast<int32_t*>(ws + pl.count);
+  int32_t* slot = reinterpret_cast<int32_t*>(ws + pl.slot);
+  int32_t* gid = group_of_cand ? group_of_cand : reinterpret_cast<int32_t*>(ws + pl.gid);
+  int32_t* offsets = group_offsets ? group_offsets : reinterpret_cast<int32_t*>(ws + pl.offsets);
+  int32_t* perm = group_perm ? group_perm : reinterpret_cast<int32_t*>(ws + pl.perm);
+  int32_t* block_sum = reinterpret_cast<int32_t*>(ws + pl.block_sum);
+
+  ATGRPO_CUDA_OK(cudaMemsetAsync(count, 0, (size_t)G * sizeof(int32_t), st));
+  if (n == 0) {
+    ATGRPO_CUDA_OK(cudaMemsetAsync(offsets, 0, ((size_t)G + 1) * sizeof(int32_t), st));
+    if (group_mean) ATGRPO_CUDA_OK(cudaMemsetAsync(group_mean, 0, (size_t)G * sizeof(float), st));
+    if (group_std) ATGRPO_CUDA_OK(cudaMemsetAsync(group_std, 0, (size_t)G * sizeof(float), st));
+    return ATGRPO_OK;
+  }
+  const bool vec = aligned16(env_id) && aligned16(role_id) && aligned16(turn_id) &&
+                   aligned16(gid) && aligned16(slot);
+  const int work = vec ? (n + 3) / 4 : n;
+  const int grid_c = (int)((work + kThreads - 1) / kThreads);
+  if (vec)
+    k_key_count<true><<<grid_c, kThreads, 0, st>>>(env_id, role_id, turn_id, n, n_env, n_role,
+                                                   n_turn, count, slot, gid, adv, device_status);
+  else
+    k_key_count<false><<<grid_c, kThreads, 0, st>>>(env_id, role_id, turn_id, n, n_env, n_role,
+                                                    n_turn, count, slot, gid, adv, device_status);
+  const int nb = (int)((G + kScanBlock - 1) / kScanBlock);
+  k_block_sums<<<nb, kThreads, 0, st>>>(count, (int)G, block_sum);
+  k_scan_offsets<<<nb, kThreads, 0, st>>>(count, (int)G, block_sum, offsets);
+  k_scatter<<<(n + kThreads - 1) / kThreads, kThreads, 0, st>>>(gid, slot, offsets, n, perm);
+  StatsArgs a{rewards, offsets, gid, perm, adv, group_mean, group_std, (int)G, n, prm.std_eps,
+              prm.ddof};
+  k_group_stats<<<(int)((G + kThreads - 1) / kThreads), kThreads, 0, st>>>(a);
+  return launch_ok();
+}
+
+}  // namespace atgrpo

@@ -1,0 +1,77 @@
+// Internal launch interfaces between the translation units of libatgrpo.
+#pragma once
+#include "common.cuh"
+
+namespace atgrpo {
+
+// ---- group_adv.cu ---------------------------------------------------------------------------
+size_t group_adv_workspace_bytes(int64_t n_cand, int64_t n_groups);
+int group_adv_launch(const float* rewards, const int32_t* env_id, const int32_t* role_id,
+                     const int32_t* turn_id, int64_t n_cand, int32_t n_env, int32_t n_role,
+                     int32_t n_turn, const atgrpo_params& prm, float* adv, int32_t* group_of_cand,
+                     int32_t* group_offsets, int32_t* group_perm, float* group_mean,
+                     float* group_std, int32_t* device_status, void* workspace, cudaStream_t st);
+
+// Padded 128-row tile schedule the GEMM kernels read.
+struct Schedule {                       // lives in device memory
+  int32_t n_heads;
+  int32_t tile_begin[ATGRPO_MAX_HEADS + 1];   // first 128-row tile of head m in the padded row space
+  int32_t rows[ATGRPO_MAX_HEADS];             // T_m
+  int32_t role_offsets[ATGRPO_MAX_HEADS + 1]; // exclusive scan of T_m
+};
+
+// ---- loss_reduce.cu -------------------------------------------------------------------------
+// Eq. 2 reduction over tokens for up to ATGRPO_MAX_HEADS policies.
+size_t loss_reduce_workspace_bytes(int64_t T);
+int loss_reduce_launch(const float* logp, const float* old_logp, const int32_t* resp_of_token,
+                       const float* adv, int64_t n_resp, const int32_t* role_of_token,
+                       const int32_t* head_of_role, int32_t n_role, int32_t M, int64_t T,
+                       const atgrpo_params& prm, float* loss, float* coef, int64_t* clip_counts,
+                       int32_t* device_status, void* workspace, cudaStream_t st);
+
+// coef[j] = grad_loss[m]*A*rho*[gradient passes]/T_m for every token (0 where unroutable).
+int coef_launch(const float* logp, const float* old_logp, const int32_t* resp_of_token,
+                const float* adv, int64_t n_resp, const int32_t* role_of_token,
+                const int32_t* head_of_role, int32_t n_role, int32_t M, int64_t T,
+                const atgrpo_params& prm, const float* grad_loss, const Schedule* sched,
+                float* coef, int32_t* device_status, cudaStream_t st);
+
+// Stable routing of tokens to heads plus the padded 128-row tile schedule the GEMM kernels read.
+size_t routing_workspace_bytes(int64_t T, int32_t M);
+// Writes sched, row_of_token[T] (padded row of each token, -1 if unroutable) and tok_of_row[T_pad]
+// (-1 for padding rows); optional role_offsets / role_perm outputs.
+int routing_launch(const int32_t* role_of_token, const int32_t* head_of_role, int32_t n_role,
+                   int32_t M, int64_t T, int64_t T_pad, Schedule* sched, int32_t* row_of_token,
+                   int32_t* tok_of_row, int32_t* role_offsets, int32_t* role_perm,
+                   int32_t* device_status, void* workspace, cudaStream_t st);
+// Hs[row] = H[tok_of_row[row]] (zeros for padding rows); rows of d bf16, 16-byte vectors.
+int gather_rows_launch(const void* H, int64_t ldH, const int32_t* tok_of_row, int64_t T_pad,
+                       int32_t d, void* Hs, cudaStream_t st);
+
+// ---- lm_head.cu -----------------------------------------------------------------------------
+struct LmHeadProblem {
+  const void* A_rows;        // bf16 [rows_total, d] rows in padded order (H itself when M == 1)
+  int64_t ldA;               // row stride of A_rows in elements
+  int64_t rows_bound;        // rows addressable through A_rows (T when M == 1, T_pad otherwise)
+  const void* W[ATGRPO_MAX_HEADS];
+  int32_t M, d, V;
+  int64_t T, T_pad;
+  const Schedule* sched;     // device
+  const int32_t* tok_of_row; // device, [T_pad]
+  const int32_t* target;     // device, [T] in token order
+  int32_t* device_status;
+  int32_t n_sm;
+};
+size_t lm_head_fwd_workspace_bytes(int64_t T_pad, int32_t d, int32_t V, int32_t n_sm);
+// lse[T], logp[T] in token order.
+int lm_head_fwd_launch(const LmHeadProblem& p, float* lse, float* logp, void* workspace,
+                       cudaStream_t st);
+size_t lm_head_bwd_workspace_bytes(int64_t T_pad, int32_t d, int32_t V, int32_t M, int32_t n_sm,
+                                   bool dH_direct);
+// coef[T] in token order (0 for tokens that pass no gradient); dH / dW as the C ABI documents.
+int lm_head_bwd_launch(const LmHeadProblem& p, const float* lse, const float* coef,
+                       const int32_t* row_of_token, const atgrpo_params& prm, void* dH,
+                       void* const* dW, void* workspace, cudaStream_t st);
+int device_sm_count(int* n_sm, int* cc_major);
+
+}  // namespace atgrpo

@@ -1,0 +1,691 @@
+// LM-head contractions of the policy loss (pi_theta of Eq. 2 and the gradient of Eq. 2) on the
+// sm_100a tensor cores.  One warp-specialised persistent kernel template serves four modes:
+//
+//   kFwd : z = H W_m^T tile by tile, streaming logsumexp and target-logit gather in the epilogue;
+//          the logits only ever exist in tensor memory.
+//   kDz  : the same contraction for one vocabulary chunk; the epilogue turns the logits into
+//          dZ = coef*(softmax - onehot) and writes them as bf16 into the chunk buffer.
+//   kDh  : dH_rows += dZ_chunk * W_m[chunk, :]          (A K-major, B MN-major)
+//   kDw  : dW_m[chunk, :] = dZ_chunk^T * H_rows          (A and B MN-major)
+//
+// CTA layout (192 threads): warp 0 = TMA producer, warp 1 = tcgen05.mma issuer and TMEM owner,
+// warps 2-5 = epilogue (one TMEM lane quarter each).  Tiles are 128 x 256 x 64 (bf16), operands
+// are staged by TMA into a 4-deep ring of 128-byte-swizzled shared-memory tiles, the fp32
+// accumulator is double buffered in the 512 TMEM columns so the epilogue of tile i overlaps the
+// MMAs of tile i+1.  Rows are addressed in the "padded row space": the tokens of policy m occupy
+// whole 128-row tiles starting at tile_begin[m], so no tile mixes two heads (grouped GEMM).
+#include <cuda_bf16.h>
+#include <cstring>
+#include "internal.h"
+#include "sm100.cuh"
+
+namespace atgrpo {
+namespace {
+using namespace sm100;
+
+constexpr int BM = 128, BN = 256, BK = 64;
+constexpr int kStages = 4;
+constexpr int kABytes = BM * BK * 2;               // 16 KiB
+constexpr int kBBytes = BN * BK * 2;               // 32 KiB
+constexpr int kStageBytes = kABytes + kBBytes;     // 48 KiB
+constexpr int kBoxBytes = 64 * 64 * 2;             // one 64 x 64 MN-major box, 8 KiB
+constexpr int kGemmThreads = 192;
+constexpr int kTmemCols = 512;
+constexpr int kSmemBytes = kStages * kStageBytes + 1024 /* alignment slack */ + 256 /* barriers */;
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+
+enum Mode { kFwd = 0, kDz = 1, kDh = 2, kDw = 3 };
+
+struct Maps {
+  CUtensorMap a;
+  CUtensorMap b[ATGRPO_MAX_HEADS];
+};
+
+struct GemmArgs {
+  const Schedule* sched;
+  const int32_t* tok_of_row;
+  const int32_t* target;
+  int32_t* status;
+  int V, d, M;
+  int64_t T_pad;
+  // kFwd / kDz: vocabulary tiling
+  int v_begin;            // first vocabulary row of this launch (0 for kFwd)
+  int n_vtiles;           // 256-wide vocabulary tiles in this launch
+  int tiles_per_chunk;    // kFwd: tiles one work item sweeps (1 for kDz)
+  int n_chunks;
+  float* part_m;          // kFwd out: running max (log2 domain) [n_chunks, T_pad]
+  float* part_s;          // kFwd out: sum of 2^(t - max)        [n_chunks, T_pad]
+  float* zt;              // kFwd out: target logit              [T_pad]
+  const float* lse;       // kDz in, token order
+  const float* coef;      // kDz in, token order
+  __nv_bfloat16* dz;      // kDz out / kDh, kDw in: [T_pad, vc]
+  int vc;                 // chunk buffer width (multiple of 256)
+  int vc_valid;           // vocabulary rows of this chunk that exist (<= vc)
+  // kDh
+  float* dh_acc;          // [T_pad, d] fp32
+  int first_chunk;
+  // kDw
+  void* dW[ATGRPO_MAX_HEADS];
+  int dw_bf16, dw_accumulate;
+};
+
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+struct Tile {
+  int head;
+  int row0;        // first padded row (kFwd/kDz/kDh) or first K row (kDw)
+  int rows_valid;  // valid token rows of this tile (kFwd/kDz/kDh)
+  int n0;          // first vocabulary row (kFwd/kDz, absolute) or first d column (kDh/kDw)
+  int v0;          // kDw: first vocabulary row of the tile inside the chunk buffer
+  int k_steps;
+  int chunk;       // kFwd: work-item chunk index
+  int nt_begin, nt_end;   // kFwd: tiles of the item
+};
+
+__device__ __forceinline__ int head_of_tile(const Schedule* s, int M, int mt) {
+  int h = 0;
+  for (int m = 1; m < M; ++m)
+    if (mt >= s->tile_begin[m]) h = m;
+  return h;
+}
+
+template <int kMode>
+__device__ __forceinline__ int total_items(const GemmArgs& g) {
+  const int n_mt = g.sched->tile_begin[g.M];
+  const int n_dt = (g.d + BN - 1) / BN;
+  if (kMode == kFwd || kMode == kDz) return n_mt * g.n_chunks;
+  if (kMode == kDh) return n_mt * n_dt;
+  return g.M * ((g.vc_valid + BM - 1) / BM) * n_dt;
+}
+
+template <int kMode>
+__device__ __forceinline__ Tile decode_item(const GemmArgs& g, int it) {
+  Tile t;
+  const Schedule* s = g.sched;
+  const int n_dt = (g.d + BN - 1) / BN;
+  t.v0 = 0, t.chunk = 0, t.nt_begin = 0, t.nt_end = 1;
+  if (kMode == kFwd || kMode == kDz) {
+    const int n_mt = s->tile_begin[g.M];
+    const int c = it / n_mt, mt = it - c * n_mt;       // row tiles fastest: co-resident CTAs
+    t.head = head_of_tile(s, g.M, mt);                 // sweep the same vocabulary slice
+    t.row0 = mt * BM;
+    t.rows_valid = min(BM, s->rows[t.head] - (mt - s->tile_begin[t.head]) * BM);
+    t.chunk = c;
+    t.nt_begin = c * g.tiles_per_chunk;
+    t.nt_end = min(t.nt_begin + g.tiles_per_chunk, g.n_vtiles);
+    t.n0 = g.v_begin + t.nt_begin * BN;
+    t.k_steps = (g.d + BK - 1) / BK;
+  } else if (kMode == kDh) {
+    const int mt = it / n_dt, dt = it - mt * n_dt;     // d tiles fastest: they share the dZ tile
+    t.head = head_of_tile(s, g.M, mt);
+    t.row0 = mt * BM;
+    t.rows_valid = min(BM, s->rows[t.head] - (mt - s->tile_begin[t.head]) * BM);
+    t.n0 = dt * BN;
+    t.k_steps = (g.vc_valid + BK - 1) / BK;
+  } else {
+    const int n_vt = (g.vc_valid + BM - 1) / BM;
+    const int dt = it % n_dt, rest = it / n_dt;
+    const int vt = rest % n_vt;
+    t.head = rest / n_vt;
+    t.row0 = s->tile_begin[t.head] * BM;
+    t.rows_valid = 0;
+    t.n0 = dt * BN;
+    t.v0 = vt * BM;
+    t.k_steps = (s->tile_begin[t.head + 1] - s->tile_begin[t.head]) * (BM / BK);
+  }
+  return t;
+}
+
+template <int kMode>
+__global__ void __launch_bounds__(kGemmThreads, 1)
+k_lm_head(const __grid_constant__ Maps maps, const GemmArgs g) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t bar_base = smem_base + kStages * kStageBytes;
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (kStages + s); };
+  auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * kStages + a); };
+  auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * kStages + 2 + a); };
+  uint8_t* smem_aligned = smem_raw + (smem_base - smem_u32(smem_raw));
+  volatile uint32_t* s_tmem = reinterpret_cast<volatile uint32_t*>(
+      smem_aligned + kStages * kStageBytes + 8 * (2 * kStages + 4));
+  volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(full_bar(s), 1);
+      mbar_init(empty_bar(s), 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(tfull_bar(a), 1);
+      mbar_init(tempty_bar(a), 128);
+    }
+    *s_abort = 0;
+    fence_mbar_init();
+    prefetch_tmap(&maps.a);
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32(const_cast<uint32_t*>(s_tmem)), kTmemCols);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *s_tmem;
+  const int n_items = total_items<kMode>(g);
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int it = blockIdx.x; ok && it < n_items; it += gridDim.x) {
+        const Tile t = decode_item<kMode>(g, it);
+        for (int nt = t.nt_begin; ok && nt < t.nt_end; ++nt) {
+          const int n0 = t.n0 + (nt - t.nt_begin) * BN;
+          for (int ks = 0; ks < t.k_steps; ++ks) {
+            if (!(ok = mbar_wait(empty_bar(stage), phase ^ 1u, s_abort, g.status))) break;
+            const uint32_t sa = smem_base + stage * kStageBytes, sb = sa + kABytes;
+            const uint32_t fb = full_bar(stage);
+            mbar_expect_tx(fb, kStageBytes);
+            if (kMode == kFwd || kMode == kDz) {
+              tma_load_2d(sa, &maps.a, ks * BK, t.row0, fb);
+              tma_load_2d(sb, &maps.b[t.head], ks * BK, n0, fb);
+            } else if (kMode == kDh) {
+              tma_load_2d(sa, &maps.a, ks * BK, t.row0, fb);
+#pragma unroll
+              for (int b = 0; b < 4; ++b)
+                tma_load_2d(sb + b * kBoxBytes, &maps.b[t.head], n0 + 64 * b, g.v_begin + ks * BK, fb);
+            } else {
+#pragma unroll
+              for (int b = 0; b < 2; ++b)
+                tma_load_2d(sa + b * kBoxBytes, &maps.a, t.v0 + 64 * b, t.row0 + ks * BK, fb);
+#pragma unroll
+              for (int b = 0; b < 4; ++b)
+                tma_load_2d(sb + b * kBoxBytes, &maps.b[0], n0 + 64 * b, t.row0 + ks * BK, fb);
+            }
+            if (++stage == kStages) stage = 0, phase ^= 1u;
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      constexpr bool a_mn = (kMode == kDw), b_mn = (kMode == kDh || kMode == kDw);
+      constexpr uint32_t idesc = idesc_bf16(BM, BN, a_mn, b_mn);
+      int stage = 0, acc = 0;
+      uint32_t phase = 0, acc_phase = 0;
+      bool ok = true;
+      for (int it = blockIdx.x; ok && it < n_items; it += gridDim.x) {
+        const Tile t = decode_item<kMode>(g, it);
+        if (t.k_steps == 0) continue;
+        for (int nt = t.nt_begin; ok && nt < t.nt_end; ++nt) {
+          if (!(ok = mbar_wait(tempty_bar(acc), acc_phase ^ 1u, s_abort, g.status))) break;
+          tc_fence_after();
+          const uint32_t d_tmem = tmem_base + acc * BN;
+          for (int ks = 0; ks < t.k_steps; ++ks) {
+            if (!(ok = mbar_wait(full_bar(stage), phase, s_abort, g.status))) break;
+            tc_fence_after();
+            const uint32_t sa = smem_base + stage * kStageBytes, sb = sa + kABytes;
+#pragma unroll
+            for (int kk = 0; kk < BK / 16; ++kk) {
+              const uint64_t ad = a_mn ? smem_desc(sa + kk * 2048, kBoxBytes, 1024)
+                                       : smem_desc(sa + kk * 32, 16, 1024);
+              const uint64_t bd = b_mn ? smem_desc(sb + kk * 2048, kBoxBytes, 1024)
+                                       : smem_desc(sb + kk * 32, 16, 1024);
+              umma_bf16(d_tmem, ad, bd, idesc, (ks | kk) != 0 ? 1u : 0u);
+            }
+            umma_commit(empty_bar(stage));        // frees the stage once these MMAs have read it
+            if (++stage == kStages) stage = 0, phase ^= 1u;
+          }
+          if (!ok) break;
+          umma_commit(tfull_bar(acc));            // accumulator complete
+          if (++acc == 2) acc = 0, acc_phase ^= 1u;
+        }
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue warps
+    const int quarter = warp & 3;
+    const int r_in_tile = quarter * 32 + lane;
+    const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16);
+    int acc = 0;
+    uint32_t acc_phase = 0;
+    bool ok = true;
+    for (int it = blockIdx.x; ok && it < n_items; it += gridDim.x) {
+      const Tile t = decode_item<kMode>(g, it);
+      uint32_t r[32];
+
+      if (kMode == kFwd || kMode == kDz) {
+        const int row = t.row0 + r_in_tile;
+        const bool valid = r_in_tile < t.rows_valid;
+        const int tok = valid ? g.tok_of_row[row] : -1;
+        int y = -1;
+        if (tok >= 0) {
+          y = g.target[tok];
+          if ((unsigned)y >= (unsigned)g.V) {
+            raise_status(g.status, ATGRPO_ERR_BAD_INDEX);
+            y = 0;
+          }
+        }
+        float m2 = -INFINITY, ssum = 0.f, zt = 0.f;
+        bool have_zt = false;
+        float lse2 = 0.f, cf = 0.f;
+        if (kMode == kDz && tok >= 0) lse2 = g.lse[tok] * kLog2e, cf = g.coef[tok];
+        for (int nt = t.nt_begin; ok && nt < t.nt_end; ++nt) {
+          const int n0 = t.n0 + (nt - t.nt_begin) * BN;
+          if (!(ok = mbar_wait(tfull_bar(acc), acc_phase, s_abort, g.status))) break;
+          tc_fence_after();
+          for (int c = 0; c < BN / 32; ++c) {
+            const int col0 = n0 + c * 32;
+            if (kMode == kFwd && col0 >= g.V) break;
+            __syncwarp();
+            tmem_ld32(lane_addr + acc * BN + c * 32, r);
+            tmem_ld_wait();
+            if (kMode == kFwd) {
+              if (y >= col0 && y < col0 + 32) {
+#pragma unroll
+                for (int i = 0; i < 32; ++i)
+                  if (col0 + i == y) zt = __uint_as_float(r[i]);
+                have_zt = true;
+              }
+              float tv[32];
+              float cmax = -INFINITY;
+              const bool ragged = col0 + 32 > g.V;
+#pragma unroll
+              for (int i = 0; i < 32; ++i) {
+                tv[i] = __uint_as_float(r[i]) * kLog2e;
+                if (ragged && col0 + i >= g.V) tv[i] = -INFINITY;
+                cmax = fmaxf(cmax, tv[i]);
+              }
+              const float nm = fmaxf(m2, cmax);
+              float add = 0.f;
+#pragma unroll
+              for (int i = 0; i < 32; ++i) add += ex2(tv[i] - nm);
+              ssum = ssum * ex2(m2 - nm) + add;
+              m2 = nm;
+            } else {
+              uint32_t packed[16];
+#pragma unroll
+              for (int i = 0; i < 32; i += 2) {
+                float g0 = 0.f, g1 = 0.f;
+                if (tok >= 0) {
+                  const float p0 = ex2(__uint_as_float(r[i]) * kLog2e - lse2);
+                  const float p1 = ex2(__uint_as_float(r[i + 1]) * kLog2e - lse2);
+                  g0 = (col0 + i < g.V) ? cf * (p0 - (col0 + i == y ? 1.f : 0.f)) : 0.f;
+                  g1 = (col0 + i + 1 < g.V) ? cf * (p1 - (col0 + i + 1 == y ? 1.f : 0.f)) : 0.f;
+                }
+                const __nv_bfloat162 h2 = __floats2bfloat162_rn(g0, g1);
+                packed[i >> 1] = *reinterpret_cast<const uint32_t*>(&h2);
+              }
+              uint4* dst = reinterpret_cast<uint4*>(g.dz + (size_t)row * g.vc + (col0 - g.v_begin));
+#pragma unroll
+              for (int q4 = 0; q4 < 4; ++q4)
+                dst[q4] = make_uint4(packed[4 * q4], packed[4 * q4 + 1], packed[4 * q4 + 2],
+                                     packed[4 * q4 + 3]);
+            }
+          }
+          tc_fence_before();
+          mbar_arrive(tempty_bar(acc));
+          if (++acc == 2) acc = 0, acc_phase ^= 1u;
+        }
+        if (kMode == kFwd && ok && tok >= 0) {
+          g.part_m[(size_t)t.chunk * g.T_pad + row] = m2;
+          g.part_s[(size_t)t.chunk * g.T_pad + row] = ssum;
+          if (have_zt) g.zt[row] = zt;
+        }
+      } else {
+        // kDh / kDw: plain accumulator write-out
+        const bool has_acc = t.k_steps > 0;
+        if (has_acc) {
+          if (!(ok = mbar_wait(tfull_bar(acc), acc_phase, s_abort, g.status))) break;
+          tc_fence_after();
+        }
+        bool valid;
+        size_t out_row;
+        if (kMode == kDh) {
+          valid = r_in_tile < t.rows_valid;
+          out_row = (size_t)(t.row0 + r_in_tile);
+        } else {
+          const int v = g.v_begin + t.v0 + r_in_tile;
+          valid = (t.v0 + r_in_tile < g.vc_valid) && v < g.V;
+          out_row = (size_t)v;
+        }
+        for (int c = 0; c < BN / 32; ++c) {
+          const int col0 = t.n0 + c * 32;
+          if (col0 >= g.d) break;
+          if (has_acc) {
+            __syncwarp();
+            tmem_ld32(lane_addr + acc * BN + c * 32, r);
+            tmem_ld_wait();
+          } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) r[i] = 0u;
+          }
+          if (!valid) continue;
+          if (kMode == kDh || !g.dw_bf16) {
+            float* dst = (kMode == kDh ? g.dh_acc : static_cast<float*>(g.dW[t.head])) +
+                         out_row * g.d + col0;
+            const bool add = kMode == kDh ? !g.first_chunk : (g.dw_accumulate != 0);
+#pragma unroll
+            for (int q4 = 0; q4 < 8; ++q4) {
+              if (col0 + 4 * q4 < g.d) {
+                float4 v4 = make_float4(__uint_as_float(r[4 * q4]), __uint_as_float(r[4 * q4 + 1]),
+                                        __uint_as_float(r[4 * q4 + 2]), __uint_as_float(r[4 * q4 + 3]));
+                float4* p4 = reinterpret_cast<float4*>(dst) + q4;
+                if (add) {
+                  const float4 o = *p4;
+                  v4.x += o.x, v4.y += o.y, v4.z += o.z, v4.w += o.w;
+                }
+                *p4 = v4;
+              }
+            }
+          } else {
+            __nv_bfloat16* dst = static_cast<__nv_bfloat16*>(g.dW[t.head]) + out_row * g.d + col0;
+#pragma unroll
+            for (int q8 = 0; q8 < 4; ++q8) {
+              if (col0 + 8 * q8 < g.d) {
+                uint4* p4 = reinterpret_cast<uint4*>(dst) + q8;
+                float f[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) f[i] = __uint_as_float(r[8 * q8 + i]);
+                if (g.dw_accumulate) {
+                  const uint4 o = *p4;
+                  const __nv_bfloat162* oh = reinterpret_cast<const __nv_bfloat162*>(&o);
+#pragma unroll
+                  for (int i = 0; i < 4; ++i) {
+                    const float2 of = __bfloat1622float2(oh[i]);
+                    f[2 * i] += of.x, f[2 * i + 1] += of.y;
+                  }
+                }
+                uint4 w;
+                __nv_bfloat162* wh = reinterpret_cast<__nv_bfloat162*>(&w);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) wh[i] = __floats2bfloat162_rn(f[2 * i], f[2 * i + 1]);
+                *p4 = w;
+              }
+            }
+          }
+        }
+        if (has_acc) {
+          tc_fence_before();
+          mbar_arrive(tempty_bar(acc));
+          if (++acc == 2) acc = 0, acc_phase ^= 1u;
+        }
+      }
+    }
+  }
+
+  // ---------------------------------------------------------------------- teardown
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    if (*s_abort) {
+      // a wait gave up: let the loads this CTA may still have in flight land before its shared
+      // memory is handed to the next CTA
+      for (int i = 0; i < 64; ++i) __nanosleep(2000);
+    }
+    __syncwarp();
+    tc_fence_after();
+    tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+// Combines the per-chunk (max, sum) pairs into lse and logp, in token order.
+__global__ void __launch_bounds__(256)
+k_lse_combine(const Schedule* sched, int M, const int32_t* tok_of_row, int64_t T_pad, int n_chunks,
+              const float* part_m, const float* part_s, const float* zt, float* lse, float* logp) {
+  const int64_t rows = (int64_t)sched->tile_begin[M] * BM;
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  for (int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; p < rows; p += stride) {
+    const int tok = tok_of_row[p];
+    if (tok < 0) continue;
+    float mx = -INFINITY;
+    for (int c = 0; c < n_chunks; ++c) mx = fmaxf(mx, part_m[(size_t)c * T_pad + p]);
+    float s = 0.f;
+    for (int c = 0; c < n_chunks; ++c)
+      s += part_s[(size_t)c * T_pad + p] * exp2f(part_m[(size_t)c * T_pad + p] - mx);
+    const float l = (mx + log2f(s)) * kLn2;
+    lse[tok] = l;
+    logp[tok] = zt[p] - l;
+  }
+}
+
+template <bool kBf16>
+__global__ void __launch_bounds__(256)
+k_dh_finalize(const float* __restrict__ acc, const int32_t* __restrict__ row_of_token, int64_t T,
+              int d, void* __restrict__ out) {
+  const int d4 = d / 4;
+  const int64_t total = T * d4;
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += stride) {
+    const int64_t tok = i / d4;
+    const int c = (int)(i - tok * d4);
+    const int row = row_of_token[tok];
+    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (row >= 0) v = reinterpret_cast<const float4*>(acc + (size_t)row * d)[c];
+    if (kBf16) {
+      uint2 w;
+      __nv_bfloat162* wh = reinterpret_cast<__nv_bfloat162*>(&w);
+      wh[0] = __floats2bfloat162_rn(v.x, v.y);
+      wh[1] = __floats2bfloat162_rn(v.z, v.w);
+      reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(out) + (size_t)tok * d)[c] = w;
+    } else {
+      reinterpret_cast<float4*>(static_cast<float*>(out) + (size_t)tok * d)[c] = v;
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------ host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
+                                  const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                  const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (fn == nullptr) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+// bf16 matrix [outer, inner] with row stride ld elements; 128-byte swizzled boxes.
+bool make_map(CUtensorMap* m, const void* base, int64_t inner, int64_t outer, int64_t ld,
+              int box_inner, int box_outer) {
+  EncodeTiledFn fn = encode_fn();
+  if (fn == nullptr) return false;
+  const cuuint64_t dims[2] = {(cuuint64_t)inner, (cuuint64_t)(outer > 0 ? outer : 1)};
+  const cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
+  const cuuint32_t box[2] = {(cuuint32_t)box_inner, (cuuint32_t)box_outer};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box,
+            estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// Number of vocabulary chunks of the forward sweep: enough work items to fill the SMs evenly.
+int fwd_chunks(int64_t n_mt, int n_vt, int n_sm) {
+  int best = 1;
+  double best_eff = -1.0;
+  const int cmax = n_vt < 64 ? n_vt : 64;
+  for (int c = 1; c <= cmax; ++c) {
+    const int64_t per = (n_vt + c - 1) / c;
+    const int64_t real_c = (n_vt + per - 1) / per;
+    if (real_c != c) continue;
+    const int64_t items = n_mt * c;
+    const int64_t waves = (items + n_sm - 1) / n_sm;
+    const double eff = (double)(n_mt * (int64_t)n_vt) / ((double)waves * n_sm * per);
+    if (eff > best_eff + 1e-9) best_eff = eff, best = c;
+  }
+  return best;
+}
+
+// Width of the dZ chunk buffer: as wide as a 256 MiB buffer allows.
+int bwd_chunk_width(int64_t T_pad, int V) {
+  const int64_t budget = 256ll << 20;
+  int64_t vc = budget / (T_pad * 2) / BN * BN;
+  const int64_t vmax = (int64_t)(V + BN - 1) / BN * BN;
+  if (vc < BN) vc = BN;
+  if (vc > vmax) vc = vmax;
+  return (int)vc;
+}
+
+struct FwdPlan { size_t part_m, part_s, zt, total; int n_chunks, tiles_per_chunk, n_vt; };
+FwdPlan fwd_plan(int64_t T_pad, int V, int n_sm) {
+  FwdPlan p;
+  p.n_vt = (V + BN - 1) / BN;
+  const int64_t n_mt = T_pad / BM;
+  p.n_chunks = fwd_chunks(n_mt > 0 ? n_mt : 1, p.n_vt, n_sm);
+  p.tiles_per_chunk = (p.n_vt + p.n_chunks - 1) / p.n_chunks;
+  Carver c(nullptr);
+  p.part_m = c.off; c.take<float>((size_t)p.n_chunks * T_pad);
+  p.part_s = c.off; c.take<float>((size_t)p.n_chunks * T_pad);
+  p.zt = c.off; c.take<float>((size_t)T_pad);
+  p.total = c.off;
+  return p;
+}
+
+struct BwdPlan { size_t dz, dh_acc, total; int vc; };
+BwdPlan bwd_plan(int64_t T_pad, int d, int V, bool dH_direct) {
+  BwdPlan p;
+  p.vc = bwd_chunk_width(T_pad, V);
+  Carver c(nullptr);
+  p.dz = c.off; c.take<__nv_bfloat16>((size_t)T_pad * p.vc);
+  p.dh_acc = c.off;
+  if (!dH_direct) c.take<float>((size_t)T_pad * d);
+  p.total = c.off;
+  return p;
+}
+
+template <int kMode>
+int launch_gemm(const Maps& maps, const GemmArgs& g, int grid, cudaStream_t st) {
+  if (cudaFuncSetAttribute(k_lm_head<kMode>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           kSmemBytes) != cudaSuccess)
+    return ATGRPO_ERR_CUDA;
+  k_lm_head<kMode><<<grid, kGemmThreads, kSmemBytes, st>>>(maps, g);
+  return launch_ok();
+}
+
+GemmArgs base_args(const LmHeadProblem& p) {
+  GemmArgs g;
+  memset(&g, 0, sizeof(g));
+  g.sched = p.sched, g.tok_of_row = p.tok_of_row, g.target = p.target, g.status = p.device_status;
+  g.V = p.V, g.d = p.d, g.M = p.M, g.T_pad = p.T_pad;
+  return g;
+}
+
+}  // namespace
+
+int device_sm_count(int* n_sm, int* cc_major) {
+  int dev = 0;
+  ATGRPO_CUDA_OK(cudaGetDevice(&dev));
+  ATGRPO_CUDA_OK(cudaDeviceGetAttribute(n_sm, cudaDevAttrMultiProcessorCount, dev));
+  ATGRPO_CUDA_OK(cudaDeviceGetAttribute(cc_major, cudaDevAttrComputeCapabilityMajor, dev));
+  return ATGRPO_OK;
+}
+
+size_t lm_head_fwd_workspace_bytes(int64_t T_pad, int32_t d, int32_t V, int32_t n_sm) {
+  (void)d;
+  return fwd_plan(T_pad, V, n_sm).total;
+}
+
+int lm_head_fwd_launch(const LmHeadProblem& p, float* lse, float* logp, void* workspace,
+                       cudaStream_t st) {
+  const FwdPlan pl = fwd_plan(p.T_pad, p.V, p.n_sm);
+  char* ws = static_cast<char*>(workspace);
+  Maps maps;
+  if (!make_map(&maps.a, p.A_rows, p.d, p.rows_bound, p.ldA, BK, BM)) return ATGRPO_ERR_CUDA;
+  for (int m = 0; m < p.M; ++m)
+    if (!make_map(&maps.b[m], p.W[m], p.d, p.V, p.d, BK, BN)) return ATGRPO_ERR_CUDA;
+  GemmArgs g = base_args(p);
+  g.v_begin = 0, g.n_vtiles = pl.n_vt, g.tiles_per_chunk = pl.tiles_per_chunk, g.n_chunks = pl.n_chunks;
+  g.part_m = reinterpret_cast<float*>(ws + pl.part_m);
+  g.part_s = reinterpret_cast<float*>(ws + pl.part_s);
+  g.zt = reinterpret_cast<float*>(ws + pl.zt);
+  const int64_t items = (p.T_pad / BM) * pl.n_chunks;
+  const int grid = (int)(items < p.n_sm ? (items > 0 ? items : 1) : p.n_sm);
+  int rc = launch_gemm<kFwd>(maps, g, grid, st);
+  if (rc != ATGRPO_OK) return rc;
+  const int cgrid = (int)((p.T_pad + 255) / 256 > 0 ? (p.T_pad + 255) / 256 : 1);
+  k_lse_combine<<<cgrid, 256, 0, st>>>(p.sched, p.M, p.tok_of_row, p.T_pad, pl.n_chunks, g.part_m,
+                                       g.part_s, g.zt, lse, logp);
+  return launch_ok();
+}
+
+size_t lm_head_bwd_workspace_bytes(int64_t T_pad, int32_t d, int32_t V, int32_t M, int32_t n_sm,
+                                   bool dH_direct) {
+  (void)M, (void)n_sm;
+  return bwd_plan(T_pad, d, V, dH_direct).total;
+}
+
+int lm_head_bwd_launch(const LmHeadProblem& p, const float* lse, const float* coef,
+                       const int32_t* row_of_token, const atgrpo_params& prm, void* dH,
+                       void* const* dW, void* workspace, cudaStream_t st) {
+  const bool dH_direct = p.M == 1 && prm.dH_dtype == ATGRPO_F32;
+  const BwdPlan pl = bwd_plan(p.T_pad, p.d, p.V, dH_direct);
+  char* ws = static_cast<char*>(workspace);
+  __nv_bfloat16* dz = reinterpret_cast<__nv_bfloat16*>(ws + pl.dz);
+  float* dh_acc = dH_direct ? static_cast<float*>(dH) : reinterpret_cast<float*>(ws + pl.dh_acc);
+
+  Maps m_dz, m_dh, m_dw;
+  if (!make_map(&m_dz.a, p.A_rows, p.d, p.rows_bound, p.ldA, BK, BM)) return ATGRPO_ERR_CUDA;
+  if (!make_map(&m_dh.a, dz, pl.vc, p.T_pad, pl.vc, BK, BM)) return ATGRPO_ERR_CUDA;
+  if (!make_map(&m_dw.a, dz, pl.vc, p.T_pad, pl.vc, 64, 64)) return ATGRPO_ERR_CUDA;
+  if (!make_map(&m_dw.b[0], p.A_rows, p.d, p.rows_bound, p.ldA, 64, 64)) return ATGRPO_ERR_CUDA;
+  for (int m = 0; m < p.M; ++m) {
+    if (!make_map(&m_dz.b[m], p.W[m], p.d, p.V, p.d, BK, BN)) return ATGRPO_ERR_CUDA;
+    if (!make_map(&m_dh.b[m], p.W[m], p.d, p.V, p.d, 64, 64)) return ATGRPO_ERR_CUDA;
+  }
+  const int64_t n_mt = p.T_pad / BM;
+  const int n_dt = (p.d + BN - 1) / BN;
+  int chunk = 0;
+  for (int v_begin = 0; v_begin < p.V; v_begin += pl.vc, ++chunk) {
+    GemmArgs g = base_args(p);
+    g.v_begin = v_begin;
+    g.vc = pl.vc;
+    g.vc_valid = p.V - v_begin < pl.vc ? p.V - v_begin : pl.vc;
+    g.n_vtiles = (g.vc_valid + BN - 1) / BN;
+    g.tiles_per_chunk = 1;
+    g.n_chunks = g.n_vtiles;
+    g.lse = lse, g.coef = coef, g.dz = dz;
+    g.dh_acc = dh_acc, g.first_chunk = chunk == 0;
+    for (int m = 0; m < p.M; ++m) g.dW[m] = dW[m];
+    g.dw_bf16 = prm.dW_dtype == ATGRPO_BF16, g.dw_accumulate = prm.accumulate_dW;
+    auto grid_for = [&](int64_t items) {
+      return (int)(items < p.n_sm ? (items > 0 ? items : 1) : p.n_sm);
+    };
+    int rc = launch_gemm<kDz>(m_dz, g, grid_for(n_mt * g.n_vtiles), st);
+    if (rc != ATGRPO_OK) return rc;
+    rc = launch_gemm<kDh>(m_dh, g, grid_for(n_mt * n_dt), st);
+    if (rc != ATGRPO_OK) return rc;
+    rc = launch_gemm<kDw>(m_dw, g, grid_for((int64_t)p.M * ((g.vc_valid + BM - 1) / BM) * n_dt), st);
+    if (rc != ATGRPO_OK) return rc;
+  }
+  if (!dH_direct) {
+    const int64_t total = p.T * (p.d / 4);
+    int64_t grid = (total + 255) / 256;
+    if (grid > 148 * 16) grid = 148 * 16;
+    if (grid < 1) grid = 1;
+    if (prm.dH_dtype == ATGRPO_BF16)
+      k_dh_finalize<true><<<(int)grid, 256, 0, st>>>(dh_acc, row_of_token, p.T, p.d, dH);
+    else
+      k_dh_finalize<false><<<(int)grid, 256, 0, st>>>(dh_acc, row_of_token, p.T, p.d, dH);
+  }
+  return launch_ok();
+}
+
+}  // namespace atgrpo
