@@ -1,0 +1,373 @@
+#!/usr/bin/env python
+"""Benchmark of the AT-GRPO policy-update hot path on B200.
+
+One step = grouped advantages (Eq. 1) -> policy loss forward through the LM head (Eq. 2) ->
+backward to dH and dW, on one synthetic on-policy batch.  Default workload: the
+Qwen3-1.7B-shaped single-policy head (d=2048, V=151936, ~16K response tokens).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+Prints ONE JSON line (rank 0).  With --impl reference the fp64 CPU oracle is timed instead, on a
+bounded token sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2510_11062_b200 import workloads as WL  # noqa: E402
+
+METRIC = "fused AT-GRPO loss fwd+bwd tokens/sec"
+UNIT = "tokens/s"
+CPU_SAMPLE_TOKENS = 128
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return dict(hbm_gbs=p["hbm_gbs"], bf16_burst=p["bf16_tflops"],
+                    bf16_sustained=p["bf16_tflops_sustained"], source="measured")
+    return dict(hbm_gbs=6650.0, bf16_burst=1590.0, bf16_sustained=1400.0, source="fallback")
+
+
+# ------------------------------------------------------------------------------- CPU oracle leg
+def oracle_sample_seconds(batch, n_tokens):
+    """Times the oracle, as it stands, on the first n_tokens tokens of the batch (full vocabulary):
+    advantages for the whole batch, log-probs, loss and gradients for the sample."""
+    import numpy as np
+    from oracle import atgrpo_oracle as O
+    spec = batch["spec"]
+    t0 = time.perf_counter()
+    key = O.group_key(batch["env_id"], batch["role_id"], batch["turn_id"], spec.n_env, spec.n_role, spec.n_turn)
+    adv, _, _ = O.group_advantages(batch["rewards"], key, spec.n_env * spec.n_role * spec.n_turn)
+    sl = slice(0, n_tokens)
+    if spec.n_heads > 1:
+        head, _, _ = O.route_tokens(batch["role_of_token"][sl], batch["head_of_role"], spec.n_heads)
+    else:
+        head = np.zeros(n_tokens, dtype=np.int64)
+    H, y, resp = batch["H"][sl], batch["target"][sl], batch["resp_of_token"][sl]
+    logp = np.zeros(n_tokens)
+    for m in range(spec.n_heads):
+        sel = np.nonzero(head == m)[0]
+        if sel.size:
+            _, logp[sel], _ = O.token_logprobs(H[sel], batch["W"][m], y[sel])
+    old = logp + 0.05 * np.sin(np.arange(n_tokens))          # any fixed perturbation
+    O.policy_loss(logp, old, adv, resp, head, spec.n_heads)
+    O.policy_loss_grads(H, batch["W"], y, old, adv, resp, head)
+    return time.perf_counter() - t0
+
+
+def blas_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        return max([p.get("num_threads", 1) for p in threadpool_info()] or [os.cpu_count()])
+    except Exception:
+        return os.cpu_count()
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    spec = WL.SPECS[args.workload]
+    batch = WL.make_rollout(spec)
+    n = min(CPU_SAMPLE_TOKENS, batch["T"])
+    times = []
+    for i in range(args.warmup + args.steps):
+        dt = oracle_sample_seconds(batch, n)
+        if i >= args.warmup:
+            times.append(dt)
+    total = sum(times)
+    value = n * len(times) / total
+    sample = f"first {n} tokens of the batch, full vocabulary, fwd+bwd, plus advantages of all {batch['R']} candidates"
+    line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=args.gpus, steps=args.steps, warmup=args.warmup,
+                ms_per_step=1e3 * total / len(times), higher_is_better=True, scaling="weak", vs_baseline=None,
+                dtype="f64", data="synthetic", impl="reference",
+                config=dict(workload=spec.name, d=spec.d, V=spec.V, tokens=batch["T"], heads=spec.n_heads),
+                cpu_baseline=dict(value=value, unit=UNIT, cores=blas_threads(), kind="oracle", sample=sample),
+                e2e=dict(value=value, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0))
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------------------- clocks
+class ClockSampler:
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.tmp = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={gpu_index}", f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=self.tmp, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = dict(sm_mhz=None, sm_max_mhz=None, reasons=[])
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.tmp.flush()
+        self.tmp.seek(0)
+        sm, smax, power, reasons = [], [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.tmp.read().splitlines():
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 8:
+                continue
+            try:
+                sm.append(float(f[1])), smax.append(float(f[2])), power.append(float(f[3]))
+            except ValueError:
+                continue
+            for nm, v in zip(names, f[4:8]):
+                if v.lower().startswith("active"):
+                    reasons.add(nm)
+        self.tmp.close()
+        os.unlink(self.tmp.name)
+        if sm:
+            out = dict(sm_mhz=statistics.median(sm), sm_max_mhz=max(smax), power_w_max=max(power),
+                       samples=len(sm), reasons=sorted(reasons))
+        return out
+
+
+# ------------------------------------------------------------------------------- GPU leg
+class Runner:
+    """Device-resident state of one rank: inputs, outputs, workspaces; step() enqueues the path."""
+
+    def __init__(self, batch, device, A):
+        self.A = A
+        self.dev = device
+        spec = self.spec = batch["spec"]
+        self.T, self.R, self.M = batch["T"], batch["R"], spec.n_heads
+        f32, i32 = torch.float32, torch.int32
+        self.host = {k: batch[k].pin_memory() for k in
+                     ("rewards", "env_id", "role_id", "turn_id", "H", "target", "resp_of_token", "role_of_token")}
+        self.d = {k: v.to(device) for k, v in self.host.items()}
+        self.W = [w.to(device) for w in batch["W"]]
+        self.head_of_role = batch["head_of_role"].to(device) if self.M > 1 else None
+        self.role_of_token = self.d["role_of_token"] if self.M > 1 else None
+        self.prm = A.Params()
+        G = spec.n_env * spec.n_role * spec.n_turn
+        T, V, dm, M = self.T, spec.V, spec.d, self.M
+        self.adv = torch.zeros(self.R, dtype=f32, device=device)
+        self.loss = torch.zeros(M, dtype=f32, device=device)
+        self.logp = torch.zeros(T, dtype=f32, device=device)
+        self.lse = torch.zeros(T, dtype=f32, device=device)
+        self.old_logp = torch.zeros(T, dtype=f32, device=device)
+        self.dH = torch.zeros(T, dm, dtype=torch.bfloat16, device=device)
+        self.dW = [torch.zeros(V, dm, dtype=f32, device=device) for _ in range(M)]
+        self.grad_loss = None
+        self.status = A.new_status(device)
+        self.ws_adv = A.workspace(A.atgrpo_group_advantages_workspace_bytes(self.R, G), device)
+        self.ws_fwd = A.workspace(A.atgrpo_policy_loss_workspace_bytes(T, dm, V, M, False), device)
+        self.ws_bwd = A.workspace(A.atgrpo_policy_loss_workspace_bytes(T, dm, V, M, True), device)
+        self.launches = 5 + A.atgrpo_policy_loss_launch_count(T, dm, V, M, False) + \
+            A.atgrpo_policy_loss_launch_count(T, dm, V, M, True)
+        self.host_loss = torch.zeros(M, dtype=f32).pin_memory()
+        self.h2d_bytes = sum(self.host[k].numel() * self.host[k].element_size() for k in self.host
+                             if k != "role_of_token" or M > 1) + T * 4
+        self.host["old_logp"] = None
+
+    def advantages(self):
+        s, d = self.spec, self.d
+        self.A.atgrpo_group_advantages(d["rewards"], d["env_id"], d["role_id"], d["turn_id"], s.n_env, s.n_role,
+                                       s.n_turn, self.prm, self.adv, device_status=self.status, workspace=self.ws_adv)
+
+    def forward(self):
+        d = self.d
+        self.A.atgrpo_policy_loss_fwd(d["H"], self.W, d["target"], self.role_of_token, self.head_of_role,
+                                      d["resp_of_token"], self.adv, self.old_logp, self.prm, self.loss, self.logp,
+                                      self.lse, device_status=self.status, workspace=self.ws_fwd)
+
+    def backward(self):
+        d = self.d
+        self.A.atgrpo_policy_loss_bwd(d["H"], self.W, d["target"], self.role_of_token, self.head_of_role,
+                                      d["resp_of_token"], self.adv, self.old_logp, self.logp, self.lse,
+                                      self.grad_loss, self.prm, self.dH, self.dW, device_status=self.status,
+                                      workspace=self.ws_bwd)
+
+    def make_old_logp(self):
+        """Perf-only: old_logp = the library's own logp + N(0, 0.05) (parity runs use the oracle's)."""
+        self.advantages()
+        self.forward()
+        torch.cuda.synchronize()
+        old = WL.make_old_logp(self.logp.cpu(), self.spec.seed + 100, 0.05)
+        self.host["old_logp"] = old.pin_memory()
+        self.old_logp.copy_(self.host["old_logp"])
+
+    def upload(self):
+        for k, v in self.host.items():
+            if k == "old_logp":
+                self.old_logp.copy_(v, non_blocking=True)
+            elif k != "role_of_token" or self.M > 1:
+                self.d[k].copy_(v, non_blocking=True)
+
+
+def run_ours(args):
+    from paper_2510_11062_b200 import atgrpo as A
+    from paper_2510_11062_b200 import data_parallel as DP
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    A.lib()                                    # fail loudly if libatgrpo.so is missing
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    spec = WL.SPECS[args.workload]
+    if world > 1:                              # weak scaling: every rank draws its own batch
+        spec = WL.RolloutSpec(**{**spec.__dict__, "seed": spec.seed + 1000 * rank})
+    batch = WL.make_rollout(spec)
+
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        n = min(CPU_SAMPLE_TOKENS, batch["T"])
+        dt = oracle_sample_seconds(batch, n)
+        cpu_baseline = dict(value=n / dt, unit=UNIT, cores=blas_threads(), kind="oracle",
+                            sample=f"first {n} tokens, full vocabulary, fwd+bwd, plus advantages of all "
+                                   f"{batch['R']} candidates; {dt:.1f} s")
+
+    r = Runner(batch, dev, A)
+    r.make_old_logp()
+    if world > 1:
+        heads = batch["head_of_role"].long()[batch["role_of_token"].long()]
+        counts = torch.bincount(heads, minlength=r.M).to(dev)
+        r.grad_loss, _ = DP.token_mean_scale(counts)
+
+    def step():
+        r.advantages()
+        r.forward()
+        r.backward()
+        if world > 1:
+            DP.allreduce_gradients(r.dW)
+
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    if world > 1:
+        torch.distributed.barrier()
+
+    # ---- timed region: device-resident inputs
+    sampler = ClockSampler(local) if rank == 0 else None
+    marks = [[ev() for _ in range(4)] for _ in range(args.steps)]
+    torch.cuda.synchronize()
+    t_start, t_end = ev(), ev()
+    t_start.record()
+    for k in range(args.steps):
+        marks[k][0].record()
+        r.advantages()
+        marks[k][1].record()
+        r.forward()
+        marks[k][2].record()
+        r.backward()
+        if world > 1:
+            DP.allreduce_gradients(r.dW)
+        marks[k][3].record()
+    t_end.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop() if sampler else None
+    if world > 1:
+        torch.distributed.barrier()
+    ms_total = t_start.elapsed_time(t_end)
+    status = int(r.status.item())
+
+    # ---- end to end: per-step inputs start in pinned host memory, the loss is read back
+    for _ in range(2):
+        r.upload(); step()
+    torch.cuda.synchronize()
+    e_start, e_end = ev(), ev()
+    e_start.record()
+    for _ in range(args.steps):
+        r.upload()
+        step()
+        r.host_loss.copy_(r.loss, non_blocking=True)
+    e_end.record()
+    torch.cuda.synchronize()
+    ms_e2e = e_start.elapsed_time(e_end)
+
+    t = torch.tensor([ms_total, ms_e2e], dtype=torch.float64, device=dev)
+    tokens = torch.tensor([float(r.T)], dtype=torch.float64, device=dev)
+    if world > 1:
+        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+        torch.distributed.all_reduce(tokens)
+    ms_total, ms_e2e = t.tolist()
+    tokens_all = tokens.item()
+    if rank != 0:
+        return
+    if status != 0:
+        raise SystemExit(f"device status {status}: {A.status_string(status)}")
+
+    adv_ms = statistics.mean(m[0].elapsed_time(m[1]) for m in marks)
+    fwd_ms = statistics.mean(m[1].elapsed_time(m[2]) for m in marks)
+    bwd_ms = statistics.mean(m[2].elapsed_time(m[3]) for m in marks)
+    peaks = measured_peaks()
+    pass_flops = 2.0 * r.T * spec.V * spec.d                  # one T x V x d contraction
+    fwd_tf = pass_flops / (fwd_ms * 1e-3) / 1e12
+    bwd_tf = 3.0 * pass_flops / (bwd_ms * 1e-3) / 1e12      # executed: logits recompute + dH + dW
+    value = tokens_all * args.steps / (ms_total * 1e-3)
+    line = dict(
+        metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=max(args.warmup, 3),
+        ms_per_step=ms_total / args.steps, higher_is_better=True, scaling="weak", vs_baseline=None,
+        dtype="bf16", data="synthetic",
+        config=dict(workload=spec.name, d=spec.d, V=spec.V, heads=spec.n_heads, tokens_per_gpu=r.T,
+                    responses_per_gpu=r.R, parallelism=f"dp{world}",
+                    l2="inputs larger than L2 (W alone is %.0f MB)" % (spec.V * spec.d * 2 / 1e6),
+                    old_logp="library logp + N(0,0.05) (perf-only input)"),
+        gpu_launches=(r.launches) * args.steps,
+        phases_ms=dict(advantages=adv_ms, forward=fwd_ms, backward=bwd_ms),
+        roofline=dict(bound="tensor", kernel="k_lm_head<kFwd> (forward call: routing + logits/logsumexp sweep "
+                      "+ combine + Eq. 2 reduction)", achieved=fwd_tf, peak=peaks["bf16_sustained"],
+                      unit="TFLOP/s", frac=fwd_tf / peaks["bf16_sustained"], traffic=None,
+                      peak_source=peaks["source"] + " sustained cuBLAS bf16",
+                      flops_per_launch=pass_flops,
+                      backward_executed_tflops=bwd_tf, backward_frac=bwd_tf / peaks["bf16_sustained"],
+                      fwd_bwd_algorithmic_tflops=3.0 * pass_flops / ((fwd_ms + bwd_ms) * 1e-3) / 1e12,
+                      fwd_bwd_executed_tflops=4.0 * pass_flops / ((fwd_ms + bwd_ms) * 1e-3) / 1e12,
+                      frac_of_nominal_2250=4.0 * pass_flops / ((fwd_ms + bwd_ms) * 1e-3) / 1e12 / 2250.0),
+        e2e=dict(value=tokens_all * args.steps / (ms_e2e * 1e-3), unit=UNIT,
+                 h2d_bytes_per_step=r.h2d_bytes, d2h_bytes_per_step=r.M * 4),
+        clocks=clocks, cpu_baseline=cpu_baseline)
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="qwen3_1p7b", choices=sorted(WL.SPECS))
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

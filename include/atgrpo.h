@@ -135,10 +135,17 @@ int atgrpo_clipped_loss(
  * Optional: role_offsets[M+1], role_perm[T] = stable routing of tokens to policies (tokens of
  * policy m in ascending token index); clip_counts[M*2] (int64) as in atgrpo_clipped_loss.
  * Requirements: d % 8 == 0, d >= 64, V >= 1, 1 <= M <= ATGRPO_MAX_HEADS, T < 2^31 - 2^16.
- * Out-of-range target / role / head / response index: ATGRPO_ERR_BAD_INDEX in *device_status;
- * such a token gets logp = lse = 0 and contributes nothing.
+ * Out-of-range indices raise ATGRPO_ERR_BAD_INDEX in *device_status and stay in bounds: a bad
+ * target is read as token 0; a token whose role or head is out of range belongs to no policy
+ * (its logp and lse are left untouched, it enters no loss); a bad response index counts the
+ * token with A = 0.
  * ------------------------------------------------------------------------------------------ */
 size_t atgrpo_policy_loss_workspace_bytes(int64_t T, int32_t d, int32_t V, int32_t M, int32_t is_bwd);
+
+/* Number of kernels one forward (is_bwd = 0) or backward (is_bwd = 1) call enqueues for these
+ * sizes on the current device (memsets not counted).  A bookkeeping query with no counterpart in
+ * the paper: callers use it to size CUDA graphs and to report launch counts. */
+int32_t atgrpo_policy_loss_launch_count(int64_t T, int32_t d, int32_t V, int32_t M, int32_t is_bwd);
 
 int atgrpo_policy_loss_fwd(
     const void* H, int64_t ldH, const void* const* W /* host array */, int32_t M,

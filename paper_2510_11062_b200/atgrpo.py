@@ -24,7 +24,8 @@ EXPORTS = (
     "atgrpo_status_string",
     "atgrpo_group_advantages_workspace_bytes", "atgrpo_group_advantages",
     "atgrpo_clipped_loss_workspace_bytes", "atgrpo_clipped_loss",
-    "atgrpo_policy_loss_workspace_bytes", "atgrpo_policy_loss_fwd", "atgrpo_policy_loss_bwd",
+    "atgrpo_policy_loss_workspace_bytes", "atgrpo_policy_loss_launch_count",
+    "atgrpo_policy_loss_fwd", "atgrpo_policy_loss_bwd",
 )
 
 
@@ -79,6 +80,8 @@ def lib() -> ctypes.CDLL:
         L.atgrpo_clipped_loss.argtypes = [vp, vp, vp, vp, i64, i64, pp, vp, vp, vp, vp, vp, sz, vp]
         L.atgrpo_policy_loss_workspace_bytes.restype = sz
         L.atgrpo_policy_loss_workspace_bytes.argtypes = [i64, i32, i32, i32, i32]
+        L.atgrpo_policy_loss_launch_count.restype = i32
+        L.atgrpo_policy_loss_launch_count.argtypes = [i64, i32, i32, i32, i32]
         L.atgrpo_policy_loss_fwd.restype = ctypes.c_int
         L.atgrpo_policy_loss_fwd.argtypes = [vp, i64, ctypes.POINTER(vp), i32, vp, vp, vp, i32, vp, vp,
                                              i64, vp, i64, i32, i32, pp, vp, vp, vp, vp, vp, vp, vp,
@@ -167,6 +170,10 @@ def atgrpo_clipped_loss(logp, old_logp, resp_of_token, adv, params: Params, loss
 
 def atgrpo_policy_loss_workspace_bytes(T: int, d: int, V: int, M: int, is_bwd: bool) -> int:
     return int(lib().atgrpo_policy_loss_workspace_bytes(T, d, V, M, 1 if is_bwd else 0))
+
+
+def atgrpo_policy_loss_launch_count(T: int, d: int, V: int, M: int, is_bwd: bool) -> int:
+    return int(lib().atgrpo_policy_loss_launch_count(T, d, V, M, 1 if is_bwd else 0))
 
 
 def atgrpo_policy_loss_fwd(H, W, target, role_of_token, head_of_role, resp_of_token, adv, old_logp,

@@ -141,6 +141,13 @@ size_t atgrpo_policy_loss_workspace_bytes(int64_t T, int32_t d, int32_t V, int32
   return policy_plan(T, d, V, M, is_bwd != 0, false, sm_count_or_default()).total;
 }
 
+int32_t atgrpo_policy_loss_launch_count(int64_t T, int32_t d, int32_t V, int32_t M, int32_t is_bwd) {
+  if (T <= 0 || d < 1 || V < 1 || M < 1) return 0;
+  const int route = M == 1 ? 1 : 4;                  // single-head table, or hist + scan + scatter + gather
+  if (!is_bwd) return route + 3;                     // + GEMM sweep, logsumexp combine, Eq. 2 reduction
+  return route + 1 + 3 * lm_head_bwd_chunks(padded_rows(T, M), V) + 1;   // + coef, 3 GEMMs per chunk, dH cast
+}
+
 int atgrpo_policy_loss_fwd(const void* H, int64_t ldH, const void* const* W, int32_t M,
                            const int32_t* target, const int32_t* role_of_token,
                            const int32_t* head_of_role, int32_t n_role,

@@ -598,6 +598,11 @@ int device_sm_count(int* n_sm, int* cc_major) {
   return ATGRPO_OK;
 }
 
+int lm_head_bwd_chunks(int64_t T_pad, int32_t V) {
+  const int vc = bwd_chunk_width(T_pad, V);
+  return (V + vc - 1) / vc;
+}
+
 size_t lm_head_fwd_workspace_bytes(int64_t T_pad, int32_t d, int32_t V, int32_t n_sm) {
   (void)d;
   return fwd_plan(T_pad, V, n_sm).total;

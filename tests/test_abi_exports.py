@@ -1,0 +1,76 @@
+"""CPU-only checks of the boundary: the library builds, loads, exports every symbol the header
+declares, and its host-side queries and argument checks behave (no kernel runs here)."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2510_11062_b200 import atgrpo as A
+from paper_2510_11062_b200 import build as B
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    B.build()
+    return A.lib()
+
+
+def _declared_symbols():
+    text = open(os.path.join(ROOT, "include", "atgrpo.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(atgrpo_[a-z_]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(lib):
+    names = _declared_symbols()
+    assert len(names) >= 9
+    for n in names:
+        assert hasattr(lib, n), n
+    assert set(A.EXPORTS) == set(names)
+
+
+def test_status_strings(lib):
+    texts = {A.status_string(c) for c in range(7)}
+    assert len(texts) == 7 and A.status_string(99) == "unknown status"
+
+
+def test_workspace_queries_are_monotone_and_aligned(lib):
+    a = A.atgrpo_group_advantages_workspace_bytes(1000, 64)
+    b = A.atgrpo_group_advantages_workspace_bytes(2_230_914, 262_144)
+    assert 0 < a < b and a % 256 == 0 and b % 256 == 0
+    f = A.atgrpo_policy_loss_workspace_bytes(16157, 2048, 151936, 1, False)
+    g = A.atgrpo_policy_loss_workspace_bytes(16157, 2048, 151936, 1, True)
+    assert 0 < f < g < (1 << 30)                       # bounded chunk buffer, not T x V
+    assert g < 16157 * 151936 * 2 / 8
+    assert A.atgrpo_policy_loss_launch_count(16157, 2048, 151936, 1, True) > \
+        A.atgrpo_policy_loss_launch_count(16157, 2048, 151936, 1, False) > 0
+    assert A.atgrpo_clipped_loss_workspace_bytes(4_194_304) > 0
+
+
+def test_host_side_argument_checks_need_no_gpu(lib):
+    p = A.Params().c()
+    rc = lib.atgrpo_group_advantages(None, None, None, None, 4, 1, 1, 1, ctypes.byref(p), None, None, None,
+                                     None, None, None, None, None, 0, None)
+    assert rc == A.ERR_INVALID_ARG
+    rc = lib.atgrpo_group_advantages(None, None, None, None, -1, 1, 1, 1, ctypes.byref(p), None, None, None,
+                                     None, None, None, None, None, 0, None)
+    assert rc == A.ERR_INVALID_ARG
+    rc = lib.atgrpo_clipped_loss(None, None, None, None, 0, 0, ctypes.byref(p), None, None, None, None, None, 0, None)
+    assert rc == A.ERR_INVALID_ARG                     # loss pointer is required
+    W = (ctypes.c_void_p * 1)(256)
+    rc = lib.atgrpo_policy_loss_fwd(None, 2048, W, 9, None, None, None, 0, None, None, 0, None, 0, 2048, 1000,
+                                    ctypes.byref(p), None, None, None, None, None, None, None, None, 0, None)
+    assert rc == A.ERR_UNSUPPORTED                     # more heads than ATGRPO_MAX_HEADS
+    rc = lib.atgrpo_policy_loss_fwd(None, 2044, W, 1, None, None, None, 0, None, None, 0, None, 0, 2044, 1000,
+                                    ctypes.byref(p), None, None, None, None, None, None, None, None, 0, None)
+    assert rc == A.ERR_UNSUPPORTED                     # d not a multiple of 8
+
+
+def test_binding_refuses_cpu_tensors(lib):
+    import torch
+    t = torch.zeros(4)
+    with pytest.raises(A.AtgrpoError):
+        A.atgrpo_clipped_loss(t, t, t.int(), t, A.Params(), t[:1], workspace=torch.zeros(256, dtype=torch.uint8))
