@@ -30,7 +30,7 @@ from paper_2510_11062_b200 import workloads as WL  # noqa: E402
 
 METRIC = "fused AT-GRPO loss fwd+bwd tokens/sec"
 UNIT = "tokens/s"
-CPU_SAMPLE_TOKENS = 128
+CPU_SAMPLE_TOKENS = 1024
 
 
 def measured_peaks():
@@ -357,7 +357,7 @@ def run_ours(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", default="qwen3_1p7b", choices=sorted(WL.SPECS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])

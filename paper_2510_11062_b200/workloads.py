@@ -43,6 +43,8 @@ SPECS = {
     "tiny": RolloutSpec("tiny", 4, 2, 2, 4, (16, 16), (64, 64), 128, 2048, 1, 1235),
     # single policy, Qwen3-1.7B-shaped head
     "qwen3_1p7b": RolloutSpec("qwen3_1p7b", 16, 2, 2, 4, (32, 32), (96, 96), 2048, 151936, 1, 1236),
+    # the same head on a quarter of the batch: small enough for multi-pass profiler captures
+    "qwen3_1p7b_small": RolloutSpec("qwen3_1p7b_small", 4, 2, 2, 4, (32, 32), (96, 96), 2048, 151936, 1, 1242),
     # three roles, one head per role, role 0 carries about half of the tokens
     "multi3": RolloutSpec("multi3", 24, 3, 2, 4, (96, 32, 32), (128, 80, 80), 2048, 151936, 3, 1237),
     # single policy, Qwen3-8B-shaped head
