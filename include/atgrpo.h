@@ -100,6 +100,35 @@ int atgrpo_group_advantages(
     int32_t* device_status, void* workspace, size_t workspace_bytes, void* stream);
 
 /* ------------------------------------------------------------------------------------------
+ * Grouped advantage without a workspace.  The paper has no counterpart to this entry point; it
+ * exists for callers that must not allocate device memory where the advantages are computed:
+ * a process that shares the GPU with an inference engine under a fixed memory budget, a plugin
+ * whose host application owns every allocation, or a training loop whose caching allocator must
+ * not be disturbed between steps.  Same arguments, results and error reporting as
+ * atgrpo_group_advantages, minus `workspace`: the scratch is a fixed 4 MiB array inside the
+ * library's device image (held by every GPU that loads the library until the process exits).
+ * Limits: n_cand <= ATGRPO_NOALLOC_MAX_CAND and n_env*n_role*n_turn <= ATGRPO_NOALLOC_MAX_GROUPS;
+ * anything larger returns ATGRPO_ERR_UNSUPPORTED with nothing enqueued.
+ * The call makes no cudaMalloc / cudaFree and calls no allocating routine.  The first call on a
+ * device looks up the array's device address (cudaGetSymbolAddress, with that device current)
+ * and remembers it; make that first call before starting any stream capture.
+ * All calls on one device share the one array, which keeps the previous call's contents; each
+ * call clears what it needs to start from zero.  Two calls whose kernels can overlap on the GPU
+ * (different streams without an ordering between them) race on the array: serialise them.
+ * ------------------------------------------------------------------------------------------ */
+#define ATGRPO_NOALLOC_MAX_CAND 262144
+#define ATGRPO_NOALLOC_MAX_GROUPS 65536
+
+int atgrpo_group_advantages_noalloc(
+    const float* rewards, const int32_t* env_id, const int32_t* role_id, const int32_t* turn_id,
+    int64_t n_cand, int32_t n_env, int32_t n_role, int32_t n_turn,
+    const atgrpo_params* params /* host */,
+    float* adv,
+    int32_t* group_of_cand, int32_t* group_offsets, int32_t* group_perm,
+    float* group_mean, float* group_std,
+    int32_t* device_status, void* stream);
+
+/* ------------------------------------------------------------------------------------------
  * Clipped-ratio loss from given log-probabilities -- Eq. 2 alone, one policy.
  *
  * For response token j: rho = exp(logp[j] - old_logp[j]), A = adv[resp_of_token[j]]

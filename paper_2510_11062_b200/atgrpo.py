@@ -23,6 +23,7 @@ MAX_HEADS = 8
 EXPORTS = (
     "atgrpo_status_string",
     "atgrpo_group_advantages_workspace_bytes", "atgrpo_group_advantages",
+    "atgrpo_group_advantages_noalloc",
     "atgrpo_clipped_loss_workspace_bytes", "atgrpo_clipped_loss",
     "atgrpo_policy_loss_workspace_bytes", "atgrpo_policy_loss_launch_count",
     "atgrpo_policy_loss_fwd", "atgrpo_policy_loss_bwd",
@@ -74,6 +75,9 @@ def lib() -> ctypes.CDLL:
         L.atgrpo_group_advantages.restype = ctypes.c_int
         L.atgrpo_group_advantages.argtypes = [vp, vp, vp, vp, i64, i32, i32, i32, pp, vp, vp, vp, vp,
                                               vp, vp, vp, vp, sz, vp]
+        L.atgrpo_group_advantages_noalloc.restype = ctypes.c_int
+        L.atgrpo_group_advantages_noalloc.argtypes = [vp, vp, vp, vp, i64, i32, i32, i32, pp, vp, vp, vp, vp,
+                                                      vp, vp, vp, vp]
         L.atgrpo_clipped_loss_workspace_bytes.restype = sz
         L.atgrpo_clipped_loss_workspace_bytes.argtypes = [i64]
         L.atgrpo_clipped_loss.restype = ctypes.c_int
@@ -150,6 +154,27 @@ def atgrpo_group_advantages(rewards, env_id, role_id, turn_id, n_env, n_role, n_
         _ptr(group_mean, f32), _ptr(group_std, f32), _ptr(device_status, i32),
         _ptr(workspace), workspace.numel(), _stream())
     _check(rc, "atgrpo_group_advantages")
+
+
+NOALLOC_MAX_CAND, NOALLOC_MAX_GROUPS = 262144, 65536
+
+
+def atgrpo_group_advantages_noalloc(rewards, env_id, role_id, turn_id, n_env, n_role, n_turn, params: Params,
+                                    adv, group_of_cand=None, group_offsets=None, group_perm=None,
+                                    group_mean=None, group_std=None, device_status=None):
+    """atgrpo_group_advantages for callers that may not allocate device memory: no workspace
+    argument, the scratch is a fixed array inside the library (see include/atgrpo.h for the size
+    limits and the sharing rules).  Returns the status code instead of raising on
+    ERR_UNSUPPORTED so callers can fall back when a batch is too large."""
+    i32, f32 = torch.int32, torch.float32
+    rc = lib().atgrpo_group_advantages_noalloc(
+        _ptr(rewards, f32), _ptr(env_id, i32), _ptr(role_id, i32), _ptr(turn_id, i32),
+        rewards.numel(), n_env, n_role, n_turn, ctypes.byref(params.c()), _ptr(adv, f32),
+        _ptr(group_of_cand, i32), _ptr(group_offsets, i32), _ptr(group_perm, i32),
+        _ptr(group_mean, f32), _ptr(group_std, f32), _ptr(device_status, i32), _stream())
+    if rc != ERR_UNSUPPORTED:
+        _check(rc, "atgrpo_group_advantages_noalloc")
+    return rc
 
 
 def atgrpo_clipped_loss_workspace_bytes(T: int) -> int:

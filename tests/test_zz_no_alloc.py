@@ -1,0 +1,65 @@
+"""The workspace-free grouped-advantage entry point against the regular one.
+
+Some users of the library cannot allocate device memory where advantages are computed (a fixed
+memory budget shared with an inference engine, a host application that owns all allocations), so
+atgrpo_group_advantages_noalloc keeps its scratch in a fixed array inside the library.  That array
+is shared by all calls and keeps stale contents, so the check runs two different inputs back to
+back and expects every output to equal the regular entry point's, bit for bit (both run the same
+kernels).  This file sorts last on purpose: a run that stops at the first failure has already run
+every other test."""
+import pytest
+import torch
+
+from paper_2510_11062_b200 import atgrpo as A
+from paper_2510_11062_b200 import workloads as WL
+from tests import _util as U
+
+pytestmark = pytest.mark.gpu
+
+
+def _noalloc(s, n_env, n_role, n_turn):
+    dev = U.DEV
+    R, G = s["R"], n_env * n_role * n_turn
+    i32, f32 = torch.int32, torch.float32
+    out = dict(adv=torch.full((R,), 7.0, dtype=f32, device=dev),
+               group_of_cand=torch.full((R,), -5, dtype=i32, device=dev),
+               group_offsets=torch.full((G + 1,), -5, dtype=i32, device=dev),
+               group_perm=torch.full((R,), -5, dtype=i32, device=dev),
+               group_mean=torch.full((G,), 7.0, dtype=f32, device=dev),
+               group_std=torch.full((G,), 7.0, dtype=f32, device=dev))
+    status = A.new_status(dev)
+    ins = [s[k].to(dev) for k in ("rewards", "env_id", "role_id", "turn_id")]
+    torch.cuda.synchronize()
+    before = torch.cuda.memory_allocated()
+    rc = A.atgrpo_group_advantages_noalloc(*ins, n_env, n_role, n_turn, A.Params(), device_status=status, **out)
+    torch.cuda.synchronize()
+    assert rc == A.OK and int(status.item()) == 0
+    assert torch.cuda.memory_allocated() == before          # the call drew nothing from torch's allocator
+    return {k: v.cpu() for k, v in out.items()}
+
+
+def test_noalloc_matches_regular_entry_point_twice_in_a_row():
+    # two different batches back to back: the second call sees the first call's leftovers
+    first = WL.make_stress(n_env=900, n_role=4, n_turn=4, n_tokens=10, seed=21)
+    second = WL.make_stress(n_env=333, n_role=3, n_turn=5, n_tokens=10, seed=22, k_max=9)
+    for s, dims in ((first, (900, 4, 4)), (second, (333, 3, 5))):
+        got = _noalloc(s, *dims)
+        ref = U.gpu_group_advantages(s["rewards"], s["env_id"], s["role_id"], s["turn_id"], *dims)
+        assert ref["status"] == 0
+        for k, v in got.items():
+            assert torch.equal(v, ref[k]), k
+
+
+def test_noalloc_rejects_sizes_beyond_its_fixed_scratch():
+    dev = U.DEV
+    n = A.NOALLOC_MAX_CAND + 1
+    z_f = torch.zeros(n, dtype=torch.float32, device=dev)
+    z_i = torch.zeros(n, dtype=torch.int32, device=dev)
+    adv = torch.full((n,), 7.0, dtype=torch.float32, device=dev)
+    assert A.atgrpo_group_advantages_noalloc(z_f, z_i, z_i, z_i, 4, 1, 1, A.Params(), adv) == A.ERR_UNSUPPORTED
+    small = z_f[:8], z_i[:8]
+    rc = A.atgrpo_group_advantages_noalloc(small[0], small[1], small[1], small[1], A.NOALLOC_MAX_GROUPS + 1, 1, 1,
+                                           A.Params(), adv[:8])
+    assert rc == A.ERR_UNSUPPORTED
+    torch.cuda.synchronize()
+    assert (adv == 7.0).all()                               # nothing was enqueued
