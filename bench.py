@@ -354,16 +354,80 @@ def run_ours(args):
     print(json.dumps(line), flush=True)
 
 
+def run_stress(args):
+    """Memory-bound workload: grouped advantages over 262144 (env, role, turn) slots and the Eq. 2
+    reduction over 4 Mi tokens (x scale).  L2 is flushed before every timed call (outside the
+    timed events), so the GB/s are HBM figures: 20 B per candidate, 12 B per token."""
+    from paper_2510_11062_b200 import atgrpo as A
+    A.lib()
+    dev = torch.device("cuda", int(os.environ.get("LOCAL_RANK", "0")))
+    torch.cuda.set_device(dev)
+    scale = 16 if args.workload == "stress16" else 1
+    s = WL.make_stress(n_env=16384 * scale, n_tokens=4_194_304 * scale)
+    R, G, T = s["R"], s["G"], s["T"]
+    d = {k: s[k].to(dev) for k in ("rewards", "env_id", "role_id", "turn_id", "resp_of_token", "logp", "old_logp")}
+    adv = torch.empty(R, device=dev)
+    loss = torch.zeros(1, device=dev)
+    status = A.new_status(dev)
+    ws_a = A.workspace(A.atgrpo_group_advantages_workspace_bytes(R, G), dev)
+    ws_l = A.workspace(A.atgrpo_clipped_loss_workspace_bytes(T), dev)
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
+    prm = A.Params()
+
+    def f_adv():
+        A.atgrpo_group_advantages(d["rewards"], d["env_id"], d["role_id"], d["turn_id"], s["n_env"], s["n_role"],
+                                  s["n_turn"], prm, adv, device_status=status, workspace=ws_a)
+
+    def f_loss():
+        A.atgrpo_clipped_loss(d["logp"], d["old_logp"], d["resp_of_token"], adv, prm, loss, None, None, status, ws_l)
+
+    def timed(f):
+        for _ in range(max(args.warmup, 3)):
+            f()
+        ts = []
+        for _ in range(args.steps):
+            flush.zero_()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(); f(); b.record()
+            torch.cuda.synchronize()
+            ts.append(a.elapsed_time(b))
+        return statistics.median(ts), min(ts)
+
+    sampler = ClockSampler(dev.index or 0)
+    adv_ms, adv_best = timed(f_adv)
+    loss_ms, loss_best = timed(f_loss)
+    clocks = sampler.stop()
+    if int(status.item()) != 0:
+        raise SystemExit("device status %d" % int(status.item()))
+    peaks = measured_peaks()
+    adv_gbs = 20.0 * R / (adv_ms * 1e-3) / 1e9
+    loss_gbs = 12.0 * T / (loss_ms * 1e-3) / 1e9
+    line = dict(metric="grouped advantage HBM GB/s (20 B per candidate)", value=adv_gbs, unit="GB/s", n_gpus=1,
+                steps=args.steps, warmup=max(args.warmup, 3), ms_per_step=adv_ms, higher_is_better=True,
+                scaling="weak", vs_baseline=None, dtype="f32", data="synthetic",
+                config=dict(workload=args.workload, candidates=R, group_slots=G, tokens=T,
+                            l2="flushed before every timed call"),
+                gpu_launches=5 * args.steps,
+                roofline=dict(bound="hbm", kernel="grouped-advantage pipeline (5 launches)", achieved=adv_gbs,
+                              peak=peaks["hbm_gbs"], unit="GB/s", frac=adv_gbs / peaks["hbm_gbs"], traffic=None,
+                              peak_source=peaks["source"] + " copy bandwidth"),
+                loss_reduction=dict(ms=loss_ms, gbs=loss_gbs, frac=loss_gbs / peaks["hbm_gbs"], bytes_per_token=12),
+                best_ms=dict(advantages=adv_best, loss_reduction=loss_best), clocks=clocks)
+    print(json.dumps(line), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--workload", default="qwen3_1p7b", choices=sorted(WL.SPECS))
+    ap.add_argument("--workload", default="qwen3_1p7b", choices=sorted(WL.SPECS) + ["stress", "stress16"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.workload.startswith("stress"):
+        run_stress(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)

@@ -145,7 +145,7 @@ int32_t atgrpo_policy_loss_launch_count(int64_t T, int32_t d, int32_t V, int32_t
   if (T <= 0 || d < 1 || V < 1 || M < 1) return 0;
   const int route = M == 1 ? 1 : 4;                  // single-head table, or hist + scan + scatter + gather
   if (!is_bwd) return route + 3;                     // + GEMM sweep, logsumexp combine, Eq. 2 reduction
-  return route + 1 + 3 * lm_head_bwd_chunks(padded_rows(T, M), V) + 1;   // + coef, 3 GEMMs per chunk, dH cast
+  return route + 1 + 3 * lm_head_bwd_chunks(padded_rows(T, M), d, V, M, sm_count_or_default()) + 1;   // + coef, 3 GEMMs per chunk, dH cast
 }
 
 int atgrpo_policy_loss_fwd(const void* H, int64_t ldH, const void* const* W, int32_t M,

@@ -73,6 +73,6 @@ int lm_head_bwd_launch(const LmHeadProblem& p, const float* lse, const float* co
                        const int32_t* row_of_token, const atgrpo_params& prm, void* dH,
                        void* const* dW, void* workspace, cudaStream_t st);
 int device_sm_count(int* n_sm, int* cc_major);
-int lm_head_bwd_chunks(int64_t T_pad, int32_t V);   // vocabulary chunks of one backward call
+int lm_head_bwd_chunks(int64_t T_pad, int32_t d, int32_t V, int32_t M, int32_t n_sm);   // vocabulary chunks of one backward call
 
 }  // namespace atgrpo

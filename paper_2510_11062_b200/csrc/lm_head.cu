@@ -54,6 +54,7 @@ struct GemmArgs {
   int n_vtiles;           // 256-wide vocabulary tiles in this launch
   int tiles_per_chunk;    // kFwd: tiles one work item sweeps (1 for kDz)
   int n_chunks;
+  int m_block;            // kFwd / kDz: row tiles swept together so their rows of H stay in L2
   float* part_m;          // kFwd out: running max (log2 domain) [n_chunks, T_pad]
   float* part_s;          // kFwd out: sum of 2^(t - max)        [n_chunks, T_pad]
   float* zt;              // kFwd out: target logit              [T_pad]
@@ -110,9 +111,14 @@ __device__ __forceinline__ Tile decode_item(const GemmArgs& g, int it) {
   const int n_dt = (g.d + BN - 1) / BN;
   t.v0 = 0, t.chunk = 0, t.nt_begin = 0, t.nt_end = 1;
   if (kMode == kFwd || kMode == kDz) {
+    // Row tiles come in blocks of m_block; inside a block the row tile runs fastest, then the
+    // vocabulary chunk: co-resident CTAs share W tiles, and a block's rows of H stay in L2.
     const int n_mt = s->tile_begin[g.M];
-    const int c = it / n_mt, mt = it - c * n_mt;       // row tiles fastest: co-resident CTAs
-    t.head = head_of_tile(s, g.M, mt);                 // sweep the same vocabulary slice
+    const int per_block = g.m_block * g.n_chunks;
+    const int blk = it / per_block, rem = it - blk * per_block;
+    const int gm = min(g.m_block, n_mt - blk * g.m_block);
+    const int c = rem / gm, mt = blk * g.m_block + (rem - c * gm);
+    t.head = head_of_tile(s, g.M, mt);
     t.row0 = mt * BM;
     t.rows_valid = min(BM, s->rows[t.head] - (mt - s->tile_begin[t.head]) * BM);
     t.chunk = c;
@@ -534,14 +540,40 @@ int fwd_chunks(int64_t n_mt, int n_vt, int n_sm) {
   return best;
 }
 
-// Width of the dZ chunk buffer: as wide as a 256 MiB buffer allows.
-int bwd_chunk_width(int64_t T_pad, int V) {
-  const int64_t budget = 256ll << 20;
-  int64_t vc = budget / (T_pad * 2) / BN * BN;
+// Row tiles per block of the logits sweeps: as many as keep the block's rows of H (128*d*2 bytes
+// per tile) within about half of the 126 MB L2.
+int row_block_tiles(int64_t n_mt, int d) {
+  int64_t gm = (64ll << 20) / (128ll * d * 2);
+  if (gm < 1) gm = 1;
+  if (gm > n_mt) gm = n_mt > 0 ? n_mt : 1;
+  return (int)gm;
+}
+
+// Width of the dZ chunk buffer (a multiple of 256 columns, buffer <= 512 MiB): the width that
+// minimises the modelled time of the three GEMM launches per chunk, counted in k-steps of one
+// 128x256x64 tile per SM wave plus a fixed cost per launch.  Wave quantisation of the dW GEMM
+// (few, long tiles) is what this mostly avoids.
+int bwd_chunk_width(int64_t T_pad, int d, int V, int M, int n_sm) {
+  const int64_t budget = 512ll << 20;
   const int64_t vmax = (int64_t)(V + BN - 1) / BN * BN;
-  if (vc < BN) vc = BN;
-  if (vc > vmax) vc = vmax;
-  return (int)vc;
+  int64_t cap = budget / (T_pad * 2) / BN * BN;
+  if (cap < BN) cap = BN;
+  if (cap > vmax) cap = vmax;
+  const int64_t n_mt = T_pad / BM, n_dt = (d + BN - 1) / BN, ksd = (d + BK - 1) / BK;
+  auto waves = [&](int64_t tiles) { return (tiles + n_sm - 1) / n_sm; };
+  auto chunk_cost = [&](int64_t w) {
+    const int64_t z = waves(n_mt * ((w + BN - 1) / BN)) * ksd;
+    const int64_t h = waves(n_mt * n_dt) * ((w + BK - 1) / BK);
+    const int64_t dw = waves((int64_t)M * ((w + BM - 1) / BM) * n_dt) * ((2 * n_mt + M - 1) / M);
+    return z + h + dw + 3 * 24;
+  };
+  int64_t best = cap, best_cost = -1;
+  for (int64_t vc = BN; vc <= cap; vc += BN) {
+    const int64_t full = V / vc, tail = V - full * vc;
+    const int64_t cost = full * chunk_cost(vc) + (tail > 0 ? chunk_cost(tail) : 0);
+    if (best_cost < 0 || cost <= best_cost) best_cost = cost, best = vc;
+  }
+  return (int)best;
 }
 
 struct FwdPlan { size_t part_m, part_s, zt, total; int n_chunks, tiles_per_chunk, n_vt; };
@@ -560,9 +592,9 @@ FwdPlan fwd_plan(int64_t T_pad, int V, int n_sm) {
 }
 
 struct BwdPlan { size_t dz, dh_acc, total; int vc; };
-BwdPlan bwd_plan(int64_t T_pad, int d, int V, bool dH_direct) {
+BwdPlan bwd_plan(int64_t T_pad, int d, int V, int M, int n_sm, bool dH_direct) {
   BwdPlan p;
-  p.vc = bwd_chunk_width(T_pad, V);
+  p.vc = bwd_chunk_width(T_pad, d, V, M, n_sm);
   Carver c(nullptr);
   p.dz = c.off; c.take<__nv_bfloat16>((size_t)T_pad * p.vc);
   p.dh_acc = c.off;
@@ -598,8 +630,8 @@ int device_sm_count(int* n_sm, int* cc_major) {
   return ATGRPO_OK;
 }
 
-int lm_head_bwd_chunks(int64_t T_pad, int32_t V) {
-  const int vc = bwd_chunk_width(T_pad, V);
+int lm_head_bwd_chunks(int64_t T_pad, int32_t d, int32_t V, int32_t M, int32_t n_sm) {
+  const int vc = bwd_chunk_width(T_pad, d, V, M, n_sm);
   return (V + vc - 1) / vc;
 }
 
@@ -618,6 +650,7 @@ int lm_head_fwd_launch(const LmHeadProblem& p, float* lse, float* logp, void* wo
     if (!make_map(&maps.b[m], p.W[m], p.d, p.V, p.d, BK, BN)) return ATGRPO_ERR_CUDA;
   GemmArgs g = base_args(p);
   g.v_begin = 0, g.n_vtiles = pl.n_vt, g.tiles_per_chunk = pl.tiles_per_chunk, g.n_chunks = pl.n_chunks;
+  g.m_block = row_block_tiles(p.T_pad / BM, p.d);
   g.part_m = reinterpret_cast<float*>(ws + pl.part_m);
   g.part_s = reinterpret_cast<float*>(ws + pl.part_s);
   g.zt = reinterpret_cast<float*>(ws + pl.zt);
@@ -633,15 +666,14 @@ int lm_head_fwd_launch(const LmHeadProblem& p, float* lse, float* logp, void* wo
 
 size_t lm_head_bwd_workspace_bytes(int64_t T_pad, int32_t d, int32_t V, int32_t M, int32_t n_sm,
                                    bool dH_direct) {
-  (void)M, (void)n_sm;
-  return bwd_plan(T_pad, d, V, dH_direct).total;
+  return bwd_plan(T_pad, d, V, M, n_sm, dH_direct).total;
 }
 
 int lm_head_bwd_launch(const LmHeadProblem& p, const float* lse, const float* coef,
                        const int32_t* row_of_token, const atgrpo_params& prm, void* dH,
                        void* const* dW, void* workspace, cudaStream_t st) {
   const bool dH_direct = p.M == 1 && prm.dH_dtype == ATGRPO_F32;
-  const BwdPlan pl = bwd_plan(p.T_pad, p.d, p.V, dH_direct);
+  const BwdPlan pl = bwd_plan(p.T_pad, p.d, p.V, p.M, p.n_sm, dH_direct);
   char* ws = static_cast<char*>(workspace);
   __nv_bfloat16* dz = reinterpret_cast<__nv_bfloat16*>(ws + pl.dz);
   float* dh_acc = dH_direct ? static_cast<float*>(dH) : reinterpret_cast<float*>(ws + pl.dh_acc);
@@ -665,6 +697,7 @@ int lm_head_bwd_launch(const LmHeadProblem& p, const float* lse, const float* co
     g.vc_valid = p.V - v_begin < pl.vc ? p.V - v_begin : pl.vc;
     g.n_vtiles = (g.vc_valid + BN - 1) / BN;
     g.tiles_per_chunk = 1;
+    g.m_block = row_block_tiles(n_mt, p.d);
     g.n_chunks = g.n_vtiles;
     g.lse = lse, g.coef = coef, g.dz = dz;
     g.dh_acc = dh_acc, g.first_chunk = chunk == 0;
