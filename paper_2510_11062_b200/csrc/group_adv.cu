@@ -1,6 +1,18 @@
 // Agent- and turn-wise grouped advantage (Eq. 1 over the groups of Algorithm 1).
 //
-// Pipeline, all on the caller's stream, no host synchronisation:
+// Two pipelines, both on the caller's stream with no host synchronisation.
+//
+// (A) Advantages only (no bucketing output requested): a sort-free group aggregate in three
+//     passes over the candidates plus one over the groups.  Everything that is accumulated with
+//     atomics is an integer, so the result does not depend on the order of arrival:
+//       minmax  : g, per-group count, min and max reward (order-preserving integer encoding)
+//       moments : x = round((r - min)/(max - min) * 2^30); sum of x and of x^2 in 64-bit integers
+//       finalize: exact integer K*sum(x^2) - sum(x)^2 (128-bit) -> mean, 1/(std + eps) per group
+//       apply   : adv = (r - mean) * 1/(std + eps)
+//     Quantising to 2^-30 of the group's range moves mean and std by < 1e-9 of the range; a group
+//     with max == min gets exact zeros.  Random access touches only the per-group table.
+//
+// (B) Bucketing requested (group_offsets / group_perm): counting sort + ordered statistics:
 //   key_count  : g = (e*n_role + i)*n_turn + t, per-group histogram; the atomic's return value is
 //                the candidate's (arbitrary) arrival slot inside its group
 //   scan       : exclusive scan of the histogram -> group_offsets        (two launches)
@@ -147,6 +159,182 @@ k_scatter(const int32_t* __restrict__ gid, const int32_t* __restrict__ slot,
   }
 }
 
+
+// ------------------------------------------------------------------ (A) sort-free aggregate
+constexpr double kQuant = 1073741824.0;   // 2^30 steps across a group's reward range
+
+// Order-preserving map float -> uint32 (and back), so integer atomicMax orders rewards.
+__device__ __forceinline__ uint32_t enc_ordered(float f) {
+  const uint32_t b = __float_as_uint(f);
+  return b ^ ((b >> 31) ? 0xFFFFFFFFu : 0x80000000u);
+}
+__device__ __forceinline__ float dec_ordered(uint32_t e) {
+  return __uint_as_float((e & 0x80000000u) ? (e ^ 0x80000000u) : ~e);
+}
+
+struct GroupTable {            // struct of arrays over the G slots; one memset zeroes all of it
+  uint32_t* cnt;               // members
+  uint32_t* nmin;              // ~enc(min): atomicMax from 0 tracks the minimum
+  uint32_t* emax;              // enc(max)
+  unsigned long long* sum;     // sum of x;        after finalize: mean as double
+  unsigned long long* sqlo;    // sum of x^2 mod 2^32 parts; after finalize: 1/(std+eps) as double
+  unsigned long long* sqhi;    // sum of x^2 >> 32
+};
+
+__device__ __forceinline__ void minmax_one(int g, float r, const GroupTable& t) {
+  const uint32_t e = enc_ordered(r);
+  atomicAdd(&t.cnt[g], 1u);
+  atomicMax(&t.nmin[g], ~e);
+  atomicMax(&t.emax[g], e);
+}
+
+template <bool kVec>
+__global__ void __launch_bounds__(kThreads)
+k_hash_minmax(const int32_t* __restrict__ env, const int32_t* __restrict__ role,
+              const int32_t* __restrict__ turn, const float* __restrict__ rewards, int n, int n_env,
+              int n_role, int n_turn, GroupTable t, int32_t* __restrict__ gid,
+              float* __restrict__ adv, int32_t* status) {
+  const int stride = gridDim.x * blockDim.x;
+  const int tid = blockIdx.x * blockDim.x + threadIdx.x;
+  if (kVec) {
+    const int n4 = n >> 2;
+    for (int q = tid; q < n4; q += stride) {
+      const int4 e = reinterpret_cast<const int4*>(env)[q];
+      const int4 r = reinterpret_cast<const int4*>(role)[q];
+      const int4 u = reinterpret_cast<const int4*>(turn)[q];
+      const float4 w = reinterpret_cast<const float4*>(rewards)[q];
+      int4 g;
+      g.x = group_of(e.x, r.x, u.x, n_env, n_role, n_turn);
+      g.y = group_of(e.y, r.y, u.y, n_env, n_role, n_turn);
+      g.z = group_of(e.z, r.z, u.z, n_env, n_role, n_turn);
+      g.w = group_of(e.w, r.w, u.w, n_env, n_role, n_turn);
+      reinterpret_cast<int4*>(gid)[q] = g;
+      if (g.x >= 0) minmax_one(g.x, w.x, t);
+      if (g.y >= 0) minmax_one(g.y, w.y, t);
+      if (g.z >= 0) minmax_one(g.z, w.z, t);
+      if (g.w >= 0) minmax_one(g.w, w.w, t);
+      if ((g.x | g.y | g.z | g.w) < 0) {
+        raise_status(status, ATGRPO_ERR_BAD_INDEX);
+        if (g.x < 0) adv[4 * q + 0] = 0.f;
+        if (g.y < 0) adv[4 * q + 1] = 0.f;
+        if (g.z < 0) adv[4 * q + 2] = 0.f;
+        if (g.w < 0) adv[4 * q + 3] = 0.f;
+      }
+    }
+  }
+  const int first = kVec ? (n & ~3) : 0;
+  for (int c = first + tid; c < n; c += stride) {
+    const int g = group_of(env[c], role[c], turn[c], n_env, n_role, n_turn);
+    gid[c] = g;
+    if (g >= 0) {
+      minmax_one(g, rewards[c], t);
+    } else {
+      adv[c] = 0.f;
+      raise_status(status, ATGRPO_ERR_BAD_INDEX);
+    }
+  }
+}
+
+__device__ __forceinline__ void moments_one(int g, float r, const GroupTable& t) {
+  const double lo = (double)dec_ordered(~t.nmin[g]);
+  const double range = (double)dec_ordered(t.emax[g]) - lo;
+  if (!(range > 0.0)) return;                       // single member or all equal: nothing to add
+  const unsigned long long x = (unsigned long long)__double2ll_rn(((double)r - lo) * (kQuant / range));
+  const unsigned long long x2 = x * x;              // < 2^60
+  atomicAdd(&t.sum[g], x);
+  atomicAdd(&t.sqlo[g], x2 & 0xFFFFFFFFull);
+  atomicAdd(&t.sqhi[g], x2 >> 32);
+}
+
+template <bool kVec>
+__global__ void __launch_bounds__(kThreads)
+k_hash_moments(const int32_t* __restrict__ gid, const float* __restrict__ rewards, int n,
+               GroupTable t) {
+  const int stride = gridDim.x * blockDim.x;
+  const int tid = blockIdx.x * blockDim.x + threadIdx.x;
+  if (kVec) {
+    const int n4 = n >> 2;
+    for (int q = tid; q < n4; q += stride) {
+      const int4 g = reinterpret_cast<const int4*>(gid)[q];
+      const float4 w = reinterpret_cast<const float4*>(rewards)[q];
+      if (g.x >= 0) moments_one(g.x, w.x, t);
+      if (g.y >= 0) moments_one(g.y, w.y, t);
+      if (g.z >= 0) moments_one(g.z, w.z, t);
+      if (g.w >= 0) moments_one(g.w, w.w, t);
+    }
+  }
+  const int first = kVec ? (n & ~3) : 0;
+  for (int c = first + tid; c < n; c += stride) {
+    const int g = gid[c];
+    if (g >= 0) moments_one(g, rewards[c], t);
+  }
+}
+
+__global__ void __launch_bounds__(kThreads)
+k_hash_finalize(GroupTable t, int G, float std_eps, int ddof, float* __restrict__ group_mean,
+                float* __restrict__ group_std) {
+  const int g = blockIdx.x * blockDim.x + threadIdx.x;
+  if (g >= G) return;
+  const unsigned K = t.cnt[g];
+  double mu = 0.0, sd = 0.0, inv = 0.0;
+  if (K > 0) {
+    const double lo = (double)dec_ordered(~t.nmin[g]);
+    const double range = (double)dec_ordered(t.emax[g]) - lo;
+    mu = lo;
+    if (range > 0.0) {
+      const unsigned long long sx = t.sum[g];
+      const unsigned __int128 sxx = ((unsigned __int128)t.sqhi[g] << 32) + t.sqlo[g];
+      const unsigned __int128 num = (unsigned __int128)K * sxx - (unsigned __int128)sx * sx;   // exact, >= 0
+      const double step = range / kQuant;
+      mu = lo + ((double)sx / (double)K) * step;
+      const int dof = (int)K - ddof;
+      if (dof > 0) {
+        const double num_d = (double)(unsigned long long)(num >> 64) * 18446744073709551616.0 +
+                             (double)(unsigned long long)num;
+        sd = sqrt(num_d / ((double)K * (double)dof)) * step;
+      }
+    }
+    if (K > 1) inv = 1.0 / (sd + (double)std_eps);
+  }
+  t.sum[g] = (unsigned long long)__double_as_longlong(mu);
+  t.sqlo[g] = (unsigned long long)__double_as_longlong(inv);
+  if (group_mean) group_mean[g] = (float)mu;
+  if (group_std) group_std[g] = (float)sd;
+}
+
+__device__ __forceinline__ float apply_one(int g, float r, const GroupTable& t) {
+  const double mu = __longlong_as_double((long long)t.sum[g]);
+  const double inv = __longlong_as_double((long long)t.sqlo[g]);
+  return (float)(((double)r - mu) * inv);
+}
+
+template <bool kVec>
+__global__ void __launch_bounds__(kThreads)
+k_hash_apply(const int32_t* __restrict__ gid, const float* __restrict__ rewards, int n,
+             GroupTable t, float* __restrict__ adv) {
+  const int stride = gridDim.x * blockDim.x;
+  const int tid = blockIdx.x * blockDim.x + threadIdx.x;
+  if (kVec) {
+    const int n4 = n >> 2;
+    for (int q = tid; q < n4; q += stride) {
+      const int4 g = reinterpret_cast<const int4*>(gid)[q];
+      const float4 w = reinterpret_cast<const float4*>(rewards)[q];
+      float4 a;
+      a.x = g.x >= 0 ? apply_one(g.x, w.x, t) : 0.f;
+      a.y = g.y >= 0 ? apply_one(g.y, w.y, t) : 0.f;
+      a.z = g.z >= 0 ? apply_one(g.z, w.z, t) : 0.f;
+      a.w = g.w >= 0 ? apply_one(g.w, w.w, t) : 0.f;
+      reinterpret_cast<float4*>(adv)[q] = a;
+    }
+  }
+  const int first = kVec ? (n & ~3) : 0;
+  for (int c = first + tid; c < n; c += stride) {
+    const int g = gid[c];
+    adv[c] = g >= 0 ? apply_one(g, rewards[c], t) : 0.f;
+  }
+}
+
+// ------------------------------------------------------------------ (B) ordered statistics
 struct StatsArgs {
   const float* rewards;
   const int32_t* offsets;
@@ -316,18 +504,23 @@ __global__ void __launch_bounds__(kThreads) k_group_stats(StatsArgs a) {
 }
 
 struct Plan {
-  size_t count, slot, gid, offsets, perm, block_sum, total;
+  size_t count, slot, gid, offsets, perm, block_sum;   // pipeline (B)
+  size_t h_gid, h_table;                               // pipeline (A): gid[n], then 36 bytes per slot
+  size_t total;
 };
 Plan make_plan(int64_t n, int64_t G) {
-  Carver c(nullptr);
   Plan p;
+  Carver c(nullptr);
   p.count = c.off; c.take<int32_t>((size_t)G);
   p.slot = c.off; c.take<int32_t>((size_t)n);
   p.gid = c.off; c.take<int32_t>((size_t)n);
   p.offsets = c.off; c.take<int32_t>((size_t)G + 1);
   p.perm = c.off; c.take<int32_t>((size_t)n);
   p.block_sum = c.off; c.take<int32_t>((size_t)((G + kScanBlock - 1) / kScanBlock) + 1);
-  p.total = c.off;
+  Carver h(nullptr);                                   // the two pipelines never run together:
+  p.h_gid = h.off; h.take<int32_t>((size_t)n);         // they share the same bytes
+  p.h_table = h.off; h.take<unsigned long long>((size_t)G * 9 / 2 + 8);
+  p.total = c.off > h.off ? c.off : h.off;
   return p;
 }
 
@@ -354,6 +547,41 @@ int group_adv_launch(const float* rewards, const int32_t* env_id, const int32_t*
   int32_t* offsets = group_offsets ? group_offsets : reinterpret_cast<int32_t*>(ws + pl.offsets);
   int32_t* perm = group_perm ? group_perm : reinterpret_cast<int32_t*>(ws + pl.perm);
   int32_t* block_sum = reinterpret_cast<int32_t*>(ws + pl.block_sum);
+
+  if (n > 0 && group_offsets == nullptr && group_perm == nullptr) {
+    // (A) advantages only
+    int32_t* hgid = group_of_cand ? group_of_cand : reinterpret_cast<int32_t*>(ws + pl.h_gid);
+    char* tb = ws + pl.h_table;
+    GroupTable t;
+    t.sum = reinterpret_cast<unsigned long long*>(tb);
+    t.sqlo = t.sum + G;
+    t.sqhi = t.sqlo + G;
+    t.cnt = reinterpret_cast<uint32_t*>(t.sqhi + G);
+    t.nmin = t.cnt + G;
+    t.emax = t.nmin + G;
+    ATGRPO_CUDA_OK(cudaMemsetAsync(tb, 0, (size_t)G * 36, st));
+    const bool v1 = aligned16(env_id) && aligned16(role_id) && aligned16(turn_id) &&
+                    aligned16(rewards) && aligned16(hgid);
+    const bool v2 = aligned16(rewards) && aligned16(hgid);
+    const bool v3 = v2 && aligned16(adv);
+    auto grid_of = [&](bool v) {
+      int64_t b = ((v ? (n + 3) / 4 : n) + kThreads - 1) / kThreads;
+      return (int)(b > 148 * 16 ? 148 * 16 : b);
+    };
+    if (v1)
+      k_hash_minmax<true><<<grid_of(true), kThreads, 0, st>>>(env_id, role_id, turn_id, rewards, n, n_env,
+                                                              n_role, n_turn, t, hgid, adv, device_status);
+    else
+      k_hash_minmax<false><<<grid_of(false), kThreads, 0, st>>>(env_id, role_id, turn_id, rewards, n, n_env,
+                                                                n_role, n_turn, t, hgid, adv, device_status);
+    if (v2) k_hash_moments<true><<<grid_of(true), kThreads, 0, st>>>(hgid, rewards, n, t);
+    else k_hash_moments<false><<<grid_of(false), kThreads, 0, st>>>(hgid, rewards, n, t);
+    k_hash_finalize<<<(int)((G + kThreads - 1) / kThreads), kThreads, 0, st>>>(t, (int)G, prm.std_eps, prm.ddof,
+                                                                               group_mean, group_std);
+    if (v3) k_hash_apply<true><<<grid_of(true), kThreads, 0, st>>>(hgid, rewards, n, t, adv);
+    else k_hash_apply<false><<<grid_of(false), kThreads, 0, st>>>(hgid, rewards, n, t, adv);
+    return launch_ok();
+  }
 
   ATGRPO_CUDA_OK(cudaMemsetAsync(count, 0, (size_t)G * sizeof(int32_t), st));
   if (n == 0) {

@@ -26,6 +26,7 @@ struct LossArgs {
   double* part_sum;            // [grid, M]
   int64_t* part_cnt;           // [grid, M, 3] tokens, clipped-low, clipped-high
   unsigned* done;
+  int vec;                     // logp, old_logp, resp (and coef) are 16-byte aligned
 };
 
 // Per-token term of Eq. 2.  Returns l_j; `active` tells whether the unclipped branch carries the
@@ -39,44 +40,65 @@ __device__ __forceinline__ float clipped_term(float logp, float old_logp, float 
   return -fminf(u, c);
 }
 
+struct TokenAcc {
+  double sum;
+  int cnt, clo, chi;
+};
+
+template <int kHeads>
+__device__ __forceinline__ void loss_token(const LossArgs& a, int64_t j, float logp, float old_logp,
+                                           int rs, float inv_T, TokenAcc* acc) {
+  int head = 0;
+  if (kHeads != 1) {
+    const int r = a.role[j];
+    head = (unsigned)r < (unsigned)a.n_role ? a.head_of_role[r] : -1;
+    if ((unsigned)head >= (unsigned)a.M) {
+      raise_status(a.status, ATGRPO_ERR_BAD_INDEX);
+      return;
+    }
+  }
+  float A = 0.f;
+  if ((unsigned)rs < (unsigned)a.n_resp) A = a.adv[rs];
+  else raise_status(a.status, ATGRPO_ERR_BAD_INDEX);
+  float rho;
+  bool active;
+  const float l = clipped_term(logp, old_logp, A, a.lo, a.hi, rho, active);
+  if (kHeads == 1 && a.coef) a.coef[j] = active ? A * rho * inv_T : 0.f;
+#pragma unroll
+  for (int m = 0; m < (kHeads == 1 ? 1 : ATGRPO_MAX_HEADS); ++m) {
+    if (m == head) {
+      acc[m].sum += (double)l;
+      acc[m].cnt += 1;
+      acc[m].clo += rho < a.lo;
+      acc[m].chi += rho > a.hi;
+    }
+  }
+}
+
 template <int kHeads>   // 1: single policy, no routing arrays; 0: generic (a.M heads)
 __global__ void __launch_bounds__(kThreads) k_clipped_loss(LossArgs a) {
   constexpr int H = kHeads == 1 ? 1 : ATGRPO_MAX_HEADS;
-  double sum[H];
-  int cnt[H], clo[H], chi[H];
+  TokenAcc acc[H];
 #pragma unroll
-  for (int m = 0; m < H; ++m) sum[m] = 0.0, cnt[m] = 0, clo[m] = 0, chi[m] = 0;
+  for (int m = 0; m < H; ++m) acc[m].sum = 0.0, acc[m].cnt = 0, acc[m].clo = 0, acc[m].chi = 0;
   const int64_t stride = (int64_t)gridDim.x * kThreads;
+  const int64_t tid = (int64_t)blockIdx.x * kThreads + threadIdx.x;
   const float inv_T = a.T > 0 ? 1.f / (float)a.T : 0.f;
-  for (int64_t j = (int64_t)blockIdx.x * kThreads + threadIdx.x; j < a.T; j += stride) {
-    int head = 0;
-    if (kHeads != 1) {
-      const int r = a.role[j];
-      head = (unsigned)r < (unsigned)a.n_role ? a.head_of_role[r] : -1;
-      if ((unsigned)head >= (unsigned)a.M) {
-        raise_status(a.status, ATGRPO_ERR_BAD_INDEX);
-        continue;
-      }
-    }
-    const int rs = a.resp[j];
-    float A = 0.f;
-    if ((unsigned)rs < (unsigned)a.n_resp) A = a.adv[rs];
-    else raise_status(a.status, ATGRPO_ERR_BAD_INDEX);
-    float rho;
-    bool active;
-    const float l = clipped_term(a.logp[j], a.old_logp[j], A, a.lo, a.hi, rho, active);
-    if (kHeads == 1 && a.coef) a.coef[j] = active ? A * rho * inv_T : 0.f;
-#pragma unroll
-    for (int m = 0; m < H; ++m) {
-      if (m == head) {
-        sum[m] += (double)l;
-        cnt[m] += 1;
-        clo[m] += rho < a.lo;
-        chi[m] += rho > a.hi;
-      }
-    }
+  // four consecutive tokens per thread and iteration (16-byte loads) when the arrays allow it
+  const int64_t n4 = a.vec ? a.T >> 2 : 0;
+  for (int64_t q = tid; q < n4; q += stride) {
+    const float4 lp = reinterpret_cast<const float4*>(a.logp)[q];
+    const float4 lo = reinterpret_cast<const float4*>(a.old_logp)[q];
+    const int4 rs = reinterpret_cast<const int4*>(a.resp)[q];
+    loss_token<kHeads>(a, 4 * q + 0, lp.x, lo.x, rs.x, inv_T, acc);
+    loss_token<kHeads>(a, 4 * q + 1, lp.y, lo.y, rs.y, inv_T, acc);
+    loss_token<kHeads>(a, 4 * q + 2, lp.z, lo.z, rs.z, inv_T, acc);
+    loss_token<kHeads>(a, 4 * q + 3, lp.w, lo.w, rs.w, inv_T, acc);
   }
-  // block reduction in a fixed order: shuffle tree inside each warp, then warp 0 adds the warps
+  for (int64_t j = 4 * n4 + tid; j < a.T; j += stride)
+    loss_token<kHeads>(a, j, a.logp[j], a.old_logp[j], a.resp[j], inv_T, acc);
+
+  // block reduction in a fixed order: shuffle tree inside each warp, then one thread per head
   __shared__ double s_sum[kThreads / 32][H];
   __shared__ int s_cnt[kThreads / 32][H][3];
   __shared__ bool s_last;
@@ -85,8 +107,8 @@ __global__ void __launch_bounds__(kThreads) k_clipped_loss(LossArgs a) {
 #pragma unroll
   for (int m = 0; m < H; ++m) {
     if (m < M) {
-      double v = sum[m];
-      int c0 = cnt[m], c1 = clo[m], c2 = chi[m];
+      double v = acc[m].sum;
+      int c0 = acc[m].cnt, c1 = acc[m].clo, c2 = acc[m].chi;
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) {
         v += __shfl_down_sync(0xffffffffu, v, o);
@@ -113,24 +135,41 @@ __global__ void __launch_bounds__(kThreads) k_clipped_loss(LossArgs a) {
     int64_t* pc = a.part_cnt + ((size_t)blockIdx.x * M + m) * 3;
     pc[0] = c0, pc[1] = c1, pc[2] = c2;
   }
-  // the block that finishes last adds the per-block partials, again in a fixed order
+  // the block that finishes last adds the per-block partials: each thread a fixed strided
+  // subset, then a fixed tree, so the order never depends on which block came last
   __threadfence();
   __syncthreads();
   if (threadIdx.x == 0) s_last = atomicAdd(a.done, 1u) == gridDim.x - 1;
   __syncthreads();
   if (!s_last) return;
   __threadfence();
-  if ((int)threadIdx.x < M) {
-    const int m = threadIdx.x;
+  __shared__ double r_sum[kThreads];
+  __shared__ long long r_cnt[kThreads][3];
+  for (int m = 0; m < M; ++m) {
     double v = 0.0;
-    int64_t c0 = 0, c1 = 0, c2 = 0;
-    for (unsigned b = 0; b < gridDim.x; ++b) {
+    long long c0 = 0, c1 = 0, c2 = 0;
+    for (unsigned b = threadIdx.x; b < gridDim.x; b += kThreads) {
       v += a.part_sum[(size_t)b * M + m];
       const int64_t* pc = a.part_cnt + ((size_t)b * M + m) * 3;
       c0 += pc[0], c1 += pc[1], c2 += pc[2];
     }
-    a.loss[m] = c0 > 0 ? (float)(v / (double)c0) : 0.f;
-    if (a.clip_counts) a.clip_counts[2 * m] = c1, a.clip_counts[2 * m + 1] = c2;
+    r_sum[threadIdx.x] = v;
+    r_cnt[threadIdx.x][0] = c0, r_cnt[threadIdx.x][1] = c1, r_cnt[threadIdx.x][2] = c2;
+    __syncthreads();
+    for (int s2 = kThreads / 2; s2 > 0; s2 >>= 1) {
+      if ((int)threadIdx.x < s2) {
+        r_sum[threadIdx.x] += r_sum[threadIdx.x + s2];
+        r_cnt[threadIdx.x][0] += r_cnt[threadIdx.x + s2][0];
+        r_cnt[threadIdx.x][1] += r_cnt[threadIdx.x + s2][1];
+        r_cnt[threadIdx.x][2] += r_cnt[threadIdx.x + s2][2];
+      }
+      __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+      a.loss[m] = r_cnt[0][0] > 0 ? (float)(r_sum[0] / (double)r_cnt[0][0]) : 0.f;
+      if (a.clip_counts) a.clip_counts[2 * m] = r_cnt[0][1], a.clip_counts[2 * m + 1] = r_cnt[0][2];
+    }
+    __syncthreads();
   }
   if (threadIdx.x == 0) *a.done = 0;
 }
@@ -341,6 +380,8 @@ int loss_reduce_launch(const float* logp, const float* old_logp, const int32_t* 
   a.part_sum = c.take<double>((size_t)g * ATGRPO_MAX_HEADS);
   a.part_cnt = c.take<int64_t>((size_t)g * ATGRPO_MAX_HEADS * 3);
   a.done = c.take<unsigned>(1);
+  auto al16 = [](const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; };
+  a.vec = al16(logp) && al16(old_logp) && al16(resp_of_token);
   ATGRPO_CUDA_OK(cudaMemsetAsync(a.done, 0, sizeof(unsigned), st));
   if (M == 1) k_clipped_loss<1><<<g, kThreads, 0, st>>>(a);
   else k_clipped_loss<0><<<g, kThreads, 0, st>>>(a);

@@ -24,17 +24,20 @@ def to_dev(t):
 
 
 def gpu_group_advantages(rewards, env_id, role_id, turn_id, n_env, n_role, n_turn, prm=None,
-                         want_all=True):
+                         want_all=True, bucketing=True):
+    """bucketing=False leaves group_offsets / group_perm out, which selects the library's sort-free
+    pipeline; with them it runs the counting-sort pipeline."""
     prm = prm or A.Params()
     R, G = rewards.numel(), n_env * n_role * n_turn
     i32, f32 = torch.int32, torch.float32
     out = dict(adv=torch.full((R,), 7.0, dtype=f32, device=DEV))
     if want_all:
         out.update(group_of_cand=torch.full((R,), -5, dtype=i32, device=DEV),
-                   group_offsets=torch.full((G + 1,), -5, dtype=i32, device=DEV),
-                   group_perm=torch.full((R,), -5, dtype=i32, device=DEV),
                    group_mean=torch.full((G,), 7.0, dtype=f32, device=DEV),
                    group_std=torch.full((G,), 7.0, dtype=f32, device=DEV))
+        if bucketing:
+            out.update(group_offsets=torch.full((G + 1,), -5, dtype=i32, device=DEV),
+                       group_perm=torch.full((R,), -5, dtype=i32, device=DEV))
     status = A.new_status(DEV)
     ws = A.workspace(A.atgrpo_group_advantages_workspace_bytes(R, G), DEV)
     A.atgrpo_group_advantages(to_dev(rewards), to_dev(env_id), to_dev(role_id), to_dev(turn_id),

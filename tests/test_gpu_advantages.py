@@ -13,9 +13,11 @@ pytestmark = pytest.mark.gpu
 
 def _run_case(rewards, env_id, role_id, turn_id, n_env, n_role, n_turn, ddof=0):
     prm = A.Params(ddof=ddof)
-    gpu = U.gpu_group_advantages(rewards, env_id, role_id, turn_id, n_env, n_role, n_turn, prm)
     ref = U.oracle_group_advantages(rewards, env_id, role_id, turn_id, n_env, n_role, n_turn, ddof=ddof)
-    U.check_group_advantages(gpu, ref)
+    for bucketing in (False, True):          # sort-free pipeline, then counting-sort pipeline
+        gpu = U.gpu_group_advantages(rewards, env_id, role_id, turn_id, n_env, n_role, n_turn, prm,
+                                     bucketing=bucketing)
+        U.check_group_advantages(gpu, ref)
     return gpu, ref
 
 
@@ -56,6 +58,20 @@ def test_large_groups_take_the_block_path():
     role_id = ((slot // n_turn) % n_role).to(torch.int32)
     turn_id = (slot % n_turn).to(torch.int32)
     _run_case(rewards, env_id, role_id, turn_id, n_env, n_role, n_turn)
+
+
+def test_nearly_equal_and_wide_range_rewards():
+    # groups whose rewards differ in the last bit, negative rewards, and magnitudes from 1e-20 to 1e20:
+    # a sum-of-squares formula without a shift would lose these
+    one = torch.tensor(1.0)
+    up = torch.nextafter(one, torch.tensor(2.0))
+    rewards = torch.tensor([1.0, up, 1.0, up, -3.0, -3.0, -3.0, -2.9999998, 1e-20, 3e-20, 2e-20, 5e20, -5e20, 0.0,
+                            7.5], dtype=torch.float32)
+    slot = torch.tensor([0, 0, 0, 0, 1, 1, 1, 1, 2, 2, 2, 3, 3, 3, 4])
+    env = slot.to(torch.int32)
+    zero = torch.zeros_like(env)
+    _run_case(rewards, env, zero, zero, 5, 1, 1)
+    _run_case(rewards, env, zero, zero, 5, 1, 1, ddof=1)
 
 
 def test_unaligned_pointers_and_no_optional_outputs():
@@ -115,10 +131,14 @@ def test_host_side_errors_enqueue_nothing():
 
 def test_repeatable_bitwise():
     s = WL.make_stress(n_env=2000, n_role=4, n_turn=4, n_tokens=10, seed=9)
-    a = U.gpu_group_advantages(s["rewards"], s["env_id"], s["role_id"], s["turn_id"], 2000, 4, 4)
-    b = U.gpu_group_advantages(s["rewards"], s["env_id"], s["role_id"], s["turn_id"], 2000, 4, 4)
-    for k in ("adv", "group_perm", "group_offsets", "group_mean", "group_std"):
-        assert torch.equal(a[k], b[k]), k
+    for bucketing in (False, True):
+        a = U.gpu_group_advantages(s["rewards"], s["env_id"], s["role_id"], s["turn_id"], 2000, 4, 4,
+                                   bucketing=bucketing)
+        b = U.gpu_group_advantages(s["rewards"], s["env_id"], s["role_id"], s["turn_id"], 2000, 4, 4,
+                                   bucketing=bucketing)
+        for k in a:
+            if k != "status":
+                assert torch.equal(a[k], b[k]), k
 
 
 # ------------------------------------------------------------------------------- Eq. 2 reduction

@@ -113,9 +113,11 @@ def test_full_size_dense_identities():
 def test_stress_full_size():
     s = WL.make_stress()
     dims = (s["n_env"], s["n_role"], s["n_turn"])
-    gpu = U.gpu_group_advantages(s["rewards"], s["env_id"], s["role_id"], s["turn_id"], *dims)
     ref = U.oracle_group_advantages(s["rewards"], s["env_id"], s["role_id"], s["turn_id"], *dims)
-    U.check_group_advantages(gpu, ref)
+    for bucketing in (False, True):
+        gpu = U.gpu_group_advantages(s["rewards"], s["env_id"], s["role_id"], s["turn_id"], *dims,
+                                     bucketing=bucketing)
+        U.check_group_advantages(gpu, ref)
     assert (ref["adv"] == 0).sum() > 0.01 * s["G"]
     adv = torch.from_numpy(ref["adv"]).float()
     dev = U.DEV
