@@ -8,8 +8,8 @@
 //   kDh  : dH_rows += dZ_chunk * W_m[chunk, :]          (A K-major, B MN-major)
 //   kDw  : dW_m[chunk, :] = dZ_chunk^T * H_rows          (A and B MN-major)
 //
-// CTA layout (192 threads): warp 0 = TMA producer, warp 1 = tcgen05.mma issuer and TMEM owner,
-// warps 2-5 = epilogue (one TMEM lane quarter each).  Tiles are 128 x 256 x 64 (bf16), operands
+// CTA layout (320 threads): warp 0 = TMA producer, warp 1 = tcgen05.mma issuer and TMEM owner,
+// warps 2-9 = epilogue (two warps per TMEM lane quarter, each taking half of the tile's columns).  Tiles are 128 x 256 x 64 (bf16), operands
 // are staged by TMA into a 4-deep ring of 128-byte-swizzled shared-memory tiles, the fp32
 // accumulator is double buffered in the 512 TMEM columns so the epilogue of tile i overlaps the
 // MMAs of tile i+1.  Rows are addressed in the "padded row space": the tokens of policy m occupy
@@ -29,7 +29,8 @@ constexpr int kABytes = BM * BK * 2;               // 16 KiB
 constexpr int kBBytes = BN * BK * 2;               // 32 KiB
 constexpr int kStageBytes = kABytes + kBBytes;     // 48 KiB
 constexpr int kBoxBytes = 64 * 64 * 2;             // one 64 x 64 MN-major box, 8 KiB
-constexpr int kGemmThreads = 192;
+constexpr int kGemmThreads = 320;               // producer warp, MMA warp, 8 epilogue warps
+constexpr int kEpilogueThreads = 256;
 constexpr int kTmemCols = 512;
 constexpr int kSmemBytes = kStages * kStageBytes + 1024 /* alignment slack */ + 256 /* barriers */;
 constexpr float kLog2e = 1.4426950408889634f;
@@ -55,8 +56,8 @@ struct GemmArgs {
   int tiles_per_chunk;    // kFwd: tiles one work item sweeps (1 for kDz)
   int n_chunks;
   int m_block;            // kFwd / kDz: row tiles swept together so their rows of H stay in L2
-  float* part_m;          // kFwd out: running max (log2 domain) [n_chunks, T_pad]
-  float* part_s;          // kFwd out: sum of 2^(t - max)        [n_chunks, T_pad]
+  float* part_m;          // kFwd out: running max (log2 domain) [2*n_chunks, T_pad]
+  float* part_s;          // kFwd out: sum of 2^(t - max)        [2*n_chunks, T_pad]
   float* zt;              // kFwd out: target logit              [T_pad]
   const float* lse;       // kDz in, token order
   const float* coef;      // kDz in, token order
@@ -75,6 +76,13 @@ __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
+}
+
+// 256-bit global store (sm_100): p must be 32-byte aligned.
+__device__ __forceinline__ void st_global_v8(void* p, const uint32_t* v) {
+  asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(p), "r"(v[0]), "r"(v[1]),
+               "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7])
+               : "memory");
 }
 
 struct Tile {
@@ -96,8 +104,8 @@ __device__ __forceinline__ int head_of_tile(const Schedule* s, int M, int mt) {
 }
 
 template <int kMode>
-__device__ __forceinline__ int total_items(const GemmArgs& g) {
-  const int n_mt = g.sched->tile_begin[g.M];
+__device__ __forceinline__ int total_items(const GemmArgs& g, const Schedule* sched) {
+  const int n_mt = sched->tile_begin[g.M];
   const int n_dt = (g.d + BN - 1) / BN;
   if (kMode == kFwd || kMode == kDz) return n_mt * g.n_chunks;
   if (kMode == kDh) return n_mt * n_dt;
@@ -105,9 +113,8 @@ __device__ __forceinline__ int total_items(const GemmArgs& g) {
 }
 
 template <int kMode>
-__device__ __forceinline__ Tile decode_item(const GemmArgs& g, int it) {
+__device__ __forceinline__ Tile decode_item(const GemmArgs& g, const Schedule* s, int it) {
   Tile t;
-  const Schedule* s = g.sched;
   const int n_dt = (g.d + BN - 1) / BN;
   t.v0 = 0, t.chunk = 0, t.nt_begin = 0, t.nt_end = 1;
   if (kMode == kFwd || kMode == kDz) {
@@ -164,6 +171,13 @@ k_lm_head(const __grid_constant__ Maps maps, const GemmArgs g) {
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
+  // the tile schedule is read once per CTA: every role decodes its tiles from shared memory
+  __shared__ Schedule s_sched;
+  if (threadIdx.x >= 64 && threadIdx.x < 64 + sizeof(Schedule) / 4)
+    reinterpret_cast<int32_t*>(&s_sched)[threadIdx.x - 64] =
+        reinterpret_cast<const int32_t*>(g.sched)[threadIdx.x - 64];
+  const Schedule* sched = &s_sched;
+
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
       mbar_init(full_bar(s), 1);
@@ -171,7 +185,7 @@ k_lm_head(const __grid_constant__ Maps maps, const GemmArgs g) {
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(tfull_bar(a), 1);
-      mbar_init(tempty_bar(a), 128);
+      mbar_init(tempty_bar(a), kEpilogueThreads);
     }
     *s_abort = 0;
     fence_mbar_init();
@@ -185,7 +199,7 @@ k_lm_head(const __grid_constant__ Maps maps, const GemmArgs g) {
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *s_tmem;
-  const int n_items = total_items<kMode>(g);
+  const int n_items = total_items<kMode>(g, sched);
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
@@ -194,7 +208,7 @@ k_lm_head(const __grid_constant__ Maps maps, const GemmArgs g) {
       uint32_t phase = 0;
       bool ok = true;
       for (int it = blockIdx.x; ok && it < n_items; it += gridDim.x) {
-        const Tile t = decode_item<kMode>(g, it);
+        const Tile t = decode_item<kMode>(g, sched, it);
         for (int nt = t.nt_begin; ok && nt < t.nt_end; ++nt) {
           const int n0 = t.n0 + (nt - t.nt_begin) * BN;
           for (int ks = 0; ks < t.k_steps; ++ks) {
@@ -232,7 +246,7 @@ k_lm_head(const __grid_constant__ Maps maps, const GemmArgs g) {
       uint32_t phase = 0, acc_phase = 0;
       bool ok = true;
       for (int it = blockIdx.x; ok && it < n_items; it += gridDim.x) {
-        const Tile t = decode_item<kMode>(g, it);
+        const Tile t = decode_item<kMode>(g, sched, it);
         if (t.k_steps == 0) continue;
         for (int nt = t.nt_begin; ok && nt < t.nt_end; ++nt) {
           if (!(ok = mbar_wait(tempty_bar(acc), acc_phase ^ 1u, s_abort, g.status))) break;
@@ -261,14 +275,19 @@ k_lm_head(const __grid_constant__ Maps maps, const GemmArgs g) {
     }
   } else {
     // ------------------------------------------------------------------ epilogue warps
+    // Two warps per TMEM lane quarter (a warp can only read the quarter warp_id % 4): the first
+    // four epilogue warps take columns 0-127 of the tile, the other four columns 128-255, so every
+    // scheduler has two epilogue warps to hide each other's TMEM-load and MUFU latency.
     const int quarter = warp & 3;
+    const int half = (warp - 2) >> 2;
+    const int c_begin = half * (BN / 64), c_end = c_begin + BN / 64;
     const int r_in_tile = quarter * 32 + lane;
     const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16);
     int acc = 0;
     uint32_t acc_phase = 0;
     bool ok = true;
     for (int it = blockIdx.x; ok && it < n_items; it += gridDim.x) {
-      const Tile t = decode_item<kMode>(g, it);
+      const Tile t = decode_item<kMode>(g, sched, it);
       uint32_t r[32];
 
       if (kMode == kFwd || kMode == kDz) {
@@ -291,7 +310,7 @@ k_lm_head(const __grid_constant__ Maps maps, const GemmArgs g) {
           const int n0 = t.n0 + (nt - t.nt_begin) * BN;
           if (!(ok = mbar_wait(tfull_bar(acc), acc_phase, s_abort, g.status))) break;
           tc_fence_after();
-          for (int c = 0; c < BN / 32; ++c) {
+          for (int c = c_begin; c < c_end; ++c) {
             const int col0 = n0 + c * 32;
             if (kMode == kFwd && col0 >= g.V) break;
             __syncwarp();
@@ -304,40 +323,50 @@ k_lm_head(const __grid_constant__ Maps maps, const GemmArgs g) {
                   if (col0 + i == y) zt = __uint_as_float(r[i]);
                 have_zt = true;
               }
-              float tv[32];
-              float cmax = -INFINITY;
+              // running (max, sum) in the log2 domain: max on the raw logits (log2 e > 0), then
+              // one FFMA + ex2 + add per element
               const bool ragged = col0 + 32 > g.V;
+              float cmax = -INFINITY;
 #pragma unroll
               for (int i = 0; i < 32; ++i) {
-                tv[i] = __uint_as_float(r[i]) * kLog2e;
-                if (ragged && col0 + i >= g.V) tv[i] = -INFINITY;
-                cmax = fmaxf(cmax, tv[i]);
+                if (ragged && col0 + i >= g.V) r[i] = 0xff800000u;     // -inf
+                cmax = fmaxf(cmax, __uint_as_float(r[i]));
               }
-              const float nm = fmaxf(m2, cmax);
-              float add = 0.f;
+              const float nm = fmaxf(m2, cmax * kLog2e);
+              float add0 = 0.f, add1 = 0.f;
 #pragma unroll
-              for (int i = 0; i < 32; ++i) add += ex2(tv[i] - nm);
-              ssum = ssum * ex2(m2 - nm) + add;
+              for (int i = 0; i < 32; i += 2) {
+                add0 += ex2(fmaf(__uint_as_float(r[i]), kLog2e, -nm));
+                add1 += ex2(fmaf(__uint_as_float(r[i + 1]), kLog2e, -nm));
+              }
+              ssum = fmaf(ssum, ex2(m2 - nm), add0 + add1);
               m2 = nm;
             } else {
+              // dZ = coef * softmax, minus coef at the target column; zero beyond the vocabulary
+              float gz[32];
+#pragma unroll
+              for (int i = 0; i < 32; ++i)
+                gz[i] = cf * ex2(fmaf(__uint_as_float(r[i]), kLog2e, -lse2));
+              if (y >= col0 && y < col0 + 32) {
+#pragma unroll
+                for (int i = 0; i < 32; ++i)
+                  if (col0 + i == y) gz[i] -= cf;
+              }
+              if (col0 + 32 > g.V) {
+#pragma unroll
+                for (int i = 0; i < 32; ++i)
+                  if (col0 + i >= g.V) gz[i] = 0.f;
+              }
               uint32_t packed[16];
 #pragma unroll
               for (int i = 0; i < 32; i += 2) {
-                float g0 = 0.f, g1 = 0.f;
-                if (tok >= 0) {
-                  const float p0 = ex2(__uint_as_float(r[i]) * kLog2e - lse2);
-                  const float p1 = ex2(__uint_as_float(r[i + 1]) * kLog2e - lse2);
-                  g0 = (col0 + i < g.V) ? cf * (p0 - (col0 + i == y ? 1.f : 0.f)) : 0.f;
-                  g1 = (col0 + i + 1 < g.V) ? cf * (p1 - (col0 + i + 1 == y ? 1.f : 0.f)) : 0.f;
-                }
-                const __nv_bfloat162 h2 = __floats2bfloat162_rn(g0, g1);
+                const __nv_bfloat162 h2 = __floats2bfloat162_rn(gz[i], gz[i + 1]);
                 packed[i >> 1] = *reinterpret_cast<const uint32_t*>(&h2);
               }
-              uint4* dst = reinterpret_cast<uint4*>(g.dz + (size_t)row * g.vc + (col0 - g.v_begin));
-#pragma unroll
-              for (int q4 = 0; q4 < 4; ++q4)
-                dst[q4] = make_uint4(packed[4 * q4], packed[4 * q4 + 1], packed[4 * q4 + 2],
-                                     packed[4 * q4 + 3]);
+              // 32-byte stores: one full sector per lane and half as many L1 wavefronts as 16-byte ones
+              __nv_bfloat16* dst = g.dz + (size_t)row * g.vc + (col0 - g.v_begin);
+              st_global_v8(dst, packed);
+              st_global_v8(dst + 16, packed + 8);
             }
           }
           tc_fence_before();
@@ -345,8 +374,8 @@ k_lm_head(const __grid_constant__ Maps maps, const GemmArgs g) {
           if (++acc == 2) acc = 0, acc_phase ^= 1u;
         }
         if (kMode == kFwd && ok && tok >= 0) {
-          g.part_m[(size_t)t.chunk * g.T_pad + row] = m2;
-          g.part_s[(size_t)t.chunk * g.T_pad + row] = ssum;
+          g.part_m[(size_t)(2 * t.chunk + half) * g.T_pad + row] = m2;
+          g.part_s[(size_t)(2 * t.chunk + half) * g.T_pad + row] = ssum;
           if (have_zt) g.zt[row] = zt;
         }
       } else {
@@ -366,7 +395,7 @@ k_lm_head(const __grid_constant__ Maps maps, const GemmArgs g) {
           valid = (t.v0 + r_in_tile < g.vc_valid) && v < g.V;
           out_row = (size_t)v;
         }
-        for (int c = 0; c < BN / 32; ++c) {
+        for (int c = c_begin; c < c_end; ++c) {
           const int col0 = t.n0 + c * 32;
           if (col0 >= g.d) break;
           if (has_acc) {
@@ -456,9 +485,9 @@ k_lse_combine(const Schedule* sched, int M, const int32_t* tok_of_row, int64_t T
     const int tok = tok_of_row[p];
     if (tok < 0) continue;
     float mx = -INFINITY;
-    for (int c = 0; c < n_chunks; ++c) mx = fmaxf(mx, part_m[(size_t)c * T_pad + p]);
-    float s = 0.f;
-    for (int c = 0; c < n_chunks; ++c)
+    for (int c = 0; c < 2 * n_chunks; ++c) mx = fmaxf(mx, part_m[(size_t)c * T_pad + p]);
+    float s = 0.f;                       // two column halves per vocabulary chunk
+    for (int c = 0; c < 2 * n_chunks; ++c)
       s += part_s[(size_t)c * T_pad + p] * exp2f(part_m[(size_t)c * T_pad + p] - mx);
     const float l = (mx + log2f(s)) * kLn2;
     lse[tok] = l;
@@ -584,8 +613,8 @@ FwdPlan fwd_plan(int64_t T_pad, int V, int n_sm) {
   p.n_chunks = fwd_chunks(n_mt > 0 ? n_mt : 1, p.n_vt, n_sm);
   p.tiles_per_chunk = (p.n_vt + p.n_chunks - 1) / p.n_chunks;
   Carver c(nullptr);
-  p.part_m = c.off; c.take<float>((size_t)p.n_chunks * T_pad);
-  p.part_s = c.off; c.take<float>((size_t)p.n_chunks * T_pad);
+  p.part_m = c.off; c.take<float>((size_t)2 * p.n_chunks * T_pad);
+  p.part_s = c.off; c.take<float>((size_t)2 * p.n_chunks * T_pad);
   p.zt = c.off; c.take<float>((size_t)T_pad);
   p.total = c.off;
   return p;
