@@ -17,8 +17,9 @@ bool params_ok(const atgrpo_params* p) {
 }
 
 int64_t padded_rows(int64_t T, int M) {
-  const int64_t tiles = (T + 127) / 128 + (M > 1 ? M : 0);
-  return tiles * 128;
+  // every head occupies whole 256-row tiles (the row extent of a CTA pair)
+  const int64_t tiles = (T + 255) / 256 + (M > 1 ? M : 0);
+  return tiles * 256;
 }
 
 int sm_count_or_default() {

@@ -23,11 +23,12 @@ namespace atgrpo {
 namespace {
 using namespace sm100;
 
-constexpr int BM = 128, BN = 256, BK = 64;
-constexpr int kStages = 4;
-constexpr int kABytes = BM * BK * 2;               // 16 KiB
-constexpr int kBBytes = BN * BK * 2;               // 32 KiB
-constexpr int kStageBytes = kABytes + kBBytes;     // 48 KiB
+constexpr int BM = 128, BN = 256, BK = 64;          // BM rows per CTA: a CTA pair owns 2*BM = 256 rows
+constexpr int kPairRows = 2 * BM;
+constexpr int kStages = 6;
+constexpr int kABytes = BM * BK * 2;               // 16 KiB: this CTA's 128 rows of A
+constexpr int kBBytes = (BN / 2) * BK * 2;         // 16 KiB: this CTA's half of B
+constexpr int kStageBytes = kABytes + kBBytes;     // 32 KiB per CTA and k-step
 constexpr int kBoxBytes = 64 * 64 * 2;             // one 64 x 64 MN-major box, 8 KiB
 constexpr int kGemmThreads = 320;               // producer warp, MMA warp, 8 epilogue warps
 constexpr int kEpilogueThreads = 256;
@@ -103,29 +104,31 @@ __device__ __forceinline__ int head_of_tile(const Schedule* s, int M, int mt) {
   return h;
 }
 
+// Work items are tiles of a CTA pair: 256 rows x 256 columns.  `rank` selects this CTA's half.
 template <int kMode>
 __device__ __forceinline__ int total_items(const GemmArgs& g, const Schedule* sched) {
-  const int n_mt = sched->tile_begin[g.M];
+  const int n_pt = sched->tile_begin[g.M] / 2;          // heads start on even 128-row tiles
   const int n_dt = (g.d + BN - 1) / BN;
-  if (kMode == kFwd || kMode == kDz) return n_mt * g.n_chunks;
-  if (kMode == kDh) return n_mt * n_dt;
-  return g.M * ((g.vc_valid + BM - 1) / BM) * n_dt;
+  if (kMode == kFwd || kMode == kDz) return n_pt * g.n_chunks;
+  if (kMode == kDh) return n_pt * n_dt;
+  return g.M * ((g.vc_valid + kPairRows - 1) / kPairRows) * n_dt;
 }
 
 template <int kMode>
-__device__ __forceinline__ Tile decode_item(const GemmArgs& g, const Schedule* s, int it) {
+__device__ __forceinline__ Tile decode_item(const GemmArgs& g, const Schedule* s, int it, int rank) {
   Tile t;
   const int n_dt = (g.d + BN - 1) / BN;
   t.v0 = 0, t.chunk = 0, t.nt_begin = 0, t.nt_end = 1;
   if (kMode == kFwd || kMode == kDz) {
-    // Row tiles come in blocks of m_block; inside a block the row tile runs fastest, then the
-    // vocabulary chunk: co-resident CTAs share W tiles, and a block's rows of H stay in L2.
-    const int n_mt = s->tile_begin[g.M];
+    // Row tiles come in blocks of m_block pairs; inside a block the row tile runs fastest, then
+    // the vocabulary chunk: co-resident pairs share W tiles, and a block's rows of H stay in L2.
+    const int n_pt = s->tile_begin[g.M] / 2;
     const int per_block = g.m_block * g.n_chunks;
     const int blk = it / per_block, rem = it - blk * per_block;
-    const int gm = min(g.m_block, n_mt - blk * g.m_block);
-    const int c = rem / gm, mt = blk * g.m_block + (rem - c * gm);
-    t.head = head_of_tile(s, g.M, mt);
+    const int gm = min(g.m_block, n_pt - blk * g.m_block);
+    const int c = rem / gm, pt = blk * g.m_block + (rem - c * gm);
+    const int mt = 2 * pt + rank;
+    t.head = head_of_tile(s, g.M, 2 * pt);
     t.row0 = mt * BM;
     t.rows_valid = min(BM, s->rows[t.head] - (mt - s->tile_begin[t.head]) * BM);
     t.chunk = c;
@@ -134,21 +137,22 @@ __device__ __forceinline__ Tile decode_item(const GemmArgs& g, const Schedule* s
     t.n0 = g.v_begin + t.nt_begin * BN;
     t.k_steps = (g.d + BK - 1) / BK;
   } else if (kMode == kDh) {
-    const int mt = it / n_dt, dt = it - mt * n_dt;     // d tiles fastest: they share the dZ tile
-    t.head = head_of_tile(s, g.M, mt);
+    const int pt = it / n_dt, dt = it - pt * n_dt;     // d tiles fastest: they share the dZ tile
+    const int mt = 2 * pt + rank;
+    t.head = head_of_tile(s, g.M, 2 * pt);
     t.row0 = mt * BM;
     t.rows_valid = min(BM, s->rows[t.head] - (mt - s->tile_begin[t.head]) * BM);
     t.n0 = dt * BN;
     t.k_steps = (g.vc_valid + BK - 1) / BK;
   } else {
-    const int n_vt = (g.vc_valid + BM - 1) / BM;
+    const int n_vt = (g.vc_valid + kPairRows - 1) / kPairRows;
     const int dt = it % n_dt, rest = it / n_dt;
     const int vt = rest % n_vt;
     t.head = rest / n_vt;
     t.row0 = s->tile_begin[t.head] * BM;
     t.rows_valid = 0;
     t.n0 = dt * BN;
-    t.v0 = vt * BM;
+    t.v0 = vt * kPairRows + rank * BM;
     t.k_steps = (s->tile_begin[t.head + 1] - s->tile_begin[t.head]) * (BM / BK);
   }
   return t;
@@ -170,6 +174,8 @@ k_lm_head(const __grid_constant__ Maps maps, const GemmArgs g) {
   volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int rank = (int)cluster_ctarank();           // 0 = leader of the pair (issues the MMAs)
+  const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
 
   // the tile schedule is read once per CTA: every role decodes its tiles from shared memory
   __shared__ Schedule s_sched;
@@ -178,6 +184,10 @@ k_lm_head(const __grid_constant__ Maps maps, const GemmArgs g) {
         reinterpret_cast<const int32_t*>(g.sched)[threadIdx.x - 64];
   const Schedule* sched = &s_sched;
 
+  // Barrier protocol of a pair.  full[s] lives in the leader: its producer announces the bytes of
+  // both CTAs (2 x 32 KiB) and the TMA loads of both CTAs report there.  empty[s] and tfull[a] exist in both CTAs and are
+  // signalled by the leader's multicast tcgen05.commit.  tempty[a] lives in the leader: the
+  // epilogue threads of both CTAs arrive on it.
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
       mbar_init(full_bar(s), 1);
@@ -185,18 +195,19 @@ k_lm_head(const __grid_constant__ Maps maps, const GemmArgs g) {
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(tfull_bar(a), 1);
-      mbar_init(tempty_bar(a), kEpilogueThreads);
+      mbar_init(tempty_bar(a), 2 * kEpilogueThreads);
     }
     *s_abort = 0;
     fence_mbar_init();
     prefetch_tmap(&maps.a);
   }
   if (warp == 1) {
-    tmem_alloc(smem_u32(const_cast<uint32_t*>(s_tmem)), kTmemCols);
-    tmem_relinquish();
+    tmem_alloc_pair(smem_u32(const_cast<uint32_t*>(s_tmem)), kTmemCols);
+    tmem_relinquish_pair();
   }
   tc_fence_before();
   __syncthreads();
+  cluster_sync_all();                                 // peer barriers initialised, TMEM allocated
   tc_fence_after();
   const uint32_t tmem_base = *s_tmem;
   const int n_items = total_items<kMode>(g, sched);
@@ -207,30 +218,30 @@ k_lm_head(const __grid_constant__ Maps maps, const GemmArgs g) {
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      for (int it = blockIdx.x; ok && it < n_items; it += gridDim.x) {
-        const Tile t = decode_item<kMode>(g, sched, it);
+      for (int it = pair; ok && it < n_items; it += n_pairs) {
+        const Tile t = decode_item<kMode>(g, sched, it, rank);
         for (int nt = t.nt_begin; ok && nt < t.nt_end; ++nt) {
-          const int n0 = t.n0 + (nt - t.nt_begin) * BN;
+          const int n0 = t.n0 + (nt - t.nt_begin) * BN + rank * (BN / 2);   // this CTA's half of B
           for (int ks = 0; ks < t.k_steps; ++ks) {
             if (!(ok = mbar_wait(empty_bar(stage), phase ^ 1u, s_abort, g.status))) break;
             const uint32_t sa = smem_base + stage * kStageBytes, sb = sa + kABytes;
-            const uint32_t fb = full_bar(stage);
-            mbar_expect_tx(fb, kStageBytes);
+            const uint32_t fb = mapa_shared(full_bar(stage), 0);             // the leader's barrier
+            if (rank == 0) mbar_expect_tx(full_bar(stage), 2 * kStageBytes);
             if (kMode == kFwd || kMode == kDz) {
-              tma_load_2d(sa, &maps.a, ks * BK, t.row0, fb);
-              tma_load_2d(sb, &maps.b[t.head], ks * BK, n0, fb);
+              tma_load_2d_pair(sa, &maps.a, ks * BK, t.row0, fb);
+              tma_load_2d_pair(sb, &maps.b[t.head], ks * BK, n0, fb);
             } else if (kMode == kDh) {
-              tma_load_2d(sa, &maps.a, ks * BK, t.row0, fb);
+              tma_load_2d_pair(sa, &maps.a, ks * BK, t.row0, fb);
 #pragma unroll
-              for (int b = 0; b < 4; ++b)
-                tma_load_2d(sb + b * kBoxBytes, &maps.b[t.head], n0 + 64 * b, g.v_begin + ks * BK, fb);
+              for (int b = 0; b < 2; ++b)
+                tma_load_2d_pair(sb + b * kBoxBytes, &maps.b[t.head], n0 + 64 * b, g.v_begin + ks * BK, fb);
             } else {
 #pragma unroll
               for (int b = 0; b < 2; ++b)
-                tma_load_2d(sa + b * kBoxBytes, &maps.a, t.v0 + 64 * b, t.row0 + ks * BK, fb);
+                tma_load_2d_pair(sa + b * kBoxBytes, &maps.a, t.v0 + 64 * b, t.row0 + ks * BK, fb);
 #pragma unroll
-              for (int b = 0; b < 4; ++b)
-                tma_load_2d(sb + b * kBoxBytes, &maps.b[0], n0 + 64 * b, t.row0 + ks * BK, fb);
+              for (int b = 0; b < 2; ++b)
+                tma_load_2d_pair(sb + b * kBoxBytes, &maps.b[0], n0 + 64 * b, t.row0 + ks * BK, fb);
             }
             if (++stage == kStages) stage = 0, phase ^= 1u;
           }
@@ -239,14 +250,14 @@ k_lm_head(const __grid_constant__ Maps maps, const GemmArgs g) {
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
+    if (lane == 0 && rank == 0) {
       constexpr bool a_mn = (kMode == kDw), b_mn = (kMode == kDh || kMode == kDw);
-      constexpr uint32_t idesc = idesc_bf16(BM, BN, a_mn, b_mn);
+      constexpr uint32_t idesc = idesc_bf16(kPairRows, BN, a_mn, b_mn);
       int stage = 0, acc = 0;
       uint32_t phase = 0, acc_phase = 0;
       bool ok = true;
-      for (int it = blockIdx.x; ok && it < n_items; it += gridDim.x) {
-        const Tile t = decode_item<kMode>(g, sched, it);
+      for (int it = pair; ok && it < n_items; it += n_pairs) {
+        const Tile t = decode_item<kMode>(g, sched, it, rank);
         if (t.k_steps == 0) continue;
         for (int nt = t.nt_begin; ok && nt < t.nt_end; ++nt) {
           if (!(ok = mbar_wait(tempty_bar(acc), acc_phase ^ 1u, s_abort, g.status))) break;
@@ -262,13 +273,13 @@ k_lm_head(const __grid_constant__ Maps maps, const GemmArgs g) {
                                        : smem_desc(sa + kk * 32, 16, 1024);
               const uint64_t bd = b_mn ? smem_desc(sb + kk * 2048, kBoxBytes, 1024)
                                        : smem_desc(sb + kk * 32, 16, 1024);
-              umma_bf16(d_tmem, ad, bd, idesc, (ks | kk) != 0 ? 1u : 0u);
+              umma_bf16_pair(d_tmem, ad, bd, idesc, (ks | kk) != 0 ? 1u : 0u);
             }
-            umma_commit(empty_bar(stage));        // frees the stage once these MMAs have read it
+            umma_commit_pair(empty_bar(stage), 3);   // frees the stage in both CTAs
             if (++stage == kStages) stage = 0, phase ^= 1u;
           }
           if (!ok) break;
-          umma_commit(tfull_bar(acc));            // accumulator complete
+          umma_commit_pair(tfull_bar(acc), 3);        // accumulator complete in both CTAs
           if (++acc == 2) acc = 0, acc_phase ^= 1u;
         }
       }
@@ -286,8 +297,9 @@ k_lm_head(const __grid_constant__ Maps maps, const GemmArgs g) {
     int acc = 0;
     uint32_t acc_phase = 0;
     bool ok = true;
-    for (int it = blockIdx.x; ok && it < n_items; it += gridDim.x) {
-      const Tile t = decode_item<kMode>(g, sched, it);
+    const uint32_t tempty_leader0 = mapa_shared(tempty_bar(0), 0), tempty_leader1 = mapa_shared(tempty_bar(1), 0);
+    for (int it = pair; ok && it < n_items; it += n_pairs) {
+      const Tile t = decode_item<kMode>(g, sched, it, rank);
       uint32_t r[32];
 
       if (kMode == kFwd || kMode == kDz) {
@@ -370,7 +382,7 @@ k_lm_head(const __grid_constant__ Maps maps, const GemmArgs g) {
             }
           }
           tc_fence_before();
-          mbar_arrive(tempty_bar(acc));
+          mbar_arrive_cluster(acc ? tempty_leader1 : tempty_leader0);
           if (++acc == 2) acc = 0, acc_phase ^= 1u;
         }
         if (kMode == kFwd && ok && tok >= 0) {
@@ -453,7 +465,7 @@ k_lm_head(const __grid_constant__ Maps maps, const GemmArgs g) {
         }
         if (has_acc) {
           tc_fence_before();
-          mbar_arrive(tempty_bar(acc));
+          mbar_arrive_cluster(acc ? tempty_leader1 : tempty_leader0);
           if (++acc == 2) acc = 0, acc_phase ^= 1u;
         }
       }
@@ -461,8 +473,10 @@ k_lm_head(const __grid_constant__ Maps maps, const GemmArgs g) {
   }
 
   // ---------------------------------------------------------------------- teardown
+  // Neither CTA may leave while its peer can still signal its barriers or read its shared memory.
   tc_fence_before();
   __syncthreads();
+  cluster_sync_all();
   if (warp == 1) {
     if (*s_abort) {
       // a wait gave up: let the loads this CTA may still have in flight land before its shared
@@ -471,7 +485,7 @@ k_lm_head(const __grid_constant__ Maps maps, const GemmArgs g) {
     }
     __syncwarp();
     tc_fence_after();
-    tmem_dealloc(tmem_base, kTmemCols);
+    tmem_dealloc_pair(tmem_base, kTmemCols);
   }
 }
 
@@ -569,18 +583,18 @@ int fwd_chunks(int64_t n_mt, int n_vt, int n_sm) {
   return best;
 }
 
-// Row tiles per block of the logits sweeps: as many as keep the block's rows of H (128*d*2 bytes
-// per tile) within about half of the 126 MB L2.
-int row_block_tiles(int64_t n_mt, int d) {
-  int64_t gm = (64ll << 20) / (128ll * d * 2);
+// Pair tiles (256 rows) per block of the logits sweeps: as many as keep the block's rows of H
+// within about half of the 126 MB L2.
+int row_block_tiles(int64_t n_pt, int d) {
+  int64_t gm = (64ll << 20) / ((int64_t)kPairRows * d * 2);
   if (gm < 1) gm = 1;
-  if (gm > n_mt) gm = n_mt > 0 ? n_mt : 1;
+  if (gm > n_pt) gm = n_pt > 0 ? n_pt : 1;
   return (int)gm;
 }
 
 // Width of the dZ chunk buffer (a multiple of 256 columns, buffer <= 512 MiB): the width that
 // minimises the modelled time of the three GEMM launches per chunk, counted in k-steps of one
-// 128x256x64 tile per SM wave plus a fixed cost per launch.  Wave quantisation of the dW GEMM
+// 256x256x64 pair tile per wave of CTA pairs plus a fixed cost per launch.  Wave quantisation of the dW GEMM
 // (few, long tiles) is what this mostly avoids.
 int bwd_chunk_width(int64_t T_pad, int d, int V, int M, int n_sm) {
   const int64_t budget = 512ll << 20;
@@ -588,12 +602,13 @@ int bwd_chunk_width(int64_t T_pad, int d, int V, int M, int n_sm) {
   int64_t cap = budget / (T_pad * 2) / BN * BN;
   if (cap < BN) cap = BN;
   if (cap > vmax) cap = vmax;
-  const int64_t n_mt = T_pad / BM, n_dt = (d + BN - 1) / BN, ksd = (d + BK - 1) / BK;
-  auto waves = [&](int64_t tiles) { return (tiles + n_sm - 1) / n_sm; };
+  const int64_t n_pt = T_pad / kPairRows, n_dt = (d + BN - 1) / BN, ksd = (d + BK - 1) / BK;
+  const int64_t n_pairs = n_sm / 2 > 0 ? n_sm / 2 : 1;
+  auto waves = [&](int64_t tiles) { return (tiles + n_pairs - 1) / n_pairs; };
   auto chunk_cost = [&](int64_t w) {
-    const int64_t z = waves(n_mt * ((w + BN - 1) / BN)) * ksd;
-    const int64_t h = waves(n_mt * n_dt) * ((w + BK - 1) / BK);
-    const int64_t dw = waves((int64_t)M * ((w + BM - 1) / BM) * n_dt) * ((2 * n_mt + M - 1) / M);
+    const int64_t z = waves(n_pt * ((w + BN - 1) / BN)) * ksd;
+    const int64_t h = waves(n_pt * n_dt) * ((w + BK - 1) / BK);
+    const int64_t dw = waves((int64_t)M * ((w + kPairRows - 1) / kPairRows) * n_dt) * ((4 * n_pt + M - 1) / M);
     return z + h + dw + 3 * 24;
   };
   int64_t best = cap, best_cost = -1;
@@ -609,8 +624,8 @@ struct FwdPlan { size_t part_m, part_s, zt, total; int n_chunks, tiles_per_chunk
 FwdPlan fwd_plan(int64_t T_pad, int V, int n_sm) {
   FwdPlan p;
   p.n_vt = (V + BN - 1) / BN;
-  const int64_t n_mt = T_pad / BM;
-  p.n_chunks = fwd_chunks(n_mt > 0 ? n_mt : 1, p.n_vt, n_sm);
+  const int64_t n_pt = T_pad / kPairRows;
+  p.n_chunks = fwd_chunks(n_pt > 0 ? n_pt : 1, p.n_vt, n_sm / 2 > 0 ? n_sm / 2 : 1);
   p.tiles_per_chunk = (p.n_vt + p.n_chunks - 1) / p.n_chunks;
   Carver c(nullptr);
   p.part_m = c.off; c.take<float>((size_t)2 * p.n_chunks * T_pad);
@@ -632,12 +647,31 @@ BwdPlan bwd_plan(int64_t T_pad, int d, int V, int M, int n_sm, bool dH_direct) {
   return p;
 }
 
+// Launches `pairs` clusters of two CTAs (never more than can be resident at once).
 template <int kMode>
-int launch_gemm(const Maps& maps, const GemmArgs& g, int grid, cudaStream_t st) {
+int launch_gemm(const Maps& maps, const GemmArgs& g, int64_t items, int n_sm, cudaStream_t st) {
   if (cudaFuncSetAttribute(k_lm_head<kMode>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            kSmemBytes) != cudaSuccess)
     return ATGRPO_ERR_CUDA;
-  k_lm_head<kMode><<<grid, kGemmThreads, kSmemBytes, st>>>(maps, g);
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2, attr[0].val.clusterDim.y = 1, attr[0].val.clusterDim.z = 1;
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof(cfg));
+  cfg.blockDim = dim3(kGemmThreads, 1, 1);
+  cfg.dynamicSmemBytes = kSmemBytes;
+  cfg.stream = st;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  int pairs = n_sm / 2;
+  cfg.gridDim = dim3(2 * pairs, 1, 1);
+  int resident = 0;
+  if (cudaOccupancyMaxActiveClusters(&resident, k_lm_head<kMode>, &cfg) == cudaSuccess && resident > 0 &&
+      resident < pairs)
+    pairs = resident;
+  if (items < pairs) pairs = (int)(items > 0 ? items : 1);
+  cfg.gridDim = dim3(2 * pairs, 1, 1);
+  if (cudaLaunchKernelEx(&cfg, k_lm_head<kMode>, maps, g) != cudaSuccess) return ATGRPO_ERR_CUDA;
   return launch_ok();
 }
 
@@ -676,16 +710,14 @@ int lm_head_fwd_launch(const LmHeadProblem& p, float* lse, float* logp, void* wo
   Maps maps;
   if (!make_map(&maps.a, p.A_rows, p.d, p.rows_bound, p.ldA, BK, BM)) return ATGRPO_ERR_CUDA;
   for (int m = 0; m < p.M; ++m)
-    if (!make_map(&maps.b[m], p.W[m], p.d, p.V, p.d, BK, BN)) return ATGRPO_ERR_CUDA;
+    if (!make_map(&maps.b[m], p.W[m], p.d, p.V, p.d, BK, BN / 2)) return ATGRPO_ERR_CUDA;
   GemmArgs g = base_args(p);
   g.v_begin = 0, g.n_vtiles = pl.n_vt, g.tiles_per_chunk = pl.tiles_per_chunk, g.n_chunks = pl.n_chunks;
-  g.m_block = row_block_tiles(p.T_pad / BM, p.d);
+  g.m_block = row_block_tiles(p.T_pad / kPairRows, p.d);
   g.part_m = reinterpret_cast<float*>(ws + pl.part_m);
   g.part_s = reinterpret_cast<float*>(ws + pl.part_s);
   g.zt = reinterpret_cast<float*>(ws + pl.zt);
-  const int64_t items = (p.T_pad / BM) * pl.n_chunks;
-  const int grid = (int)(items < p.n_sm ? (items > 0 ? items : 1) : p.n_sm);
-  int rc = launch_gemm<kFwd>(maps, g, grid, st);
+  int rc = launch_gemm<kFwd>(maps, g, (p.T_pad / kPairRows) * pl.n_chunks, p.n_sm, st);
   if (rc != ATGRPO_OK) return rc;
   const int cgrid = (int)((p.T_pad + 255) / 256 > 0 ? (p.T_pad + 255) / 256 : 1);
   k_lse_combine<<<cgrid, 256, 0, st>>>(p.sched, p.M, p.tok_of_row, p.T_pad, pl.n_chunks, g.part_m,
@@ -713,10 +745,10 @@ int lm_head_bwd_launch(const LmHeadProblem& p, const float* lse, const float* co
   if (!make_map(&m_dw.a, dz, pl.vc, p.T_pad, pl.vc, 64, 64)) return ATGRPO_ERR_CUDA;
   if (!make_map(&m_dw.b[0], p.A_rows, p.d, p.rows_bound, p.ldA, 64, 64)) return ATGRPO_ERR_CUDA;
   for (int m = 0; m < p.M; ++m) {
-    if (!make_map(&m_dz.b[m], p.W[m], p.d, p.V, p.d, BK, BN)) return ATGRPO_ERR_CUDA;
+    if (!make_map(&m_dz.b[m], p.W[m], p.d, p.V, p.d, BK, BN / 2)) return ATGRPO_ERR_CUDA;
     if (!make_map(&m_dh.b[m], p.W[m], p.d, p.V, p.d, 64, 64)) return ATGRPO_ERR_CUDA;
   }
-  const int64_t n_mt = p.T_pad / BM;
+  const int64_t n_pt = p.T_pad / kPairRows;
   const int n_dt = (p.d + BN - 1) / BN;
   int chunk = 0;
   for (int v_begin = 0; v_begin < p.V; v_begin += pl.vc, ++chunk) {
@@ -726,20 +758,17 @@ int lm_head_bwd_launch(const LmHeadProblem& p, const float* lse, const float* co
     g.vc_valid = p.V - v_begin < pl.vc ? p.V - v_begin : pl.vc;
     g.n_vtiles = (g.vc_valid + BN - 1) / BN;
     g.tiles_per_chunk = 1;
-    g.m_block = row_block_tiles(n_mt, p.d);
+    g.m_block = row_block_tiles(n_pt, p.d);
     g.n_chunks = g.n_vtiles;
     g.lse = lse, g.coef = coef, g.dz = dz;
     g.dh_acc = dh_acc, g.first_chunk = chunk == 0;
     for (int m = 0; m < p.M; ++m) g.dW[m] = dW[m];
     g.dw_bf16 = prm.dW_dtype == ATGRPO_BF16, g.dw_accumulate = prm.accumulate_dW;
-    auto grid_for = [&](int64_t items) {
-      return (int)(items < p.n_sm ? (items > 0 ? items : 1) : p.n_sm);
-    };
-    int rc = launch_gemm<kDz>(m_dz, g, grid_for(n_mt * g.n_vtiles), st);
+    int rc = launch_gemm<kDz>(m_dz, g, n_pt * g.n_vtiles, p.n_sm, st);
     if (rc != ATGRPO_OK) return rc;
-    rc = launch_gemm<kDh>(m_dh, g, grid_for(n_mt * n_dt), st);
+    rc = launch_gemm<kDh>(m_dh, g, n_pt * n_dt, p.n_sm, st);
     if (rc != ATGRPO_OK) return rc;
-    rc = launch_gemm<kDw>(m_dw, g, grid_for((int64_t)p.M * ((g.vc_valid + BM - 1) / BM) * n_dt), st);
+    rc = launch_gemm<kDw>(m_dw, g, (int64_t)p.M * ((g.vc_valid + kPairRows - 1) / kPairRows) * n_dt, p.n_sm, st);
     if (rc != ATGRPO_OK) return rc;
   }
   if (!dH_direct) {

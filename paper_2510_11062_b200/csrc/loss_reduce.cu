@@ -282,7 +282,7 @@ k_route_scan(int M, int nb, const int32_t* blk_cnt, int32_t* blk_off, Schedule* 
       sched->rows[m] = rows;
       sched->role_offsets[m] = s_head_begin[m];
       if (role_offsets_out) role_offsets_out[m] = s_head_begin[m];
-      tile += (rows + 127) / 128;
+      tile += ((rows + 127) / 128 + 1) & ~1;      // whole 256-row pair tiles per head
     }
     sched->tile_begin[M] = tile;
     sched->role_offsets[M] = s_head_begin[M];
@@ -333,7 +333,7 @@ __global__ void k_route_single(int64_t T, int64_t T_pad, Schedule* sched, int32_
   if (blockIdx.x == 0 && threadIdx.x == 0) {
     sched->n_heads = 1;
     sched->tile_begin[0] = 0;
-    for (int m = 1; m <= ATGRPO_MAX_HEADS; ++m) sched->tile_begin[m] = (int)((T + 127) / 128);
+    for (int m = 1; m <= ATGRPO_MAX_HEADS; ++m) sched->tile_begin[m] = (int)((T + 255) / 256) * 2;
     sched->rows[0] = (int)T;
     sched->role_offsets[0] = 0;
     sched->role_offsets[1] = (int)T;
