@@ -218,6 +218,7 @@ k_lm_head(const __grid_constant__ Maps maps, const GemmArgs g) {
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
+      const uint64_t keep = l2_policy_evict_last();
       for (int it = pair; ok && it < n_items; it += n_pairs) {
         const Tile t = decode_item<kMode>(g, sched, it, rank);
         for (int nt = t.nt_begin; ok && nt < t.nt_end; ++nt) {
@@ -228,20 +229,20 @@ k_lm_head(const __grid_constant__ Maps maps, const GemmArgs g) {
             const uint32_t fb = mapa_shared(full_bar(stage), 0);             // the leader's barrier
             if (rank == 0) mbar_expect_tx(full_bar(stage), 2 * kStageBytes);
             if (kMode == kFwd || kMode == kDz) {
-              tma_load_2d_pair(sa, &maps.a, ks * BK, t.row0, fb);
+              tma_load_2d_pair_hint(sa, &maps.a, ks * BK, t.row0, fb, keep);          // rows of H: re-read per W tile
               tma_load_2d_pair(sb, &maps.b[t.head], ks * BK, n0, fb);
             } else if (kMode == kDh) {
-              tma_load_2d_pair(sa, &maps.a, ks * BK, t.row0, fb);
+              tma_load_2d_pair(sa, &maps.a, ks * BK, t.row0, fb);                      // dZ: shared by the d tiles
 #pragma unroll
-              for (int b = 0; b < 2; ++b)
-                tma_load_2d_pair(sb + b * kBoxBytes, &maps.b[t.head], n0 + 64 * b, g.v_begin + ks * BK, fb);
+              for (int b = 0; b < 2; ++b)                                             // W chunk: re-read per wave
+                tma_load_2d_pair_hint(sb + b * kBoxBytes, &maps.b[t.head], n0 + 64 * b, g.v_begin + ks * BK, fb, keep);
             } else {
 #pragma unroll
               for (int b = 0; b < 2; ++b)
                 tma_load_2d_pair(sa + b * kBoxBytes, &maps.a, t.v0 + 64 * b, t.row0 + ks * BK, fb);
 #pragma unroll
-              for (int b = 0; b < 2; ++b)
-                tma_load_2d_pair(sb + b * kBoxBytes, &maps.b[0], n0 + 64 * b, t.row0 + ks * BK, fb);
+              for (int b = 0; b < 2; ++b)                                             // H: re-read per wave
+                tma_load_2d_pair_hint(sb + b * kBoxBytes, &maps.b[0], n0 + 64 * b, t.row0 + ks * BK, fb, keep);
             }
             if (++stage == kStages) stage = 0, phase ^= 1u;
           }
@@ -584,9 +585,10 @@ int fwd_chunks(int64_t n_mt, int n_vt, int n_sm) {
 }
 
 // Pair tiles (256 rows) per block of the logits sweeps: as many as keep the block's rows of H
-// within about half of the 126 MB L2.
+// within a quarter of the 126 MB L2 (the L2 is split over two dies, and rows read from both
+// sides occupy space in each half).
 int row_block_tiles(int64_t n_pt, int d) {
-  int64_t gm = (64ll << 20) / ((int64_t)kPairRows * d * 2);
+  int64_t gm = (32ll << 20) / ((int64_t)kPairRows * d * 2);
   if (gm < 1) gm = 1;
   if (gm > n_pt) gm = n_pt > 0 ? n_pt : 1;
   return (int)gm;
