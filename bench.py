@@ -28,9 +28,16 @@ sys.path.insert(0, ROOT)
 
 from paper_2510_11062_b200 import workloads as WL  # noqa: E402
 
+# DRAM bytes (read + write) of ONE forward-sweep launch, from a 1-pass ncu capture of
+#   ncu --metrics dram__bytes_read.sum,dram__bytes_write.sum --clock-control none -k regex:k_lm_head
+#       --launch-skip 1 --launch-count 4 python bench.py --steps 1 --warmup 3 --no-cpu-baseline
+# (profiles/k_lm_head_qwen3_1p7b_dram_traffic.txt).  Valid for the kernel as captured; set the entry
+# to None when k_lm_head<kFwd> or its tiling changes.
+FWD_SWEEP_DRAM_BYTES = {"qwen3_1p7b": 1.93e9 + 17.1e6}
+
 METRIC = "fused AT-GRPO loss fwd+bwd tokens/sec"
 UNIT = "tokens/s"
-CPU_SAMPLE_TOKENS = 1024
+CPU_SAMPLE_TOKENS = 2048
 
 
 def measured_peaks():
@@ -341,7 +348,9 @@ def run_ours(args):
         phases_ms=dict(advantages=adv_ms, forward=fwd_ms, backward=bwd_ms),
         roofline=dict(bound="tensor", kernel="k_lm_head<kFwd> (forward call: routing + logits/logsumexp sweep "
                       "+ combine + Eq. 2 reduction)", achieved=fwd_tf, peak=peaks["bf16_sustained"],
-                      unit="TFLOP/s", frac=fwd_tf / peaks["bf16_sustained"], traffic=None,
+                      unit="TFLOP/s", frac=fwd_tf / peaks["bf16_sustained"],
+                      traffic=FWD_SWEEP_DRAM_BYTES.get(spec.name) if world == 1 else None,
+                      algorithmic_bytes=2.0 * spec.d * (spec.V * spec.n_heads + r.T),
                       peak_source=peaks["source"] + " sustained cuBLAS bf16",
                       flops_per_launch=pass_flops,
                       backward_executed_tflops=bwd_tf, backward_frac=bwd_tf / peaks["bf16_sustained"],

@@ -199,9 +199,10 @@ int atgrpo_policy_loss_fwd(
  *   dH[j, :]   = sum_v dZ_jv * W_m[v, :]          -> dH [T, d], row stride d, params->dH_dtype
  *   dW[m][v,:] = sum_{j of policy m} dZ_jv*H[j,:] -> dW[m] [V, d] contiguous, params->dW_dtype,
  *                overwritten or accumulated into (params->accumulate_dW).
- * dW is a HOST array of M device pointers.  A policy without tokens gets dW = 0 (or is left
- * unchanged when accumulating).  The [T, V] logits and their gradient are never materialised:
- * dZ lives in a bounded vocabulary-chunk buffer inside the workspace.
+ * dW is a HOST array of M device pointers; dH and every dW[m] must be 32-byte aligned.
+ * A policy without tokens gets dW = 0 (or is left unchanged when accumulating).  The [T, V]
+ * logits and their gradient are never materialised: dZ lives in a bounded vocabulary-chunk
+ * buffer inside the workspace.
  * ------------------------------------------------------------------------------------------ */
 int atgrpo_policy_loss_bwd(
     const void* H, int64_t ldH, const void* const* W /* host array */, int32_t M,

@@ -213,8 +213,8 @@ int atgrpo_policy_loss_bwd(const void* H, int64_t ldH, const void* const* W, int
   if (rc != ATGRPO_OK) return rc;
   if (dW == nullptr) return ATGRPO_ERR_INVALID_ARG;
   for (int m = 0; m < M; ++m)
-    if (dW[m] == nullptr || !aligned(dW[m], 16)) return ATGRPO_ERR_INVALID_ARG;
-  if (T > 0 && (logp == nullptr || lse == nullptr || dH == nullptr || !aligned(dH, 16)))
+    if (dW[m] == nullptr || !aligned(dW[m], 32)) return ATGRPO_ERR_INVALID_ARG;
+  if (T > 0 && (logp == nullptr || lse == nullptr || dH == nullptr || !aligned(dH, 32)))
     return ATGRPO_ERR_INVALID_ARG;
   int n_sm = 0, cc = 0;
   if (device_sm_count(&n_sm, &cc) != ATGRPO_OK) return ATGRPO_ERR_CUDA;

@@ -86,6 +86,13 @@ __device__ __forceinline__ void st_global_v8(void* p, const uint32_t* v) {
                : "memory");
 }
 
+__device__ __forceinline__ void ld_global_v8(const void* p, uint32_t* v) {
+  asm volatile("ld.global.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+               : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
+               : "l"(p)
+               : "memory");
+}
+
 struct Tile {
   int head;
   int row0;        // first padded row (kFwd/kDz/kDh) or first K row (kDw)
@@ -424,17 +431,21 @@ k_lm_head(const __grid_constant__ Maps maps, const GemmArgs g) {
             float* dst = (kMode == kDh ? g.dh_acc : static_cast<float*>(g.dW[t.head])) +
                          out_row * g.d + col0;
             const bool add = kMode == kDh ? !g.first_chunk : (g.dw_accumulate != 0);
+            // 32 bytes per lane and instruction (d is a multiple of 8, rows are 32-byte aligned)
 #pragma unroll
-            for (int q4 = 0; q4 < 8; ++q4) {
-              if (col0 + 4 * q4 < g.d) {
-                float4 v4 = make_float4(__uint_as_float(r[4 * q4]), __uint_as_float(r[4 * q4 + 1]),
-                                        __uint_as_float(r[4 * q4 + 2]), __uint_as_float(r[4 * q4 + 3]));
-                float4* p4 = reinterpret_cast<float4*>(dst) + q4;
+            for (int q8 = 0; q8 < 4; ++q8) {
+              if (col0 + 8 * q8 < g.d) {
+                uint32_t v[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) v[i] = r[8 * q8 + i];
                 if (add) {
-                  const float4 o = *p4;
-                  v4.x += o.x, v4.y += o.y, v4.z += o.z, v4.w += o.w;
+                  uint32_t o[8];
+                  ld_global_v8(dst + 8 * q8, o);
+#pragma unroll
+                  for (int i = 0; i < 8; ++i)
+                    v[i] = __float_as_uint(__uint_as_float(v[i]) + __uint_as_float(o[i]));
                 }
-                *p4 = v4;
+                st_global_v8(dst + 8 * q8, v);
               }
             }
           } else {
