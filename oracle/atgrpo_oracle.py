@@ -16,6 +16,9 @@ paper (arXiv 2510.11062) in the paper's order and notation:
   clipped_objective    Eq. 2, per token (token-level credit, Sec. 4.1 "Reward Mask")
   policy_loss          Eq. 2, one loss per policy m
   policy_loss_grads    gradient of Eq. 2 w.r.t. the hidden states H and the head W_m
+  grad_sumsq, clip_scale, adamw_step
+                       the update theta_m <- theta_m - eta*grad L of Sec. 3 with the optimiser
+                       settings of App. "Training Details" (Adam, weight decay, gradient clipping)
 
 Readings taken where the paper is silent (each is pinned by a test, none by the
 paper's own numbers -- the paper prints no worked example):
@@ -27,6 +30,9 @@ paper's own numbers -- the paper prints no worked example):
     mean over all response tokens of policy m's batch.
   * hash(e, i, t) is the collision-free mixed-radix index (e*N + i)*T + t.
   * no KL, entropy or temperature term (entropy coefficient 0, T_sample 1).
+  * "Adam ... weight decay 0.01 ... gradient clipping at 1.0" is read as AdamW (decoupled decay,
+    Loshchilov & Hutter) with bias correction, after scaling the gradient by
+    min(1, max_norm / (global L2 norm + 1e-6)).
 Parity status: every function below is pinned by tests/test_oracle_pins.py
 against closed forms, invariants, brute force, finite differences or an
 independent library routine.  The *readings* above (std convention, eps
@@ -40,7 +46,7 @@ import numpy as np
 __all__ = [
     "group_key", "bucket_by_key", "group_advantages", "route_tokens",
     "token_logprobs", "clipped_objective", "policy_loss", "dloss_dlogp", "policy_loss_grads",
-    "policy_loss_grad_rows",
+    "policy_loss_grad_rows", "grad_sumsq", "clip_scale", "adamw_step",
 ]
 
 
@@ -268,3 +274,33 @@ def policy_loss_grad_rows(H, W, target, lse, coef, token_rows=None, vocab_rows=N
         dz += c[:, None] * (y[:, None] == vs[None, :])
         out_w = dz.T @ Hd
     return out_h, out_w
+
+
+# --------------------------------------------------------------------------- parameter update
+def grad_sumsq(grads):
+    """Sum of squares of one policy's gradient tensors (the square of its global L2 norm)."""
+    return float(sum((_f64(g) ** 2).sum() for g in grads))
+
+
+def clip_scale(sumsq, max_norm):
+    """Gradient clipping at max_norm: factor min(1, max_norm / (||g|| + 1e-6)); max_norm <= 0 = off."""
+    if max_norm is None or max_norm <= 0:
+        return 1.0
+    return min(1.0, max_norm / (np.sqrt(sumsq) + 1e-6))
+
+
+def adamw_step(theta, m, v, grad, step, lr=1e-6, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.01,
+               scale=1.0):
+    """One AdamW step on one tensor (all float64): returns (theta, m, v) after step number `step` >= 1.
+
+      g = scale * grad
+      m = beta1*m + (1-beta1)*g            v = beta2*v + (1-beta2)*g^2
+      theta = theta*(1 - lr*weight_decay) - lr * (m/(1-beta1^step)) / (sqrt(v/(1-beta2^step)) + eps)
+    """
+    theta, m, v, g = _f64(theta), _f64(m), _f64(v), _f64(grad) * scale
+    m = beta1 * m + (1.0 - beta1) * g
+    v = beta2 * v + (1.0 - beta2) * g * g
+    m_hat = m / (1.0 - beta1 ** step)
+    v_hat = v / (1.0 - beta2 ** step)
+    theta = theta * (1.0 - lr * weight_decay) - lr * m_hat / (np.sqrt(v_hat) + eps)
+    return theta, m, v

@@ -336,3 +336,38 @@ def test_clipped_and_zero_advantage_tokens_have_zero_dH():
     assert (~active).any() and active.any()
     assert (dH[~active] == 0.0).all()
     assert (np.abs(dH[active]).sum(1) > 0).all()
+
+
+# ----------------------------------------------------------------------------- parameter update
+def test_adamw_matches_torch_optimizer_over_several_steps():
+    g = torch.Generator().manual_seed(5)
+    theta = torch.randn(37, 11, dtype=torch.float64, generator=g)
+    p = theta.clone().requires_grad_()
+    opt = torch.optim.AdamW([p], lr=3e-3, betas=(0.8, 0.95), eps=1e-7, weight_decay=0.05)
+    th, m, v = theta.numpy().copy(), np.zeros((37, 11)), np.zeros((37, 11))
+    for step in range(1, 6):
+        grad = torch.randn(37, 11, dtype=torch.float64, generator=g) * (10.0 if step == 3 else 0.1)
+        total = float(grad.norm())
+        p.grad = grad.clone()
+        torch.nn.utils.clip_grad_norm_([p], max_norm=1.0)          # independent library routine
+        opt.step()
+        scale = O.clip_scale(O.grad_sumsq([grad.numpy()]), 1.0)
+        assert scale == pytest.approx(min(1.0, 1.0 / (total + 1e-6)), rel=1e-12)
+        th, m, v = O.adamw_step(th, m, v, grad.numpy(), step, lr=3e-3, beta1=0.8, beta2=0.95, eps=1e-7,
+                                weight_decay=0.05, scale=scale)
+        np.testing.assert_allclose(th, p.detach().numpy(), rtol=1e-12, atol=1e-14)
+
+
+def test_adamw_closed_forms():
+    # first step from zero state: update = -lr*sign(g)/(1+eps/|g|) - lr*wd*theta
+    th, m, v = O.adamw_step(np.array([2.0, -3.0]), np.zeros(2), np.zeros(2), np.array([0.5, -4.0]), 1, lr=0.1,
+                            beta1=0.9, beta2=0.999, eps=0.0, weight_decay=0.1)
+    np.testing.assert_allclose(th, [2.0 * 0.99 - 0.1, -3.0 * 0.99 + 0.1], rtol=1e-12)
+    np.testing.assert_allclose(m, [0.05, -0.4], rtol=1e-12)
+    np.testing.assert_allclose(v, [0.00025, 0.016], rtol=1e-12)
+    # zero gradient: only the decoupled decay acts
+    th, m, v = O.adamw_step(np.array([1.0]), np.zeros(1), np.zeros(1), np.zeros(1), 1, lr=0.5, weight_decay=0.2)
+    assert th[0] == pytest.approx(0.9) and m[0] == 0 and v[0] == 0
+    assert O.clip_scale(4.0, 0.0) == 1.0 and O.clip_scale(0.25, 1.0) == 1.0
+    assert O.clip_scale(16.0, 1.0) == pytest.approx(1.0 / (4.0 + 1e-6))
+    assert O.grad_sumsq([np.array([3.0, 4.0]), np.array([[12.0]])]) == pytest.approx(169.0)
