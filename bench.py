@@ -425,16 +425,64 @@ def run_stress(args):
     print(json.dumps(line), flush=True)
 
 
+def run_adamw(args):
+    """Memory-bound update of one Qwen3-1.7B-shaped head (V*d = 311 M parameters): gradient sum of
+    squares + clipped AdamW step; 4 B (norm pass) + 30 B (update pass) per parameter with fp32 dW."""
+    from paper_2510_11062_b200 import atgrpo as A
+    A.lib()
+    dev = torch.device("cuda", int(os.environ.get("LOCAL_RANK", "0")))
+    torch.cuda.set_device(dev)
+    n = 151936 * 2048
+    g = torch.Generator(device=dev).manual_seed(1)
+    grad = torch.randn(n, device=dev, generator=g) * 1e-3
+    master = torch.randn(n, device=dev, generator=g) * 0.02
+    m, v = torch.zeros(n, device=dev), torch.zeros(n, device=dev)
+    w = torch.empty(n, dtype=torch.bfloat16, device=dev)
+    sumsq = torch.zeros(1, dtype=torch.float64, device=dev)
+    ws = A.workspace(A.atgrpo_grad_sumsq_workspace_bytes(), dev)
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    t_norm, t_step = [], []
+    sampler = ClockSampler(dev.index or 0)
+    for i in range(max(args.warmup, 3) + args.steps):
+        a, b, c = ev(), ev(), ev()
+        a.record()
+        A.atgrpo_grad_sumsq(grad, sumsq, ws)
+        b.record()
+        A.atgrpo_adamw_step(grad, master, m, v, w, sumsq, A.AdamWParams(step=i + 1))
+        c.record()
+        torch.cuda.synchronize()
+        if i >= max(args.warmup, 3):
+            t_norm.append(a.elapsed_time(b)), t_step.append(b.elapsed_time(c))
+    clocks = sampler.stop()
+    peaks = measured_peaks()
+    ms_n, ms_s = statistics.median(t_norm), statistics.median(t_step)
+    gbs = 30.0 * n / (ms_s * 1e-3) / 1e9
+    line = dict(metric="AdamW head update HBM GB/s (30 B per parameter)", value=gbs, unit="GB/s", n_gpus=1,
+                steps=args.steps, warmup=max(args.warmup, 3), ms_per_step=ms_n + ms_s, higher_is_better=True,
+                scaling="weak", vs_baseline=None, dtype="f32", data="synthetic",
+                config=dict(workload="adamw", parameters=n, l2="arrays larger than L2 (5.6 GB touched per step)"),
+                gpu_launches=2 * args.steps,
+                roofline=dict(bound="hbm", kernel="k_adamw", achieved=gbs, peak=peaks["hbm_gbs"], unit="GB/s",
+                              frac=gbs / peaks["hbm_gbs"], traffic=None,
+                              peak_source=peaks["source"] + " copy bandwidth"),
+                grad_norm=dict(ms=ms_n, gbs=4.0 * n / (ms_n * 1e-3) / 1e9,
+                               frac=4.0 * n / (ms_n * 1e-3) / 1e9 / peaks["hbm_gbs"]),
+                clocks=clocks)
+    print(json.dumps(line), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--workload", default="qwen3_1p7b", choices=sorted(WL.SPECS) + ["stress", "stress16"])
+    ap.add_argument("--workload", default="qwen3_1p7b", choices=sorted(WL.SPECS) + ["stress", "stress16", "adamw"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
-    if args.workload.startswith("stress"):
+    if args.workload == "adamw":
+        run_adamw(args)
+    elif args.workload.startswith("stress"):
         run_stress(args)
     elif args.impl == "reference":
         run_reference(args)

@@ -214,6 +214,42 @@ int atgrpo_policy_loss_bwd(
     void* dH, void* const* dW /* host array */,
     int32_t* device_status, void* workspace, size_t workspace_bytes, void* stream);
 
+/* ------------------------------------------------------------------------------------------
+ * Parameter update of one policy's LM head -- theta_m <- theta_m - eta * grad L(theta_m) (Sec. 3)
+ * with the optimiser settings of App. "Training Details": gradient clipping at a global L2 norm,
+ * Adam with weight decay (read as AdamW: decoupled decay, bias-corrected moments).
+ *
+ * atgrpo_grad_sumsq: sumsq[0] = sum of squares of the n gradient elements (fp64, device), summed
+ * in a fixed order.  The caller may add the squared norm of the policy's other parameters (the
+ * transformer trunk is not in this library) before passing it on.
+ *
+ * atgrpo_adamw_step, for step number `step` >= 1, per element:
+ *   g = grad * min(1, max_grad_norm / (sqrt(*grad_sumsq) + 1e-6))    (no clipping if grad_sumsq is
+ *                                                                      NULL or max_grad_norm <= 0)
+ *   m = beta1*m + (1-beta1)*g          v = beta2*v + (1-beta2)*g*g
+ *   master = master*(1 - lr*weight_decay) - lr*(m/(1-beta1^step)) / (sqrt(v/(1-beta2^step)) + eps)
+ *   w_bf16 = bf16(master)              (optional output, NULL to skip: the head the loss kernels read)
+ * grad has grad_dtype (ATGRPO_F32 or ATGRPO_BF16); master, m, v are fp32 and updated in place.
+ * All arrays hold n elements and are 16-byte aligned.  fp32 arithmetic.
+ * ------------------------------------------------------------------------------------------ */
+typedef struct atgrpo_adamw_params {
+  float lr;            /* 1e-6 in the paper */
+  float beta1, beta2;  /* not given in the paper; 0.9, 0.999 are the usual defaults */
+  float eps;           /* 1e-8 */
+  float weight_decay;  /* 0.01 in the paper */
+  float max_grad_norm; /* 1.0 in the paper */
+  int32_t step;        /* 1-based step count */
+} atgrpo_adamw_params;
+
+size_t atgrpo_grad_sumsq_workspace_bytes(void);
+
+int atgrpo_grad_sumsq(const void* grad, int32_t grad_dtype, int64_t n, double* sumsq,
+                      void* workspace, size_t workspace_bytes, void* stream);
+
+int atgrpo_adamw_step(const void* grad, int32_t grad_dtype, float* master, float* m, float* v,
+                      void* w_bf16, int64_t n, const double* grad_sumsq,
+                      const atgrpo_adamw_params* params /* host */, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -27,6 +27,7 @@ EXPORTS = (
     "atgrpo_clipped_loss_workspace_bytes", "atgrpo_clipped_loss",
     "atgrpo_policy_loss_workspace_bytes", "atgrpo_policy_loss_launch_count",
     "atgrpo_policy_loss_fwd", "atgrpo_policy_loss_bwd",
+    "atgrpo_grad_sumsq_workspace_bytes", "atgrpo_grad_sumsq", "atgrpo_adamw_step",
 )
 
 
@@ -39,6 +40,27 @@ class _Params(ctypes.Structure):
                 ("std_eps", ctypes.c_float), ("ddof", ctypes.c_int32),
                 ("dH_dtype", ctypes.c_int32), ("dW_dtype", ctypes.c_int32),
                 ("accumulate_dW", ctypes.c_int32)]
+
+
+class _AdamWParams(ctypes.Structure):
+    _fields_ = [("lr", ctypes.c_float), ("beta1", ctypes.c_float), ("beta2", ctypes.c_float),
+                ("eps", ctypes.c_float), ("weight_decay", ctypes.c_float), ("max_grad_norm", ctypes.c_float),
+                ("step", ctypes.c_int32)]
+
+
+@dataclass
+class AdamWParams:
+    lr: float = 1e-6
+    beta1: float = 0.9
+    beta2: float = 0.999
+    eps: float = 1e-8
+    weight_decay: float = 0.01
+    max_grad_norm: float = 1.0
+    step: int = 1
+
+    def c(self) -> _AdamWParams:
+        return _AdamWParams(self.lr, self.beta1, self.beta2, self.eps, self.weight_decay, self.max_grad_norm,
+                            self.step)
 
 
 @dataclass
@@ -94,6 +116,12 @@ def lib() -> ctypes.CDLL:
         L.atgrpo_policy_loss_bwd.argtypes = [vp, i64, ctypes.POINTER(vp), i32, vp, vp, vp, i32, vp, vp,
                                              i64, vp, vp, vp, vp, i64, i32, i32, pp, vp,
                                              ctypes.POINTER(vp), vp, vp, sz, vp]
+        L.atgrpo_grad_sumsq_workspace_bytes.restype = sz
+        L.atgrpo_grad_sumsq_workspace_bytes.argtypes = []
+        L.atgrpo_grad_sumsq.restype = ctypes.c_int
+        L.atgrpo_grad_sumsq.argtypes = [vp, i32, i64, vp, vp, sz, vp]
+        L.atgrpo_adamw_step.restype = ctypes.c_int
+        L.atgrpo_adamw_step.argtypes = [vp, i32, vp, vp, vp, vp, i64, vp, ctypes.POINTER(_AdamWParams), vp]
         _lib = L
     return _lib
 
@@ -239,3 +267,25 @@ def atgrpo_policy_loss_bwd(H, W, target, role_of_token, head_of_role, resp_of_to
         _ptr(dH, dh_t), _ptr_array(dW, dw_t), _ptr(device_status, i32), _ptr(workspace),
         workspace.numel(), _stream())
     _check(rc, "atgrpo_policy_loss_bwd")
+
+
+def atgrpo_grad_sumsq_workspace_bytes() -> int:
+    return int(lib().atgrpo_grad_sumsq_workspace_bytes())
+
+
+def atgrpo_grad_sumsq(grad, sumsq, workspace):
+    """sumsq[0] (float64, device) = sum of squares of `grad` (fp32 or bf16); see include/atgrpo.h."""
+    dt = BF16 if grad.dtype == torch.bfloat16 else F32
+    rc = lib().atgrpo_grad_sumsq(_ptr(grad), dt, grad.numel(), _ptr(sumsq, torch.float64), _ptr(workspace),
+                                 workspace.numel(), _stream())
+    _check(rc, "atgrpo_grad_sumsq")
+
+
+def atgrpo_adamw_step(grad, master, m, v, w_bf16, grad_sumsq, params: AdamWParams):
+    """Clipped AdamW step on one head, in place on master / m / v; see include/atgrpo.h."""
+    f32 = torch.float32
+    dt = BF16 if grad.dtype == torch.bfloat16 else F32
+    rc = lib().atgrpo_adamw_step(_ptr(grad), dt, _ptr(master, f32), _ptr(m, f32), _ptr(v, f32),
+                                 _ptr(w_bf16, torch.bfloat16), master.numel(),
+                                 _ptr(grad_sumsq, torch.float64), ctypes.byref(params.c()), _stream())
+    _check(rc, "atgrpo_adamw_step")

@@ -255,4 +255,33 @@ int atgrpo_policy_loss_bwd(const void* H, int64_t ldH, const void* const* W, int
   return lm_head_bwd_launch(p, lse, coef, row_of_token, *params, dH, dW, ws + pl.gemm, st);
 }
 
+size_t atgrpo_grad_sumsq_workspace_bytes(void) { return grad_sumsq_workspace_bytes(); }
+
+int atgrpo_grad_sumsq(const void* grad, int32_t grad_dtype, int64_t n, double* sumsq, void* workspace,
+                      size_t workspace_bytes, void* stream) {
+  if (n < 0 || sumsq == nullptr || (grad_dtype != ATGRPO_F32 && grad_dtype != ATGRPO_BF16))
+    return ATGRPO_ERR_INVALID_ARG;
+  if (n > 0 && (grad == nullptr || !aligned(grad, 16))) return ATGRPO_ERR_INVALID_ARG;
+  if (workspace == nullptr || !aligned(workspace, 256) || workspace_bytes < grad_sumsq_workspace_bytes())
+    return ATGRPO_ERR_WORKSPACE;
+  return grad_sumsq_launch(grad, grad_dtype, n, sumsq, workspace, static_cast<cudaStream_t>(stream));
+}
+
+int atgrpo_adamw_step(const void* grad, int32_t grad_dtype, float* master, float* m, float* v,
+                      void* w_bf16, int64_t n, const double* grad_sumsq,
+                      const atgrpo_adamw_params* p, void* stream) {
+  if (p == nullptr || n < 0 || (grad_dtype != ATGRPO_F32 && grad_dtype != ATGRPO_BF16))
+    return ATGRPO_ERR_INVALID_ARG;
+  if (p->step < 1 || !(p->beta1 >= 0.f && p->beta1 < 1.f) || !(p->beta2 >= 0.f && p->beta2 < 1.f) ||
+      !(p->eps >= 0.f) || !(p->lr >= 0.f) || !(p->weight_decay >= 0.f))
+    return ATGRPO_ERR_INVALID_ARG;
+  if (n == 0) return ATGRPO_OK;
+  if (grad == nullptr || master == nullptr || m == nullptr || v == nullptr) return ATGRPO_ERR_INVALID_ARG;
+  if (!aligned(grad, 16) || !aligned(master, 16) || !aligned(m, 16) || !aligned(v, 16) ||
+      (w_bf16 != nullptr && !aligned(w_bf16, 16)))
+    return ATGRPO_ERR_INVALID_ARG;
+  return adamw_launch(grad, grad_dtype, master, m, v, w_bf16, n, grad_sumsq, p->lr, p->beta1, p->beta2,
+                      p->eps, p->weight_decay, p->max_grad_norm, p->step, static_cast<cudaStream_t>(stream));
+}
+
 }  // extern "C"

@@ -48,6 +48,14 @@ int routing_launch(const int32_t* role_of_token, const int32_t* head_of_role, in
 int gather_rows_launch(const void* H, int64_t ldH, const int32_t* tok_of_row, int64_t T_pad,
                        int32_t d, void* Hs, cudaStream_t st);
 
+// ---- optimizer.cu ---------------------------------------------------------------------------
+size_t grad_sumsq_workspace_bytes();
+int grad_sumsq_launch(const void* grad, int grad_dtype, int64_t n, double* sumsq_out, void* workspace,
+                      cudaStream_t st);
+int adamw_launch(const void* grad, int grad_dtype, float* master, float* m, float* v, void* w_bf16,
+                 int64_t n, const double* sumsq, float lr, float beta1, float beta2, float eps,
+                 float weight_decay, float max_norm, int step, cudaStream_t st);
+
 // ---- lm_head.cu -----------------------------------------------------------------------------
 struct LmHeadProblem {
   const void* A_rows;        // bf16 [rows_total, d] rows in padded order (H itself when M == 1)
