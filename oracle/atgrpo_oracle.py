@@ -14,7 +14,8 @@ paper (arXiv 2510.11062) in the paper's order and notation:
   route_tokens         Sec. 3 "Role-sharing vs. Role-specialized", B_m = U_{sigma(i)=m} D_i
   token_logprobs       pi_theta in Eq. 2: log-softmax of the LM-head logits at the sampled token
   clipped_objective    Eq. 2, per token (token-level credit, Sec. 4.1 "Reward Mask")
-  policy_loss          Eq. 2, one loss per policy m
+  policy_loss          Eq. 2, one loss per policy m (token-level reading)
+  policy_loss_sequence Eq. 2 as printed: one ratio per response, mean over the responses of B_m
   policy_loss_grads    gradient of Eq. 2 w.r.t. the hidden states H and the head W_m
   grad_sumsq, clip_scale, adamw_step
                        the update theta_m <- theta_m - eta*grad L of Sec. 3 with the optimiser
@@ -46,6 +47,7 @@ import numpy as np
 __all__ = [
     "group_key", "bucket_by_key", "group_advantages", "route_tokens",
     "token_logprobs", "clipped_objective", "policy_loss", "dloss_dlogp", "policy_loss_grads",
+    "policy_loss_sequence", "dloss_dlogp_sequence",
     "policy_loss_grad_rows", "grad_sumsq", "clip_scale", "adamw_step",
 ]
 
@@ -214,8 +216,55 @@ def dloss_dlogp(logp, old_logp, adv, resp_of_token, head_of_token, n_heads, grad
     return -(g[head] / denom[head]) * A * r * active
 
 
+def _sequence_terms(logp, old_logp, adv, resp_of_token, head_of_token, eps_low, eps_high):
+    """Per response c that owns at least one token: r_c = pi(o_c|q)/pi_old(o_c|q) =
+    exp(sum_j logp_j - sum_j old_logp_j) over its tokens, the Eq. 2 term, and its policy."""
+    lp, lo = _f64(logp), _f64(old_logp)
+    A_all = _f64(adv)
+    resp, head = _i64(resp_of_token), _i64(head_of_token)
+    ids = np.unique(resp)                                   # responses present in the batch
+    delta = np.array([(lp[resp == c] - lo[resp == c]).sum() for c in ids])
+    head_c = np.array([head[np.nonzero(resp == c)[0][0]] for c in ids], dtype=np.int64)
+    term, r, active = clipped_objective(delta, np.zeros_like(delta), A_all[ids], eps_low, eps_high)
+    return ids, head_c, term, r, active
+
+
+def policy_loss_sequence(logp, old_logp, adv, resp_of_token, head_of_token, n_heads,
+                         eps_low=0.2, eps_high=0.2):
+    """Eq. 2 read literally: L_m = -(1/R_m) sum_{responses c of policy m} min(r_c A_c, clip(r_c) A_c)
+    with the sequence-level ratio r_c; R_m counts the responses of policy m that have tokens.
+    Returns (loss[n_heads], R_m[n_heads], clip_counts[n_heads, 2]) (clip counts per response)."""
+    ids, head_c, term, r, _ = _sequence_terms(logp, old_logp, adv, resp_of_token, head_of_token,
+                                              eps_low, eps_high)
+    loss = np.zeros(n_heads)
+    count = np.zeros(n_heads, dtype=np.int64)
+    cc = np.zeros((n_heads, 2), dtype=np.int64)
+    for m in range(n_heads):
+        sel = head_c == m
+        count[m] = sel.sum()
+        if count[m]:
+            loss[m] = -term[sel].sum() / count[m]
+            cc[m, 0] = (r[sel] < 1.0 - eps_low).sum()
+            cc[m, 1] = (r[sel] > 1.0 + eps_high).sum()
+    return loss, count, cc
+
+
+def dloss_dlogp_sequence(logp, old_logp, adv, resp_of_token, head_of_token, n_heads, grad_loss=None,
+                         eps_low=0.2, eps_high=0.2):
+    """c_j = d(sum_m grad_loss_m L_m)/d logp_j for the sequence-level loss: every token of response c
+    gets -grad_loss_m * A_c * r_c * active_c / R_m (d r_c / d logp_j = r_c)."""
+    ids, head_c, _, r, active = _sequence_terms(logp, old_logp, adv, resp_of_token, head_of_token,
+                                                eps_low, eps_high)
+    resp = _i64(resp_of_token)
+    A_all = _f64(adv)
+    g = np.ones(n_heads) if grad_loss is None else _f64(grad_loss)
+    count = np.bincount(head_c, minlength=n_heads).astype(np.float64)
+    per_resp = {int(c): -(g[h] / count[h]) * A_all[c] * rc * ac for c, h, rc, ac in zip(ids, head_c, r, active)}
+    return np.array([per_resp[int(c)] for c in resp])
+
+
 def policy_loss_grads(H, W_list, target, old_logp, adv, resp_of_token, head_of_token,
-                      grad_loss=None, eps_low=0.2, eps_high=0.2):
+                      grad_loss=None, eps_low=0.2, eps_high=0.2, reduction="token"):
     """Gradient of sum_m grad_loss_m * L_m (Eq. 2) w.r.t. H and every head W_m.
 
     With c_j = dL/dlogp_j and p_jv = softmax(z_j)_v:
@@ -236,7 +285,8 @@ def policy_loss_grads(H, W_list, target, old_logp, adv, resp_of_token, head_of_t
         lse = np.log(np.exp(z - z.max(axis=1, keepdims=True)).sum(axis=1)) + z.max(axis=1)
         P[m] = np.exp(z - lse[:, None])
         logp[sel] = z[np.arange(sel.size), y[sel]] - lse
-    c = dloss_dlogp(logp, old_logp, adv, resp_of_token, head, M, grad_loss, eps_low, eps_high)
+    dl = dloss_dlogp if reduction == "token" else dloss_dlogp_sequence
+    c = dl(logp, old_logp, adv, resp_of_token, head, M, grad_loss, eps_low, eps_high)
     dH = np.zeros_like(Hd)
     dW = []
     for m in range(M):

@@ -371,3 +371,70 @@ def test_adamw_closed_forms():
     assert O.clip_scale(4.0, 0.0) == 1.0 and O.clip_scale(0.25, 1.0) == 1.0
     assert O.clip_scale(16.0, 1.0) == pytest.approx(1.0 / (4.0 + 1e-6))
     assert O.grad_sumsq([np.array([3.0, 4.0]), np.array([[12.0]])]) == pytest.approx(169.0)
+
+
+# ----------------------------------------------------------------------------- sequence-level Eq. 2
+def test_sequence_loss_reduces_to_token_loss_for_one_token_responses():
+    T = 30
+    lp, lo, A = -rng.random(T), -rng.random(T), rng.standard_normal(T)
+    head = rng.integers(0, 2, T)
+    a, ca, cca = O.policy_loss_sequence(lp, lo, A, np.arange(T), head, 2)
+    b, cb, ccb = O.policy_loss(lp, lo, A, np.arange(T), head, 2)
+    np.testing.assert_allclose(a, b, atol=1e-15)
+    assert (ca == cb).all() and (cca == ccb).all()
+    np.testing.assert_allclose(O.dloss_dlogp_sequence(lp, lo, A, np.arange(T), head, 2),
+                               O.dloss_dlogp(lp, lo, A, np.arange(T), head, 2), atol=1e-15)
+
+
+def test_sequence_loss_closed_forms():
+    # two responses of policy 0 (3 and 2 tokens), one of policy 1; response 2 has no token
+    resp = np.array([0, 0, 0, 1, 1, 3])
+    head = np.array([0, 0, 0, 0, 0, 1])
+    adv = np.array([2.0, -1.0, 5.0, 0.5])
+    lo = np.zeros(6)
+    lp = np.array([0.1, 0.2, -0.1, 0.3, 0.2, -0.05])          # r = e^0.2, e^0.5 (clipped: A<0, r>1+eps unclipped), e^-0.05
+    loss, count, cc = O.policy_loss_sequence(lp, lo, adv, resp, head, 2)
+    r0, r1, r3 = np.exp(0.2), np.exp(0.5), np.exp(-0.05)
+    want0 = -(min(r0 * 2.0, 1.2 * 2.0) + min(r1 * -1.0, 1.2 * -1.0)) / 2
+    assert loss[0] == pytest.approx(want0, rel=1e-14) and loss[1] == pytest.approx(-r3 * 0.5, rel=1e-14)
+    assert count.tolist() == [2, 1] and cc.tolist() == [[0, 2], [0, 0]]
+    # ratio 1 everywhere: minus the mean advantage over RESPONSES (not tokens)
+    loss, _, _ = O.policy_loss_sequence(lo, lo, adv, resp, head, 2)
+    assert loss[0] == pytest.approx(-(2.0 - 1.0) / 2) and loss[1] == pytest.approx(-0.5)
+
+
+def test_sequence_gradients_by_finite_differences_and_autograd():
+    T, d, V, R, M = 40, 6, 30, 7, 2
+    g = torch.Generator().manual_seed(23)
+    H = torch.randn(T, d, dtype=torch.float64, generator=g, requires_grad=True)
+    W = [(torch.randn(V, d, dtype=torch.float64, generator=g) * 0.4).requires_grad_() for _ in range(M)]
+    y = torch.randint(0, V, (T,), generator=g)
+    resp = torch.sort(torch.randint(0, R, (T,), generator=g)).values
+    role_of_resp = torch.randint(0, M, (R,), generator=g)
+    head = role_of_resp[resp]
+    adv = torch.randn(R, dtype=torch.float64, generator=g)
+    gl = torch.tensor([1.0, 0.7], dtype=torch.float64)
+    with torch.no_grad():
+        logp0 = torch.stack([torch.log_softmax(H[j] @ W[head[j]].T, 0)[y[j]] for j in range(T)])
+    old = logp0 + torch.randn(T, dtype=torch.float64, generator=g) * 0.08
+    total = 0.0
+    for m in range(M):
+        terms = []
+        for c in torch.unique(resp).tolist():
+            sel = (resp == c).nonzero().squeeze(1)
+            if head[sel[0]] != m:
+                continue
+            lp = torch.log_softmax(H[sel] @ W[m].T, 1)[torch.arange(sel.numel()), y[sel]]
+            r = torch.exp((lp - old[sel]).sum())
+            terms.append(torch.minimum(r * adv[c], torch.clamp(r, 0.8, 1.2) * adv[c]))
+        if terms:
+            total = total + gl[m] * (-torch.stack(terms).mean())
+    total.backward()
+    dH, dW = O.policy_loss_grads(H.detach().numpy(), [w.detach().numpy() for w in W], y.numpy(), old.numpy(),
+                                 adv.numpy(), resp.numpy(), head.numpy(), grad_loss=gl.numpy(),
+                                 reduction="sequence")
+    np.testing.assert_allclose(dH, H.grad.numpy(), atol=1e-13)
+    for m in range(M):
+        np.testing.assert_allclose(dW[m], W[m].grad.numpy(), atol=1e-13)
+    loss, _, _ = O.policy_loss_sequence(logp0.numpy(), old.numpy(), adv.numpy(), resp.numpy(), head.numpy(), M)
+    assert float((torch.from_numpy(loss) * gl).sum()) == pytest.approx(float(total), rel=1e-12)
