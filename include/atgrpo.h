@@ -63,7 +63,18 @@ typedef struct atgrpo_params {
   int32_t dH_dtype;      /* ATGRPO_BF16 (default) or ATGRPO_F32: element type of dH            */
   int32_t dW_dtype;      /* ATGRPO_F32 (default) or ATGRPO_BF16: element type of every dW_m    */
   int32_t accumulate_dW; /* 0: dW_m is overwritten; 1: dW_m += gradient (gradient accumulation)*/
+  int32_t reduction;     /* ATGRPO_REDUCE_TOKEN_MEAN (default) or ATGRPO_REDUCE_SEQUENCE           */
 } atgrpo_params;
+
+/* Readings of the expectation in Eq. 2.
+ * TOKEN_MEAN: one ratio per response token, loss_m = mean over all response tokens of policy m.
+ * SEQUENCE  : Eq. 2 as printed -- one ratio per response, r_c = pi(o_c|q)/pi_old(o_c|q) =
+ *             exp(sum of logp - old_logp over the response's tokens), loss_m = mean over the
+ *             responses of policy m that have tokens; every token of response c then carries
+ *             coef = grad_loss[m]*A_c*r_c*[unclipped branch active]/R_m.  Requires the tokens packed
+ *             response by response (resp_of_token non-decreasing; a violation raises
+ *             ATGRPO_ERR_BAD_INDEX); clip counts are per response. */
+enum { ATGRPO_REDUCE_TOKEN_MEAN = 0, ATGRPO_REDUCE_SEQUENCE = 1 };
 
 /* Text for a status code (static storage, never NULL). */
 const char* atgrpo_status_string(int status);

@@ -13,6 +13,7 @@ bool params_ok(const atgrpo_params* p) {
   if (p->ddof != 0 && p->ddof != 1) return false;
   if (p->dH_dtype != ATGRPO_BF16 && p->dH_dtype != ATGRPO_F32) return false;
   if (p->dW_dtype != ATGRPO_BF16 && p->dW_dtype != ATGRPO_F32) return false;
+  if (p->reduction != ATGRPO_REDUCE_TOKEN_MEAN && p->reduction != ATGRPO_REDUCE_SEQUENCE) return false;
   return true;
 }
 
@@ -49,7 +50,7 @@ PolicyPlan policy_plan(int64_t T, int d, int V, int M, bool is_bwd, bool dH_dire
   c.off += align_up(is_bwd ? lm_head_bwd_workspace_bytes(p.T_pad, d, V, M, n_sm, dH_direct)
                            : lm_head_fwd_workspace_bytes(p.T_pad, d, V, n_sm), 256);
   p.loss = c.off;
-  if (!is_bwd) c.off += align_up(loss_reduce_workspace_bytes(T), 256);
+  c.off += align_up(loss_reduce_workspace_bytes(T), 256);
   p.total = c.off;
   return p;
 }
@@ -132,7 +133,7 @@ int atgrpo_clipped_loss(const float* logp, const float* old_logp, const int32_t*
       workspace_bytes < loss_reduce_workspace_bytes(T))
     return ATGRPO_ERR_WORKSPACE;
   return loss_reduce_launch(logp, old_logp, resp_of_token, adv, n_resp, nullptr, nullptr, 0, 1, T,
-                            *params, loss, coef, clip_counts, device_status, workspace,
+                            *params, nullptr, loss, coef, clip_counts, device_status, workspace,
                             static_cast<cudaStream_t>(stream));
 }
 
@@ -195,7 +196,7 @@ int atgrpo_policy_loss_fwd(const void* H, int64_t ldH, const void* const* W, int
   rc = lm_head_fwd_launch(p, lse, logp, ws + pl.gemm, st);
   if (rc != ATGRPO_OK) return rc;
   return loss_reduce_launch(logp, old_logp, resp_of_token, adv, n_resp, role_of_token, head_of_role,
-                            n_role, M, T, *params, loss, nullptr, clip_counts, device_status,
+                            n_role, M, T, *params, nullptr, loss, nullptr, clip_counts, device_status,
                             ws + pl.loss, st);
 }
 
@@ -238,8 +239,13 @@ int atgrpo_policy_loss_bwd(const void* H, int64_t ldH, const void* const* W, int
   rc = routing_launch(role_of_token, head_of_role, n_role, M, T, pl.T_pad, sched, row_of_token,
                       tok_of_row, nullptr, nullptr, device_status, ws + pl.routing, st);
   if (rc != ATGRPO_OK) return rc;
-  rc = coef_launch(logp, old_logp, resp_of_token, adv, n_resp, role_of_token, head_of_role, n_role,
-                   M, T, *params, grad_loss, sched, coef, device_status, st);
+  if (params->reduction == ATGRPO_REDUCE_SEQUENCE)
+    rc = loss_reduce_launch(logp, old_logp, resp_of_token, adv, n_resp, role_of_token, head_of_role,
+                            n_role, M, T, *params, grad_loss, nullptr, coef, nullptr, device_status,
+                            ws + pl.loss, st);
+  else
+    rc = coef_launch(logp, old_logp, resp_of_token, adv, n_resp, role_of_token, head_of_role, n_role,
+                     M, T, *params, grad_loss, sched, coef, device_status, st);
   if (rc != ATGRPO_OK) return rc;
   LmHeadProblem p;
   p.A_rows = H, p.ldA = ldH, p.rows_bound = T;

@@ -21,13 +21,15 @@ struct Schedule {                       // lives in device memory
 };
 
 // ---- loss_reduce.cu -------------------------------------------------------------------------
-// Eq. 2 reduction over tokens for up to ATGRPO_MAX_HEADS policies.
+// Eq. 2 reduction for up to ATGRPO_MAX_HEADS policies: token mean (coef only for M == 1) or,
+// with prm.reduction == ATGRPO_REDUCE_SEQUENCE, per-response ratios and the mean over responses
+// (coef for any M, scaled by grad_loss[m] / R_m; loss may be NULL).
 size_t loss_reduce_workspace_bytes(int64_t T);
 int loss_reduce_launch(const float* logp, const float* old_logp, const int32_t* resp_of_token,
                        const float* adv, int64_t n_resp, const int32_t* role_of_token,
                        const int32_t* head_of_role, int32_t n_role, int32_t M, int64_t T,
-                       const atgrpo_params& prm, float* loss, float* coef, int64_t* clip_counts,
-                       int32_t* device_status, void* workspace, cudaStream_t st);
+                       const atgrpo_params& prm, const float* grad_loss, float* loss, float* coef,
+                       int64_t* clip_counts, int32_t* device_status, void* workspace, cudaStream_t st);
 
 // coef[j] = grad_loss[m]*A*rho*[gradient passes]/T_m for every token (0 where unroutable).
 int coef_launch(const float* logp, const float* old_logp, const int32_t* resp_of_token,

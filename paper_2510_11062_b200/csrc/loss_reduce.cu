@@ -27,6 +27,9 @@ struct LossArgs {
   int64_t* part_cnt;           // [grid, M, 3] tokens, clipped-low, clipped-high
   unsigned* done;
   int vec;                     // logp, old_logp, resp (and coef) are 16-byte aligned
+  int64_t* head_cnt;           // optional [M]: items counted per head (sequence mode keeps it for backward)
+  const float* seg_term;       // sequence mode: per-response term, stored at the response's first token
+  const int32_t* seg_flags;    // sequence mode: bit 0 ratio below 1-eps_low, bit 1 above 1+eps_high
 };
 
 // Per-token term of Eq. 2.  Returns l_j; `active` tells whether the unclipped branch carries the
@@ -75,30 +78,12 @@ __device__ __forceinline__ void loss_token(const LossArgs& a, int64_t j, float l
   }
 }
 
-template <int kHeads>   // 1: single policy, no routing arrays; 0: generic (a.M heads)
-__global__ void __launch_bounds__(kThreads) k_clipped_loss(LossArgs a) {
+// Fixed-order reduction of the per-thread accumulators: shuffle tree inside each warp, one thread
+// per head across the warps, per-block partials, and the block that finishes last adds the
+// partials (fixed strided subsets, fixed tree), so the result never depends on block timing.
+template <int kHeads>
+__device__ __forceinline__ void reduce_and_finish(TokenAcc* acc, const LossArgs& a) {
   constexpr int H = kHeads == 1 ? 1 : ATGRPO_MAX_HEADS;
-  TokenAcc acc[H];
-#pragma unroll
-  for (int m = 0; m < H; ++m) acc[m].sum = 0.0, acc[m].cnt = 0, acc[m].clo = 0, acc[m].chi = 0;
-  const int64_t stride = (int64_t)gridDim.x * kThreads;
-  const int64_t tid = (int64_t)blockIdx.x * kThreads + threadIdx.x;
-  const float inv_T = a.T > 0 ? 1.f / (float)a.T : 0.f;
-  // four consecutive tokens per thread and iteration (16-byte loads) when the arrays allow it
-  const int64_t n4 = a.vec ? a.T >> 2 : 0;
-  for (int64_t q = tid; q < n4; q += stride) {
-    const float4 lp = reinterpret_cast<const float4*>(a.logp)[q];
-    const float4 lo = reinterpret_cast<const float4*>(a.old_logp)[q];
-    const int4 rs = reinterpret_cast<const int4*>(a.resp)[q];
-    loss_token<kHeads>(a, 4 * q + 0, lp.x, lo.x, rs.x, inv_T, acc);
-    loss_token<kHeads>(a, 4 * q + 1, lp.y, lo.y, rs.y, inv_T, acc);
-    loss_token<kHeads>(a, 4 * q + 2, lp.z, lo.z, rs.z, inv_T, acc);
-    loss_token<kHeads>(a, 4 * q + 3, lp.w, lo.w, rs.w, inv_T, acc);
-  }
-  for (int64_t j = 4 * n4 + tid; j < a.T; j += stride)
-    loss_token<kHeads>(a, j, a.logp[j], a.old_logp[j], a.resp[j], inv_T, acc);
-
-  // block reduction in a fixed order: shuffle tree inside each warp, then one thread per head
   __shared__ double s_sum[kThreads / 32][H];
   __shared__ int s_cnt[kThreads / 32][H][3];
   __shared__ bool s_last;
@@ -166,12 +151,141 @@ __global__ void __launch_bounds__(kThreads) k_clipped_loss(LossArgs a) {
       __syncthreads();
     }
     if (threadIdx.x == 0) {
-      a.loss[m] = r_cnt[0][0] > 0 ? (float)(r_sum[0] / (double)r_cnt[0][0]) : 0.f;
+      if (a.head_cnt) a.head_cnt[m] = r_cnt[0][0];
+      if (a.loss) a.loss[m] = r_cnt[0][0] > 0 ? (float)(r_sum[0] / (double)r_cnt[0][0]) : 0.f;
       if (a.clip_counts) a.clip_counts[2 * m] = r_cnt[0][1], a.clip_counts[2 * m + 1] = r_cnt[0][2];
     }
     __syncthreads();
   }
   if (threadIdx.x == 0) *a.done = 0;
+}
+
+template <int kHeads>   // 1: single policy, no routing arrays; 0: generic (a.M heads)
+__global__ void __launch_bounds__(kThreads) k_clipped_loss(LossArgs a) {
+  constexpr int H = kHeads == 1 ? 1 : ATGRPO_MAX_HEADS;
+  TokenAcc acc[H];
+#pragma unroll
+  for (int m = 0; m < H; ++m) acc[m].sum = 0.0, acc[m].cnt = 0, acc[m].clo = 0, acc[m].chi = 0;
+  const int64_t stride = (int64_t)gridDim.x * kThreads;
+  const int64_t tid = (int64_t)blockIdx.x * kThreads + threadIdx.x;
+  const float inv_T = a.T > 0 ? 1.f / (float)a.T : 0.f;
+  // four consecutive tokens per thread and iteration (16-byte loads) when the arrays allow it
+  const int64_t n4 = a.vec ? a.T >> 2 : 0;
+  for (int64_t q = tid; q < n4; q += stride) {
+    const float4 lp = reinterpret_cast<const float4*>(a.logp)[q];
+    const float4 lo = reinterpret_cast<const float4*>(a.old_logp)[q];
+    const int4 rs = reinterpret_cast<const int4*>(a.resp)[q];
+    loss_token<kHeads>(a, 4 * q + 0, lp.x, lo.x, rs.x, inv_T, acc);
+    loss_token<kHeads>(a, 4 * q + 1, lp.y, lo.y, rs.y, inv_T, acc);
+    loss_token<kHeads>(a, 4 * q + 2, lp.z, lo.z, rs.z, inv_T, acc);
+    loss_token<kHeads>(a, 4 * q + 3, lp.w, lo.w, rs.w, inv_T, acc);
+  }
+  for (int64_t j = 4 * n4 + tid; j < a.T; j += stride)
+    loss_token<kHeads>(a, j, a.logp[j], a.old_logp[j], a.resp[j], inv_T, acc);
+
+  reduce_and_finish<kHeads>(acc, a);
+}
+
+// ------------------------------------------------------------------ sequence-level Eq. 2
+// Eq. 2 as printed: one ratio per response, r_c = exp(sum_j logp_j - sum_j old_logp_j), and the
+// mean over the responses of the policy's batch.  Tokens are packed response by response
+// (resp_of_token non-decreasing), so a response is a segment found by binary search; one warp per
+// response sums its tokens in a fixed order.  Per-response results are parked at the response's
+// first token, which keeps the scratch proportional to T.
+__device__ __forceinline__ int64_t lower_bound_resp(const int32_t* resp, int64_t T, int c) {
+  int64_t lo = 0, hi = T;
+  while (lo < hi) {
+    const int64_t mid = (lo + hi) >> 1;
+    if (resp[mid] < c) lo = mid + 1;
+    else hi = mid;
+  }
+  return lo;
+}
+
+__global__ void __launch_bounds__(kThreads)
+k_seq_resp(const float* __restrict__ logp, const float* __restrict__ old_logp,
+           const int32_t* __restrict__ resp, const float* __restrict__ adv, int64_t n_resp, int64_t T,
+           float lo, float hi, float* __restrict__ seg_term, int32_t* __restrict__ seg_flags,
+           float* __restrict__ coef_un) {
+  const int lane = threadIdx.x & 31;
+  const int64_t warps = (int64_t)gridDim.x * (kThreads / 32);
+  for (int64_t c = (int64_t)blockIdx.x * (kThreads / 32) + (threadIdx.x >> 5); c < n_resp; c += warps) {
+    const int64_t beg = lower_bound_resp(resp, T, (int)c);
+    const int64_t end = lower_bound_resp(resp, T, (int)c + 1);
+    if (beg >= end) continue;                                  // a response without tokens
+    double part = 0.0;
+    for (int64_t j = beg + lane; j < end; j += 32) part += (double)logp[j] - (double)old_logp[j];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
+    const double A = (double)adv[c];
+    const double rho = exp(part);
+    const double rc = fmin(fmax(rho, (double)lo), (double)hi);
+    const double u = rho * A, cl = rc * A;
+    const bool active = (u <= cl) && (A != 0.0);
+    if (lane == 0) {
+      seg_term[beg] = (float)(-fmin(u, cl));
+      seg_flags[beg] = (rho < (double)lo ? 1 : 0) | (rho > (double)hi ? 2 : 0);
+    }
+    if (coef_un) {
+      const float cu = active ? (float)(A * rho) : 0.f;
+      for (int64_t j = beg + lane; j < end; j += 32) coef_un[j] = cu;
+    }
+  }
+}
+
+template <int kHeads>
+__global__ void __launch_bounds__(kThreads) k_seq_reduce(LossArgs a) {
+  constexpr int H = kHeads == 1 ? 1 : ATGRPO_MAX_HEADS;
+  TokenAcc acc[H];
+#pragma unroll
+  for (int m = 0; m < H; ++m) acc[m].sum = 0.0, acc[m].cnt = 0, acc[m].clo = 0, acc[m].chi = 0;
+  const int64_t stride = (int64_t)gridDim.x * kThreads;
+  for (int64_t j = (int64_t)blockIdx.x * kThreads + threadIdx.x; j < a.T; j += stride) {
+    const int rs = a.resp[j];
+    const int prev = j > 0 ? a.resp[j - 1] : -1;
+    if (rs < prev || (unsigned)rs >= (unsigned)a.n_resp) raise_status(a.status, ATGRPO_ERR_BAD_INDEX);
+    if (rs == prev || (unsigned)rs >= (unsigned)a.n_resp) continue;        // not the first token of a response
+    int head = 0;
+    if (kHeads != 1) {
+      const int r = a.role[j];
+      head = (unsigned)r < (unsigned)a.n_role ? a.head_of_role[r] : -1;
+      if ((unsigned)head >= (unsigned)a.M) {
+        raise_status(a.status, ATGRPO_ERR_BAD_INDEX);
+        continue;
+      }
+    }
+    const float term = a.seg_term[j];
+    const int fl = a.seg_flags[j];
+#pragma unroll
+    for (int m = 0; m < H; ++m) {
+      if (m == head) {
+        acc[m].sum += (double)term;
+        acc[m].cnt += 1;
+        acc[m].clo += fl & 1;
+        acc[m].chi += (fl >> 1) & 1;
+      }
+    }
+  }
+  reduce_and_finish<kHeads>(acc, a);
+}
+
+// coef[j] (holding A*rho*[active] of the token's response) *= grad_loss[m] / R_m.
+__global__ void __launch_bounds__(kThreads)
+k_seq_scale(float* __restrict__ coef, const int32_t* __restrict__ role,
+            const int32_t* __restrict__ head_of_role, int n_role, int M, int64_t T,
+            const float* __restrict__ grad_loss, const int64_t* __restrict__ head_cnt) {
+  const int64_t stride = (int64_t)gridDim.x * kThreads;
+  for (int64_t j = (int64_t)blockIdx.x * kThreads + threadIdx.x; j < T; j += stride) {
+    int head = 0;
+    if (M > 1) {
+      const int r = role[j];
+      head = (unsigned)r < (unsigned)n_role ? head_of_role[r] : -1;
+    }
+    float s = 0.f;
+    if ((unsigned)head < (unsigned)M && head_cnt[head] > 0)
+      s = (grad_loss ? grad_loss[head] : 1.f) / (float)head_cnt[head];
+    coef[j] *= s;
+  }
 }
 
 __global__ void __launch_bounds__(kThreads)
@@ -362,14 +476,17 @@ size_t loss_reduce_workspace_bytes(int64_t T) {
   c.take<double>((size_t)g * ATGRPO_MAX_HEADS);
   c.take<int64_t>((size_t)g * ATGRPO_MAX_HEADS * 3);
   c.take<unsigned>(1);
+  c.take<int64_t>(ATGRPO_MAX_HEADS);                 // sequence mode: responses per head
+  c.take<float>((size_t)(T < 0 ? 0 : T) + 1);        // sequence mode: per-response term
+  c.take<int32_t>((size_t)(T < 0 ? 0 : T) + 1);      // sequence mode: per-response clip flags
   return c.off;
 }
 
 int loss_reduce_launch(const float* logp, const float* old_logp, const int32_t* resp_of_token,
                        const float* adv, int64_t n_resp, const int32_t* role_of_token,
                        const int32_t* head_of_role, int32_t n_role, int32_t M, int64_t T,
-                       const atgrpo_params& prm, float* loss, float* coef, int64_t* clip_counts,
-                       int32_t* device_status, void* workspace, cudaStream_t st) {
+                       const atgrpo_params& prm, const float* grad_loss, float* loss, float* coef,
+                       int64_t* clip_counts, int32_t* device_status, void* workspace, cudaStream_t st) {
   Carver c(workspace);
   const int g = loss_grid(T);
   LossArgs a;
@@ -380,9 +497,28 @@ int loss_reduce_launch(const float* logp, const float* old_logp, const int32_t* 
   a.part_sum = c.take<double>((size_t)g * ATGRPO_MAX_HEADS);
   a.part_cnt = c.take<int64_t>((size_t)g * ATGRPO_MAX_HEADS * 3);
   a.done = c.take<unsigned>(1);
+  int64_t* head_cnt = c.take<int64_t>(ATGRPO_MAX_HEADS);
+  float* seg_term = c.take<float>((size_t)T + 1);
+  int32_t* seg_flags = c.take<int32_t>((size_t)T + 1);
+  a.head_cnt = nullptr, a.seg_term = nullptr, a.seg_flags = nullptr;
   auto al16 = [](const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; };
   a.vec = al16(logp) && al16(old_logp) && al16(resp_of_token);
   ATGRPO_CUDA_OK(cudaMemsetAsync(a.done, 0, sizeof(unsigned), st));
+  if (prm.reduction == ATGRPO_REDUCE_SEQUENCE) {
+    // per-response ratios, then the mean over responses; coef (if asked for) is scaled afterwards
+    int64_t rg = (n_resp + kThreads / 32 - 1) / (kThreads / 32);
+    if (rg > kMaxBlocks) rg = kMaxBlocks;
+    if (rg < 1) rg = 1;
+    k_seq_resp<<<(int)rg, kThreads, 0, st>>>(logp, old_logp, resp_of_token, adv, n_resp, T, a.lo, a.hi,
+                                             seg_term, seg_flags, coef);
+    a.head_cnt = head_cnt, a.seg_term = seg_term, a.seg_flags = seg_flags;
+    a.coef = nullptr;
+    if (M == 1) k_seq_reduce<1><<<g, kThreads, 0, st>>>(a);
+    else k_seq_reduce<0><<<g, kThreads, 0, st>>>(a);
+    if (coef)
+      k_seq_scale<<<g, kThreads, 0, st>>>(coef, role_of_token, head_of_role, n_role, M, T, grad_loss, head_cnt);
+    return launch_ok();
+  }
   if (M == 1) k_clipped_loss<1><<<g, kThreads, 0, st>>>(a);
   else k_clipped_loss<0><<<g, kThreads, 0, st>>>(a);
   return launch_ok();
