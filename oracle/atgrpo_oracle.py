@@ -11,6 +11,8 @@ paper (arXiv 2510.11062) in the paper's order and notation:
   group_key            Algorithm 1, "define group key g <- hash(e, i, t)"
   bucket_by_key        Algorithm 1 / Sec. 4.1 "Agent- and Turn-wise Grouping"
   group_advantages     Eq. 1 (group-relative advantage)
+  mix_rewards          Eq. 3 (agent-wise credit assignment: team + local reward)
+  group_argmax         Algorithm 1, tree-structured sampling: c* = argmax_c r^(c) inside a group
   route_tokens         Sec. 3 "Role-sharing vs. Role-specialized", B_m = U_{sigma(i)=m} D_i
   token_logprobs       pi_theta in Eq. 2: log-softmax of the LM-head logits at the sampled token
   clipped_objective    Eq. 2, per token (token-level credit, Sec. 4.1 "Reward Mask")
@@ -45,7 +47,7 @@ from __future__ import annotations
 import numpy as np
 
 __all__ = [
-    "group_key", "bucket_by_key", "group_advantages", "route_tokens",
+    "group_key", "bucket_by_key", "group_advantages", "mix_rewards", "group_argmax", "route_tokens",
     "token_logprobs", "clipped_objective", "policy_loss", "dloss_dlogp", "policy_loss_grads",
     "policy_loss_sequence", "dloss_dlogp_sequence",
     "policy_loss_grad_rows", "grad_sumsq", "clip_scale", "adamw_step",
@@ -126,6 +128,25 @@ def group_advantages(rewards, key, n_slots, std_eps=1e-6, ddof=0):
         if K > 1:
             adv[members] = (R - mu) / (sd + std_eps)
     return adv, mean, std
+
+
+def mix_rewards(r_team, r_loc, alpha=1.0):
+    """Eq. 3: r_{t,i} = alpha * r_team_t + r_loc_{t,i}, per candidate.  The mixed reward is a
+    float32 quantity (it is what Eq. 1 consumes), so the float64 sum is rounded to float32."""
+    return (alpha * _f64(r_team) + _f64(r_loc)).astype(np.float32)
+
+
+def group_argmax(rewards, key, n_slots):
+    """Greedy selection of tree-structured sampling (Algorithm 1): for every group the candidate
+    with the highest reward continues the rollout; ties go to the lowest candidate index; an empty
+    slot reports -1."""
+    r, key = _f64(rewards), _i64(key)
+    best = np.full(n_slots, -1, dtype=np.int64)
+    for c in range(r.size):                       # ascending index, strict '>' keeps the first maximum
+        s = key[c]
+        if best[s] < 0 or r[c] > r[best[s]]:
+            best[s] = c
+    return best
 
 
 # --------------------------------------------------------------------------- routing

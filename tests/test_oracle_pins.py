@@ -438,3 +438,30 @@ def test_sequence_gradients_by_finite_differences_and_autograd():
         np.testing.assert_allclose(dW[m], W[m].grad.numpy(), atol=1e-13)
     loss, _, _ = O.policy_loss_sequence(logp0.numpy(), old.numpy(), adv.numpy(), resp.numpy(), head.numpy(), M)
     assert float((torch.from_numpy(loss) * gl).sum()) == pytest.approx(float(total), rel=1e-12)
+
+
+# ----------------------------------------------------------------------------- Eq. 3 and greedy selection
+def test_reward_mix_and_group_argmax():
+    team = np.array([1.0, 0.0, 1.0, 0.25], dtype=np.float32)
+    loc = np.array([0.5, 0.75, 0.125, 0.0], dtype=np.float32)
+    np.testing.assert_array_equal(O.mix_rewards(team, loc, 1.0), [1.5, 0.75, 1.125, 0.25])
+    np.testing.assert_array_equal(O.mix_rewards(team, loc, 0.5), [1.0, 0.75, 0.625, 0.125])
+    np.testing.assert_array_equal(O.mix_rewards(team, loc, 0.0), loc)
+    assert O.mix_rewards(team, loc).dtype == np.float32
+    # argmax: brute force, ties to the lowest index, empty slot -1
+    key = np.array([2, 0, 2, 0, 2, 3, 0])
+    r = np.array([0.3, 0.9, 0.7, 0.9, 0.7, -1.0, 0.1])
+    best = O.group_argmax(r, key, 5)
+    assert best.tolist() == [1, -1, 2, 5, -1]
+    for s_ in range(5):
+        members = [c for c in range(7) if key[c] == s_]
+        if members:
+            top = max(r[c] for c in members)
+            assert best[s_] == min(c for c in members if r[c] == top)
+    # a constant team reward shared by a whole group cancels in Eq. 1
+    k = np.repeat(np.arange(3), 4)
+    loc = rng.random(12).astype(np.float32)
+    team = np.repeat(np.array([0.0, 0.5, 1.0], dtype=np.float32), 4)
+    a0, _, _ = O.group_advantages(O.mix_rewards(team, loc, 1.0), k, 3, std_eps=0.0)
+    a1, _, _ = O.group_advantages(loc, k, 3, std_eps=0.0)
+    np.testing.assert_allclose(a0, a1, atol=1e-5)
