@@ -111,6 +111,27 @@ int atgrpo_group_advantages(
     int32_t* device_status, void* workspace, size_t workspace_bytes, void* stream);
 
 /* ------------------------------------------------------------------------------------------
+ * Credit assignment, advantage and greedy selection in one call -- Eq. 3, Eq. 1 and the
+ * tree-structured sampling step of Algorithm 1 ("c* <- argmax_c r^(c)").
+ *
+ * rewards[c] = alpha*r_team[c] + r_loc[c] (Eq. 3, one fused multiply-add, fp32); advantages as in
+ * atgrpo_group_advantages over these rewards; group_best[g] = the candidate of group g with the
+ * highest reward (ties: lowest candidate index; -1 for an empty slot), i.e. the action that
+ * continues the rollout.  Optional outputs (NULL to skip): rewards_out[n_cand], group_best[G],
+ * group_of_cand, group_mean, group_std.  No bucketing outputs here (use atgrpo_group_advantages).
+ * ------------------------------------------------------------------------------------------ */
+size_t atgrpo_group_select_workspace_bytes(int64_t n_cand, int64_t n_groups);
+
+int atgrpo_group_select(
+    const float* r_team, const float* r_loc, float alpha,
+    const int32_t* env_id, const int32_t* role_id, const int32_t* turn_id,
+    int64_t n_cand, int32_t n_env, int32_t n_role, int32_t n_turn,
+    const atgrpo_params* params /* host */,
+    float* rewards_out, float* adv, int32_t* group_best,
+    int32_t* group_of_cand, float* group_mean, float* group_std,
+    int32_t* device_status, void* workspace, size_t workspace_bytes, void* stream);
+
+/* ------------------------------------------------------------------------------------------
  * Grouped advantage without a workspace.  The paper has no counterpart to this entry point; it
  * exists for callers that must not allocate device memory where the advantages are computed:
  * a process that shares the GPU with an inference engine under a fixed memory budget, a plugin

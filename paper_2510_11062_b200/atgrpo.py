@@ -25,6 +25,7 @@ EXPORTS = (
     "atgrpo_status_string",
     "atgrpo_group_advantages_workspace_bytes", "atgrpo_group_advantages",
     "atgrpo_group_advantages_noalloc",
+    "atgrpo_group_select_workspace_bytes", "atgrpo_group_select",
     "atgrpo_clipped_loss_workspace_bytes", "atgrpo_clipped_loss",
     "atgrpo_policy_loss_workspace_bytes", "atgrpo_policy_loss_launch_count",
     "atgrpo_policy_loss_fwd", "atgrpo_policy_loss_bwd",
@@ -102,6 +103,11 @@ def lib() -> ctypes.CDLL:
         L.atgrpo_group_advantages_noalloc.restype = ctypes.c_int
         L.atgrpo_group_advantages_noalloc.argtypes = [vp, vp, vp, vp, i64, i32, i32, i32, pp, vp, vp, vp, vp,
                                                       vp, vp, vp, vp]
+        L.atgrpo_group_select_workspace_bytes.restype = sz
+        L.atgrpo_group_select_workspace_bytes.argtypes = [i64, i64]
+        L.atgrpo_group_select.restype = ctypes.c_int
+        L.atgrpo_group_select.argtypes = [vp, vp, ctypes.c_float, vp, vp, vp, i64, i32, i32, i32, pp, vp, vp, vp,
+                                          vp, vp, vp, vp, vp, sz, vp]
         L.atgrpo_clipped_loss_workspace_bytes.restype = sz
         L.atgrpo_clipped_loss_workspace_bytes.argtypes = [i64]
         L.atgrpo_clipped_loss.restype = ctypes.c_int
@@ -205,6 +211,24 @@ def atgrpo_group_advantages_noalloc(rewards, env_id, role_id, turn_id, n_env, n_
     if rc != ERR_UNSUPPORTED:
         _check(rc, "atgrpo_group_advantages_noalloc")
     return rc
+
+
+def atgrpo_group_select_workspace_bytes(n_cand: int, n_groups: int) -> int:
+    return int(lib().atgrpo_group_select_workspace_bytes(n_cand, n_groups))
+
+
+def atgrpo_group_select(r_team, r_loc, alpha, env_id, role_id, turn_id, n_env, n_role, n_turn, params: Params,
+                        adv, rewards_out=None, group_best=None, group_of_cand=None, group_mean=None,
+                        group_std=None, device_status=None, workspace=None):
+    """Eq. 3 mix + Eq. 1 advantages + per-group greedy argmax in one call; see include/atgrpo.h."""
+    i32, f32 = torch.int32, torch.float32
+    rc = lib().atgrpo_group_select(
+        _ptr(r_team, f32), _ptr(r_loc, f32), float(alpha), _ptr(env_id, i32), _ptr(role_id, i32),
+        _ptr(turn_id, i32), r_team.numel(), n_env, n_role, n_turn, ctypes.byref(params.c()),
+        _ptr(rewards_out, f32), _ptr(adv, f32), _ptr(group_best, i32), _ptr(group_of_cand, i32),
+        _ptr(group_mean, f32), _ptr(group_std, f32), _ptr(device_status, i32), _ptr(workspace),
+        workspace.numel(), _stream())
+    _check(rc, "atgrpo_group_select")
 
 
 def atgrpo_clipped_loss_workspace_bytes(T: int) -> int:

@@ -120,6 +120,32 @@ int atgrpo_group_advantages(const float* rewards, const int32_t* env_id, const i
                           device_status, workspace, static_cast<cudaStream_t>(stream));
 }
 
+size_t atgrpo_group_select_workspace_bytes(int64_t n_cand, int64_t n_groups) {
+  return group_select_workspace_bytes(n_cand, n_groups);
+}
+
+int atgrpo_group_select(const float* r_team, const float* r_loc, float alpha, const int32_t* env_id,
+                        const int32_t* role_id, const int32_t* turn_id, int64_t n_cand, int32_t n_env,
+                        int32_t n_role, int32_t n_turn, const atgrpo_params* params, float* rewards_out,
+                        float* adv, int32_t* group_best, int32_t* group_of_cand, float* group_mean,
+                        float* group_std, int32_t* device_status, void* workspace, size_t workspace_bytes,
+                        void* stream) {
+  if (!params_ok(params)) return ATGRPO_ERR_INVALID_ARG;
+  if (n_cand < 0 || n_env < 1 || n_role < 1 || n_turn < 1) return ATGRPO_ERR_INVALID_ARG;
+  const int64_t G = (int64_t)n_env * n_role * n_turn;
+  if (G >= 2147483647ll || n_cand >= 2147483647ll) return ATGRPO_ERR_UNSUPPORTED;
+  if (n_cand > 0 && (r_team == nullptr || r_loc == nullptr || env_id == nullptr || role_id == nullptr ||
+                     turn_id == nullptr || adv == nullptr))
+    return ATGRPO_ERR_INVALID_ARG;
+  if (workspace == nullptr || !aligned(workspace, 256) ||
+      workspace_bytes < group_select_workspace_bytes(n_cand, G))
+    return ATGRPO_ERR_WORKSPACE;
+  GroupExtras ex{r_team, r_loc, alpha, rewards_out, group_best};
+  return group_adv_launch(nullptr, env_id, role_id, turn_id, n_cand, n_env, n_role, n_turn, *params, adv,
+                          group_of_cand, nullptr, nullptr, group_mean, group_std, device_status, workspace,
+                          static_cast<cudaStream_t>(stream), &ex);
+}
+
 size_t atgrpo_clipped_loss_workspace_bytes(int64_t T) { return loss_reduce_workspace_bytes(T); }
 
 int atgrpo_clipped_loss(const float* logp, const float* old_logp, const int32_t* resp_of_token,

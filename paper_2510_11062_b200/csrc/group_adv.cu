@@ -179,13 +179,15 @@ struct GroupTable {            // struct of arrays over the G slots; one memset 
   unsigned long long* sum;     // sum of x;        after finalize: mean as double
   unsigned long long* sqlo;    // sum of x^2 mod 2^32 parts; after finalize: 1/(std+eps) as double
   unsigned long long* sqhi;    // sum of x^2 >> 32
+  unsigned long long* best;    // optional: max of (enc(reward) << 32 | ~candidate): argmax, ties to the lowest index
 };
 
-__device__ __forceinline__ void minmax_one(int g, float r, const GroupTable& t) {
+__device__ __forceinline__ void minmax_one(int g, float r, int c, const GroupTable& t) {
   const uint32_t e = enc_ordered(r);
   atomicAdd(&t.cnt[g], 1u);
   atomicMax(&t.nmin[g], ~e);
   atomicMax(&t.emax[g], e);
+  if (t.best) atomicMax(&t.best[g], ((unsigned long long)e << 32) | (0xFFFFFFFFu - (uint32_t)c));
 }
 
 template <bool kVec>
@@ -209,10 +211,10 @@ k_hash_minmax(const int32_t* __restrict__ env, const int32_t* __restrict__ role,
       g.z = group_of(e.z, r.z, u.z, n_env, n_role, n_turn);
       g.w = group_of(e.w, r.w, u.w, n_env, n_role, n_turn);
       reinterpret_cast<int4*>(gid)[q] = g;
-      if (g.x >= 0) minmax_one(g.x, w.x, t);
-      if (g.y >= 0) minmax_one(g.y, w.y, t);
-      if (g.z >= 0) minmax_one(g.z, w.z, t);
-      if (g.w >= 0) minmax_one(g.w, w.w, t);
+      if (g.x >= 0) minmax_one(g.x, w.x, 4 * q + 0, t);
+      if (g.y >= 0) minmax_one(g.y, w.y, 4 * q + 1, t);
+      if (g.z >= 0) minmax_one(g.z, w.z, 4 * q + 2, t);
+      if (g.w >= 0) minmax_one(g.w, w.w, 4 * q + 3, t);
       if ((g.x | g.y | g.z | g.w) < 0) {
         raise_status(status, ATGRPO_ERR_BAD_INDEX);
         if (g.x < 0) adv[4 * q + 0] = 0.f;
@@ -227,7 +229,7 @@ k_hash_minmax(const int32_t* __restrict__ env, const int32_t* __restrict__ role,
     const int g = group_of(env[c], role[c], turn[c], n_env, n_role, n_turn);
     gid[c] = g;
     if (g >= 0) {
-      minmax_one(g, rewards[c], t);
+      minmax_one(g, rewards[c], c, t);
     } else {
       adv[c] = 0.f;
       raise_status(status, ATGRPO_ERR_BAD_INDEX);
@@ -272,7 +274,7 @@ k_hash_moments(const int32_t* __restrict__ gid, const float* __restrict__ reward
 
 __global__ void __launch_bounds__(kThreads)
 k_hash_finalize(GroupTable t, int G, float std_eps, int ddof, float* __restrict__ group_mean,
-                float* __restrict__ group_std) {
+                float* __restrict__ group_std, int32_t* __restrict__ group_best) {
   const int g = blockIdx.x * blockDim.x + threadIdx.x;
   if (g >= G) return;
   const unsigned K = t.cnt[g];
@@ -300,6 +302,15 @@ k_hash_finalize(GroupTable t, int G, float std_eps, int ddof, float* __restrict_
   t.sqlo[g] = (unsigned long long)__double_as_longlong(inv);
   if (group_mean) group_mean[g] = (float)mu;
   if (group_std) group_std[g] = (float)sd;
+  if (group_best) group_best[g] = K > 0 ? (int32_t)(0xFFFFFFFFu - (uint32_t)(t.best[g] & 0xFFFFFFFFull)) : -1;
+}
+
+// Eq. 3: reward = alpha * team + local, one fused multiply-add per candidate (correctly rounded).
+__global__ void __launch_bounds__(kThreads)
+k_mix_rewards(const float* __restrict__ team, const float* __restrict__ loc, float alpha, int n,
+              float* __restrict__ out) {
+  const int stride = gridDim.x * blockDim.x;
+  for (int c = blockIdx.x * blockDim.x + threadIdx.x; c < n; c += stride) out[c] = fmaf(alpha, team[c], loc[c]);
 }
 
 __device__ __forceinline__ float apply_one(int g, float r, const GroupTable& t) {
@@ -528,6 +539,14 @@ inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 
 }  // namespace
 
+size_t group_select_workspace_bytes(int64_t n_cand, int64_t n_groups) {
+  const int64_t n = n_cand < 0 ? 0 : n_cand, G = n_groups < 0 ? 0 : n_groups;
+  Carver x(nullptr);
+  x.take<float>((size_t)n + 1);
+  x.take<unsigned long long>((size_t)G + 1);
+  return make_plan(n, G).total + x.off;
+}
+
 size_t group_adv_workspace_bytes(int64_t n_cand, int64_t n_groups) {
   return make_plan(n_cand < 0 ? 0 : n_cand, n_groups < 0 ? 0 : n_groups).total;
 }
@@ -536,11 +555,31 @@ int group_adv_launch(const float* rewards, const int32_t* env_id, const int32_t*
                      const int32_t* turn_id, int64_t n_cand, int32_t n_env, int32_t n_role,
                      int32_t n_turn, const atgrpo_params& prm, float* adv, int32_t* group_of_cand,
                      int32_t* group_offsets, int32_t* group_perm, float* group_mean,
-                     float* group_std, int32_t* device_status, void* workspace, cudaStream_t st) {
+                     float* group_std, int32_t* device_status, void* workspace, cudaStream_t st,
+                     const GroupExtras* ex) {
   const int64_t G = (int64_t)n_env * n_role * n_turn;
   const int n = (int)n_cand;
   const Plan pl = make_plan(n_cand, G);
   char* ws = static_cast<char*>(workspace);
+  // Optional Eq. 3 mix and greedy argmax: their scratch follows the regular plan.
+  unsigned long long* best = nullptr;
+  int32_t* group_best = nullptr;
+  if (ex != nullptr) {
+    Carver x(ws + pl.total);
+    float* mixed = x.take<float>((size_t)n + 1);
+    best = x.take<unsigned long long>((size_t)G + 1);
+    group_best = ex->group_best;
+    if (ex->r_team != nullptr && n > 0) {
+      float* dst = ex->rewards_out ? ex->rewards_out : mixed;
+      int64_t mg = ((int64_t)n + kThreads - 1) / kThreads;
+      if (mg > 148 * 16) mg = 148 * 16;
+      k_mix_rewards<<<(int)mg, kThreads, 0, st>>>(ex->r_team, ex->r_loc, ex->alpha, n, dst);
+      rewards = dst;
+    }
+    if (group_best == nullptr) best = nullptr;
+    else if (n == 0) ATGRPO_CUDA_OK(cudaMemsetAsync(group_best, 0xFF, (size_t)G * sizeof(int32_t), st));
+    else ATGRPO_CUDA_OK(cudaMemsetAsync(best, 0, (size_t)G * sizeof(unsigned long long), st));
+  }
   int32_t* count = reinterpret_cast<int32_t*>(ws + pl.count);
   int32_t* slot = reinterpret_cast<int32_t*>(ws + pl.slot);
   int32_t* gid = group_of_cand ? group_of_cand : reinterpret_cast<int32_t*>(ws + pl.gid);
@@ -559,6 +598,7 @@ int group_adv_launch(const float* rewards, const int32_t* env_id, const int32_t*
     t.cnt = reinterpret_cast<uint32_t*>(t.sqhi + G);
     t.nmin = t.cnt + G;
     t.emax = t.nmin + G;
+    t.best = best;
     ATGRPO_CUDA_OK(cudaMemsetAsync(tb, 0, (size_t)G * 36, st));
     const bool v1 = aligned16(env_id) && aligned16(role_id) && aligned16(turn_id) &&
                     aligned16(rewards) && aligned16(hgid);
@@ -577,7 +617,7 @@ int group_adv_launch(const float* rewards, const int32_t* env_id, const int32_t*
     if (v2) k_hash_moments<true><<<grid_of(true), kThreads, 0, st>>>(hgid, rewards, n, t);
     else k_hash_moments<false><<<grid_of(false), kThreads, 0, st>>>(hgid, rewards, n, t);
     k_hash_finalize<<<(int)((G + kThreads - 1) / kThreads), kThreads, 0, st>>>(t, (int)G, prm.std_eps, prm.ddof,
-                                                                               group_mean, group_std);
+                                                                               group_mean, group_std, group_best);
     if (v3) k_hash_apply<true><<<grid_of(true), kThreads, 0, st>>>(hgid, rewards, n, t, adv);
     else k_hash_apply<false><<<grid_of(false), kThreads, 0, st>>>(hgid, rewards, n, t, adv);
     return launch_ok();

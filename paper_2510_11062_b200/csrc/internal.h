@@ -5,12 +5,24 @@
 namespace atgrpo {
 
 // ---- group_adv.cu ---------------------------------------------------------------------------
+// Optional extras of the advantage pipeline: Eq. 3 reward mix (rewards = alpha*r_team + r_loc,
+// written to rewards_out if given) and the per-group argmax candidate (group_best[G], -1 = empty).
+// Only with the sort-free pipeline (no bucketing outputs).
+struct GroupExtras {
+  const float* r_team;
+  const float* r_loc;
+  float alpha;
+  float* rewards_out;
+  int32_t* group_best;
+};
+size_t group_select_workspace_bytes(int64_t n_cand, int64_t n_groups);
 size_t group_adv_workspace_bytes(int64_t n_cand, int64_t n_groups);
 int group_adv_launch(const float* rewards, const int32_t* env_id, const int32_t* role_id,
                      const int32_t* turn_id, int64_t n_cand, int32_t n_env, int32_t n_role,
                      int32_t n_turn, const atgrpo_params& prm, float* adv, int32_t* group_of_cand,
                      int32_t* group_offsets, int32_t* group_perm, float* group_mean,
-                     float* group_std, int32_t* device_status, void* workspace, cudaStream_t st);
+                     float* group_std, int32_t* device_status, void* workspace, cudaStream_t st,
+                     const GroupExtras* extras = nullptr);
 
 // Padded 128-row tile schedule the GEMM kernels read.
 struct Schedule {                       // lives in device memory
