@@ -50,9 +50,9 @@ def _sparse_case(name, n_active_resp=6, n_sample=160):
                 logp_s=logp_s, act_pos=act_pos, old=old)
 
 
-@pytest.mark.parametrize("name", ["qwen3_1p7b", "multi3", "qwen3_8b"])
+@pytest.mark.parametrize("name", ["qwen3_1p7b", "multi3", "qwen3_8b", "long_resp"])
 def test_full_size_sparse_advantages(name):
-    c = _sparse_case(name)
+    c = _sparse_case(name, n_active_resp=2) if name == "long_resp" else _sparse_case(name)
     b, head, act, M = c["b"], c["head"], c["act"], c["b"]["spec"].n_heads
     case = U.PolicyCase(b, c["adv"], c["old"])
     out = case.fwd()
