@@ -611,6 +611,7 @@ int row_block_tiles(int64_t n_pt, int d) {
 // (few, long tiles) is what this mostly avoids.
 int bwd_chunk_width(int64_t T_pad, int d, int V, int M, int n_sm) {
   const int64_t budget = 512ll << 20;
+  if (T_pad < kPairRows) T_pad = kPairRows;            // T = 0: keep the arithmetic below defined
   const int64_t vmax = (int64_t)(V + BN - 1) / BN * BN;
   int64_t cap = budget / (T_pad * 2) / BN * BN;
   if (cap < BN) cap = BN;

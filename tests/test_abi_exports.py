@@ -48,6 +48,10 @@ def test_workspace_queries_are_monotone_and_aligned(lib):
     assert A.atgrpo_policy_loss_launch_count(16157, 2048, 151936, 1, True) > \
         A.atgrpo_policy_loss_launch_count(16157, 2048, 151936, 1, False) > 0
     assert A.atgrpo_clipped_loss_workspace_bytes(4_194_304) > 0
+    for bwd in (False, True):                          # degenerate sizes must not trip the planners
+        assert A.atgrpo_policy_loss_workspace_bytes(0, 64, 512, 1, bwd) > 0
+        assert A.atgrpo_policy_loss_workspace_bytes(1, 64, 1, 8, bwd) > 0
+    assert A.atgrpo_group_advantages_workspace_bytes(0, 1) >= 0
 
 
 def test_host_side_argument_checks_need_no_gpu(lib):
