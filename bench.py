@@ -188,7 +188,7 @@ class Runner:
         self.ws_adv = A.workspace(A.atgrpo_group_advantages_workspace_bytes(self.R, G), device)
         self.ws_fwd = A.workspace(A.atgrpo_policy_loss_workspace_bytes(T, dm, V, M, False), device)
         self.ws_bwd = A.workspace(A.atgrpo_policy_loss_workspace_bytes(T, dm, V, M, True), device)
-        self.launches = 5 + A.atgrpo_policy_loss_launch_count(T, dm, V, M, False) + \
+        self.launches = 4 + A.atgrpo_policy_loss_launch_count(T, dm, V, M, False) + \
             A.atgrpo_policy_loss_launch_count(T, dm, V, M, True)
         self.host_loss = torch.zeros(M, dtype=f32).pin_memory()
         self.h2d_bytes = sum(self.host[k].numel() * self.host[k].element_size() for k in self.host
@@ -416,7 +416,7 @@ def run_stress(args):
                 scaling="weak", vs_baseline=None, dtype="f32", data="synthetic",
                 config=dict(workload=args.workload, candidates=R, group_slots=G, tokens=T,
                             l2="flushed before every timed call"),
-                gpu_launches=5 * args.steps,
+                gpu_launches=4 * args.steps,
                 roofline=dict(bound="hbm", kernel="grouped-advantage pipeline (5 launches)", achieved=adv_gbs,
                               peak=peaks["hbm_gbs"], unit="GB/s", frac=adv_gbs / peaks["hbm_gbs"], traffic=None,
                               peak_source=peaks["source"] + " copy bandwidth"),
