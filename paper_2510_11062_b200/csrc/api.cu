@@ -43,7 +43,7 @@ PolicyPlan policy_plan(int64_t T, int d, int V, int M, bool is_bwd, bool dH_dire
   p.row_of_token = c.off; c.take<int32_t>((size_t)T + 1);
   p.routing = c.off; c.off += align_up(routing_workspace_bytes(T, M), 256);
   p.Hs = c.off;
-  if (M > 1) c.take<uint16_t>((size_t)p.T_pad * d);
+  if (M > 1 || is_bwd) c.take<uint16_t>((size_t)p.T_pad * d);   // backward always gathers the rows it keeps
   p.coef = c.off;
   if (is_bwd) c.take<float>((size_t)T + 1);
   p.gemm = c.off;
@@ -171,9 +171,11 @@ size_t atgrpo_policy_loss_workspace_bytes(int64_t T, int32_t d, int32_t V, int32
 
 int32_t atgrpo_policy_loss_launch_count(int64_t T, int32_t d, int32_t V, int32_t M, int32_t is_bwd) {
   if (T <= 0 || d < 1 || V < 1 || M < 1) return 0;
-  const int route = M == 1 ? 1 : 4;                  // single-head table, or hist + scan + scatter + gather
-  if (!is_bwd) return route + 3;                     // + GEMM sweep, logsumexp combine, Eq. 2 reduction
-  return route + 1 + 3 * lm_head_bwd_chunks(padded_rows(T, M), d, V, M, sm_count_or_default()) + 1;   // + coef, 3 GEMMs per chunk, dH cast
+  const int route = M == 1 ? 1 : 3;                  // single-head table, or histogram + scan + scatter
+  if (!is_bwd) return route + (M > 1 ? 1 : 0) + 3;   // (+ row gather) + GEMM sweep, logsumexp combine, Eq. 2 reduction
+  // routing for the counts, coef, routing of the gradient-carrying tokens, row gather,
+  // three GEMMs per vocabulary chunk, dH cast
+  return route + 1 + 3 + 1 + 3 * lm_head_bwd_chunks(padded_rows(T, M), d, V, M, sm_count_or_default()) + 1;
 }
 
 int atgrpo_policy_loss_fwd(const void* H, int64_t ldH, const void* const* W, int32_t M,
@@ -246,8 +248,7 @@ int atgrpo_policy_loss_bwd(const void* H, int64_t ldH, const void* const* W, int
   int n_sm = 0, cc = 0;
   if (device_sm_count(&n_sm, &cc) != ATGRPO_OK) return ATGRPO_ERR_CUDA;
   if (cc != 10) return ATGRPO_ERR_UNSUPPORTED;
-  const bool dH_direct = M == 1 && params->dH_dtype == ATGRPO_F32;
-  const PolicyPlan pl = policy_plan(T, d, V, M, true, dH_direct, n_sm);
+  const PolicyPlan pl = policy_plan(T, d, V, M, true, false, n_sm);
   if (workspace_bytes < pl.total) return ATGRPO_ERR_WORKSPACE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   char* ws = static_cast<char*>(workspace);
@@ -273,13 +274,16 @@ int atgrpo_policy_loss_bwd(const void* H, int64_t ldH, const void* const* W, int
     rc = coef_launch(logp, old_logp, resp_of_token, adv, n_resp, role_of_token, head_of_role, n_role,
                      M, T, *params, grad_loss, sched, coef, device_status, st);
   if (rc != ATGRPO_OK) return rc;
+  // Tokens whose coef is zero (clipped ratio, zero advantage -- e.g. every token of a group whose
+  // candidates all got the same reward) contribute exactly nothing to dH and dW: route only the
+  // others, so the three backward GEMMs run on the rows that carry a gradient.
+  rc = routing_launch(role_of_token, head_of_role, n_role, M, T, pl.T_pad, sched, row_of_token,
+                      tok_of_row, nullptr, nullptr, nullptr, ws + pl.routing, st, coef);
+  if (rc != ATGRPO_OK) return rc;
+  rc = gather_rows_launch(H, ldH, tok_of_row, pl.T_pad, d, ws + pl.Hs, st);
+  if (rc != ATGRPO_OK) return rc;
   LmHeadProblem p;
-  p.A_rows = H, p.ldA = ldH, p.rows_bound = T;
-  if (M > 1) {
-    rc = gather_rows_launch(H, ldH, tok_of_row, pl.T_pad, d, ws + pl.Hs, st);
-    if (rc != ATGRPO_OK) return rc;
-    p.A_rows = ws + pl.Hs, p.ldA = d, p.rows_bound = pl.T_pad;
-  }
+  p.A_rows = ws + pl.Hs, p.ldA = d, p.rows_bound = pl.T_pad;
   for (int m = 0; m < M; ++m) p.W[m] = W[m];
   p.M = M, p.d = d, p.V = V, p.T = T, p.T_pad = pl.T_pad;
   p.sched = sched, p.tok_of_row = tok_of_row, p.target = target, p.device_status = device_status;

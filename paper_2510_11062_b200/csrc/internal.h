@@ -53,11 +53,13 @@ int coef_launch(const float* logp, const float* old_logp, const int32_t* resp_of
 // Stable routing of tokens to heads plus the padded 128-row tile schedule the GEMM kernels read.
 size_t routing_workspace_bytes(int64_t T, int32_t M);
 // Writes sched, row_of_token[T] (padded row of each token, -1 if unroutable) and tok_of_row[T_pad]
-// (-1 for padding rows); optional role_offsets / role_perm outputs.
+// (-1 for padding rows); optional role_offsets / role_perm outputs.  With keep_if_nonzero[T] only
+// the tokens with a non-zero entry are routed (the others get row -1).
 int routing_launch(const int32_t* role_of_token, const int32_t* head_of_role, int32_t n_role,
                    int32_t M, int64_t T, int64_t T_pad, Schedule* sched, int32_t* row_of_token,
                    int32_t* tok_of_row, int32_t* role_offsets, int32_t* role_perm,
-                   int32_t* device_status, void* workspace, cudaStream_t st);
+                   int32_t* device_status, void* workspace, cudaStream_t st,
+                   const float* keep_if_nonzero = nullptr);
 // Hs[row] = H[tok_of_row[row]] (zeros for padding rows); rows of d bf16, 16-byte vectors.
 int gather_rows_launch(const void* H, int64_t ldH, const int32_t* tok_of_row, int64_t T_pad,
                        int32_t d, void* Hs, cudaStream_t st);

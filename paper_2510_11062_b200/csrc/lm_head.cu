@@ -747,7 +747,7 @@ size_t lm_head_bwd_workspace_bytes(int64_t T_pad, int32_t d, int32_t V, int32_t 
 int lm_head_bwd_launch(const LmHeadProblem& p, const float* lse, const float* coef,
                        const int32_t* row_of_token, const atgrpo_params& prm, void* dH,
                        void* const* dW, void* workspace, cudaStream_t st) {
-  const bool dH_direct = p.M == 1 && prm.dH_dtype == ATGRPO_F32;
+  const bool dH_direct = false;   // rows are compacted: dH always goes through the accumulator
   const BwdPlan pl = bwd_plan(p.T_pad, p.d, p.V, p.M, p.n_sm, dH_direct);
   char* ws = static_cast<char*>(workspace);
   __nv_bfloat16* dz = reinterpret_cast<__nv_bfloat16*>(ws + pl.dz);

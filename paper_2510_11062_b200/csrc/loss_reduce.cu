@@ -327,8 +327,13 @@ int loss_grid(int64_t T) {
 // ------------------------------------------------------------------------------- routing
 constexpr int kRouteThreads = 1024;
 
+// Head of token j, or -1 if it is routed nowhere.  `keep` (optional) drops tokens whose entry is
+// zero: the backward pass routes only the tokens that carry a gradient.
 __device__ __forceinline__ int head_of_token(const int32_t* role, const int32_t* head_of_role,
-                                             int n_role, int M, int64_t j, int32_t* status) {
+                                             int n_role, int M, int64_t j, const float* keep,
+                                             int32_t* status) {
+  if (keep != nullptr && keep[j] == 0.f) return -1;
+  if (role == nullptr) return 0;                       // single policy
   const int r = role[j];
   const int h = (unsigned)r < (unsigned)n_role ? head_of_role[r] : -1;
   if ((unsigned)h >= (unsigned)M) {
@@ -340,12 +345,12 @@ __device__ __forceinline__ int head_of_token(const int32_t* role, const int32_t*
 
 __global__ void __launch_bounds__(kRouteThreads)
 k_route_hist(const int32_t* role, const int32_t* head_of_role, int n_role, int M, int64_t T,
-             int nb, int32_t* blk_cnt, int32_t* status) {
+             int nb, const float* keep, int32_t* blk_cnt, int32_t* status) {
   __shared__ int s_cnt[ATGRPO_MAX_HEADS];
   if (threadIdx.x < ATGRPO_MAX_HEADS) s_cnt[threadIdx.x] = 0;
   __syncthreads();
   const int64_t j = (int64_t)blockIdx.x * kRouteThreads + threadIdx.x;
-  const int h = j < T ? head_of_token(role, head_of_role, n_role, M, j, status) : -1;
+  const int h = j < T ? head_of_token(role, head_of_role, n_role, M, j, keep, status) : -1;
   for (int m = 0; m < M; ++m) {
     const unsigned b = __ballot_sync(0xffffffffu, h == m);
     if ((threadIdx.x & 31) == 0 && b) atomicAdd(&s_cnt[m], __popc(b));   // integer: order-free
@@ -407,12 +412,12 @@ k_route_scan(int M, int nb, const int32_t* blk_cnt, int32_t* blk_off, Schedule* 
 
 __global__ void __launch_bounds__(kRouteThreads)
 k_route_scatter(const int32_t* role, const int32_t* head_of_role, int n_role, int M, int64_t T,
-                int nb, const int32_t* blk_off, const Schedule* sched, int32_t* row_of_token,
+                int nb, const float* keep, const int32_t* blk_off, const Schedule* sched, int32_t* row_of_token,
                 int32_t* tok_of_row, int32_t* role_perm) {
   __shared__ int s_warp[ATGRPO_MAX_HEADS][kRouteThreads / 32];
   const int64_t j = (int64_t)blockIdx.x * kRouteThreads + threadIdx.x;
   const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-  const int h = j < T ? head_of_token(role, head_of_role, n_role, M, j, nullptr) : -1;
+  const int h = j < T ? head_of_token(role, head_of_role, n_role, M, j, keep, nullptr) : -1;
   int rank_in_warp = 0;
   for (int m = 0; m < M; ++m) {
     const unsigned b = __ballot_sync(0xffffffffu, h == m);
@@ -547,8 +552,8 @@ size_t routing_workspace_bytes(int64_t T, int32_t M) {
 int routing_launch(const int32_t* role_of_token, const int32_t* head_of_role, int32_t n_role,
                    int32_t M, int64_t T, int64_t T_pad, Schedule* sched, int32_t* row_of_token,
                    int32_t* tok_of_row, int32_t* role_offsets, int32_t* role_perm,
-                   int32_t* device_status, void* workspace, cudaStream_t st) {
-  if (M == 1) {
+                   int32_t* device_status, void* workspace, cudaStream_t st, const float* keep) {
+  if (M == 1 && keep == nullptr) {
     const int grid = (int)((T_pad + 255) / 256 > 0 ? (T_pad + 255) / 256 : 1);
     k_route_single<<<grid, 256, 0, st>>>(T, T_pad, sched, tok_of_row, row_of_token, role_offsets,
                                          role_perm);
@@ -560,12 +565,12 @@ int routing_launch(const int32_t* role_of_token, const int32_t* head_of_role, in
   int32_t* blk_off = c.take<int32_t>((size_t)(nb + 1) * M);
   ATGRPO_CUDA_OK(cudaMemsetAsync(tok_of_row, 0xFF, (size_t)T_pad * sizeof(int32_t), st));
   if (nb > 0)
-    k_route_hist<<<nb, kRouteThreads, 0, st>>>(role_of_token, head_of_role, n_role, M, T, nb,
-                                               blk_cnt, device_status);
+    k_route_hist<<<nb, kRouteThreads, 0, st>>>(M == 1 ? nullptr : role_of_token, head_of_role, n_role, M, T, nb,
+                                               keep, blk_cnt, device_status);
   k_route_scan<<<1, kRouteThreads, 0, st>>>(M, nb, blk_cnt, blk_off, sched, role_offsets);
   if (nb > 0)
-    k_route_scatter<<<nb, kRouteThreads, 0, st>>>(role_of_token, head_of_role, n_role, M, T, nb,
-                                                  blk_off, sched, row_of_token, tok_of_row,
+    k_route_scatter<<<nb, kRouteThreads, 0, st>>>(M == 1 ? nullptr : role_of_token, head_of_role, n_role, M, T, nb,
+                                                  keep, blk_off, sched, row_of_token, tok_of_row,
                                                   role_perm);
   return launch_ok();
 }
