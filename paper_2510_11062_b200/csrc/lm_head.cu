@@ -578,19 +578,20 @@ bool make_map(CUtensorMap* m, const void* base, int64_t inner, int64_t outer, in
             CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// Number of vocabulary chunks of the forward sweep: enough work items to fill the SMs evenly.
-int fwd_chunks(int64_t n_mt, int n_vt, int n_sm) {
-  int best = 1;
+// Number of vocabulary chunks of the forward sweep.  Items are kept short (at most kMaxSweep
+// tiles): the pairs that share a W tile then stay within a tile or two of each other, so the tile
+// is still in L2 when the last of them reads it (with long items they drift apart and every pair
+// ends up fetching W from HBM on its own).  Among the short sweeps, the one that fills the pairs
+// most evenly wins.
+constexpr int kMaxSweep = 4;
+int fwd_chunks(int64_t n_pt, int n_vt, int n_pairs) {
+  int best = n_vt;
   double best_eff = -1.0;
-  const int cmax = n_vt < 64 ? n_vt : 64;
-  for (int c = 1; c <= cmax; ++c) {
-    const int64_t per = (n_vt + c - 1) / c;
-    const int64_t real_c = (n_vt + per - 1) / per;
-    if (real_c != c) continue;
-    const int64_t items = n_mt * c;
-    const int64_t waves = (items + n_sm - 1) / n_sm;
-    const double eff = (double)(n_mt * (int64_t)n_vt) / ((double)waves * n_sm * per);
-    if (eff > best_eff + 1e-9) best_eff = eff, best = c;
+  for (int per = 1; per <= kMaxSweep && per <= n_vt; ++per) {
+    const int c = (n_vt + per - 1) / per;
+    const int64_t waves = (n_pt * c + n_pairs - 1) / n_pairs;
+    const double eff = (double)(n_pt * (int64_t)n_vt) / ((double)waves * n_pairs * per);
+    if (eff >= best_eff - 1e-9) best_eff = eff, best = c;       // ties: the longer sweep
   }
   return best;
 }
