@@ -109,3 +109,44 @@ def test_strided_hidden_states():
     torch.cuda.synchronize()
     assert int(st.item()) == 0
     assert np.abs(lp.cpu().numpy() - logp).max() <= 1e-3
+
+
+@pytest.mark.parametrize("seed", range(8))
+def test_random_shapes(seed):
+    """Seeded random shapes: d any multiple of 8, V anywhere around the tile sizes, 1-4 heads, short and
+    long responses, both reductions -- forward, backward and routing against the oracle."""
+    g = np.random.default_rng(1000 + seed)
+    n_role = int(g.integers(1, 5))
+    heads = n_role if g.random() < 0.6 else 1
+    d = int(g.integers(8, 65)) * 8                                  # 64 .. 512
+    V = int(g.choice([int(g.integers(1, 300)), int(g.integers(300, 3000)), 256, 512, 1024 + int(g.integers(0, 3))]))
+    lo = tuple(int(x) for x in g.integers(1, 20, n_role))
+    hi = tuple(int(l + g.integers(0, 120)) for l in lo)
+    spec = WL.RolloutSpec(f"rnd{seed}", int(g.integers(1, 5)), n_role, int(g.integers(1, 4)), int(g.integers(1, 6)),
+                          lo, hi, d, V, heads, 7000 + seed, 1)
+    b = WL.make_rollout(spec)
+    _check(b, sigma=0.3)
+    if seed % 2 == 0:                                               # sequence-level reduction on half of them
+        lse, logp = U.oracle_logprobs(b)
+        adv = U.batch_advantages(b)
+        old = WL.make_old_logp(torch.from_numpy(logp), 13, 0.02)
+        head, _, _ = U.oracle_heads(b)
+        resp = b["resp_of_token"].numpy()
+        delta = logp - old.double().numpy()
+        for c in np.unique(resp):                                   # keep sequence ratios off the kinks
+            r = np.exp(delta[resp == c].sum())
+            if abs(r - 0.8) < 3e-3 or abs(r - 1.2) < 3e-3:
+                old[torch.from_numpy(resp == c)] = torch.from_numpy(logp).float()[torch.from_numpy(resp == c)]
+        prm = A.Params(reduction=A.REDUCE_SEQUENCE)
+        case = U.PolicyCase(b, adv, old, prm=prm)
+        out = case.fwd()
+        rl, _, _ = O.policy_loss_sequence(logp, old, adv, b["resp_of_token"], head, heads)
+        np.testing.assert_allclose(out["loss"].numpy(), rl, rtol=1e-3, atol=1e-7)
+        gr = case.bwd(torch.from_numpy(logp).float(), torch.from_numpy(lse).float())
+        dH, dW = O.policy_loss_grads(b["H"], b["W"], b["target"], old, adv, b["resp_of_token"], head,
+                                     reduction="sequence")
+        if np.linalg.norm(dH) > 0:
+            assert U.rel_fro(gr["dH"].numpy(), dH) <= 5e-3
+        for m in range(heads):
+            if np.linalg.norm(dW[m]) > 0:
+                assert U.rel_fro(gr["dW"][m].numpy(), dW[m]) <= 5e-3
