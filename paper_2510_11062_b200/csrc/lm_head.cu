@@ -8,12 +8,16 @@
 //   kDh  : dH_rows += dZ_chunk * W_m[chunk, :]          (A K-major, B MN-major)
 //   kDw  : dW_m[chunk, :] = dZ_chunk^T * H_rows          (A and B MN-major)
 //
-// CTA layout (320 threads): warp 0 = TMA producer, warp 1 = tcgen05.mma issuer and TMEM owner,
-// warps 2-9 = epilogue (two warps per TMEM lane quarter, each taking half of the tile's columns).  Tiles are 128 x 256 x 64 (bf16), operands
-// are staged by TMA into a 4-deep ring of 128-byte-swizzled shared-memory tiles, the fp32
-// accumulator is double buffered in the 512 TMEM columns so the epilogue of tile i overlaps the
-// MMAs of tile i+1.  Rows are addressed in the "padded row space": the tokens of policy m occupy
-// whole 128-row tiles starting at tile_begin[m], so no tile mixes two heads (grouped GEMM).
+// The kernel runs on CTA pairs (clusters of two, cta_group::2): a pair owns a 256 x 256 output
+// tile, each CTA stages its own 128 rows of A and half of B (32 KiB per k-step of 64) through TMA
+// into a 6-deep ring of 128-byte-swizzled shared-memory tiles, the pair's leader issues
+// tcgen05.mma (M = 256, N = 256, K = 16) over both CTAs' shared memory, and each CTA's 128
+// accumulator rows live in its own tensor memory, double buffered in the 512 TMEM columns so the
+// epilogue of tile i overlaps the MMAs of tile i+1.
+// CTA layout (320 threads): warp 0 = TMA producer, warp 1 = MMA issuer (leader only) and TMEM
+// owner, warps 2-9 = epilogue (two warps per TMEM lane quarter, each taking half of the columns).
+// Rows are addressed in the "padded row space": the tokens of policy m occupy whole 256-row pair
+// tiles starting at tile_begin[m], so no tile mixes two heads (grouped GEMM).
 #include <cuda_bf16.h>
 #include <cstring>
 #include "internal.h"
