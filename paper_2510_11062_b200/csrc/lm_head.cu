@@ -332,7 +332,7 @@ k_lm_head(const __grid_constant__ Maps maps, const GemmArgs g) {
         if (kMode == kDz && tok >= 0) lse2 = g.lse[tok] * kLog2e, cf = g.coef[tok];
         for (int nt = t.nt_begin; ok && nt < t.nt_end; ++nt) {
           const int n0 = t.n0 + (nt - t.nt_begin) * BN;
-          if (!(ok = mbar_wait(tfull_bar(acc), acc_phase, s_abort, g.status))) break;
+          if (!(ok = mbar_wait_backoff(tfull_bar(acc), acc_phase, s_abort, g.status))) break;
           tc_fence_after();
           for (int c = c_begin; c < c_end; ++c) {
             const int col0 = n0 + c * 32;
@@ -406,7 +406,7 @@ k_lm_head(const __grid_constant__ Maps maps, const GemmArgs g) {
         // kDh / kDw: plain accumulator write-out
         const bool has_acc = t.k_steps > 0;
         if (has_acc) {
-          if (!(ok = mbar_wait(tfull_bar(acc), acc_phase, s_abort, g.status))) break;
+          if (!(ok = mbar_wait_backoff(tfull_bar(acc), acc_phase, s_abort, g.status))) break;
           tc_fence_after();
         }
         bool valid;
