@@ -323,6 +323,9 @@ def run_ours(args):
         torch.distributed.all_reduce(tokens)
     ms_total, ms_e2e = t.tolist()
     tokens_all = tokens.item()
+    if world > 1:
+        torch.distributed.barrier()
+        torch.distributed.destroy_process_group()
     if rank != 0:
         return
     if status != 0:
