@@ -505,24 +505,46 @@ k_lm_head(const __grid_constant__ Maps maps, const GemmArgs g) {
   }
 }
 
-// Combines the per-chunk (max, sum) pairs into lse and logp, in token order.
+// Combines the per-item (max, sum) pairs into lse and logp, in token order.  Block = 32 rows x 8
+// part groups: consecutive threads read consecutive rows of one part (coalesced), each thread
+// merges every eighth part online, and thread group 0 merges the eight results in a fixed order.
 __global__ void __launch_bounds__(256)
-k_lse_combine(const Schedule* sched, int M, const int32_t* tok_of_row, int64_t T_pad, int n_chunks,
-              const float* part_m, const float* part_s, const float* zt, float* lse, float* logp) {
+k_lse_combine(const Schedule* sched, int M, const int32_t* tok_of_row, int64_t T_pad, int n_parts,
+              const float* __restrict__ part_m, const float* __restrict__ part_s,
+              const float* __restrict__ zt, float* lse, float* logp) {
+  __shared__ float s_m[8][32], s_s[8][32];
   const int64_t rows = (int64_t)sched->tile_begin[M] * BM;
-  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
-  for (int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; p < rows; p += stride) {
-    const int tok = tok_of_row[p];
-    if (tok < 0) continue;
-    float mx = -INFINITY;
-    for (int c = 0; c < 2 * n_chunks; ++c) mx = fmaxf(mx, part_m[(size_t)c * T_pad + p]);
-    float s = 0.f;                       // two column halves per vocabulary chunk
-    for (int c = 0; c < 2 * n_chunks; ++c)
-      s += part_s[(size_t)c * T_pad + p] * exp2f(part_m[(size_t)c * T_pad + p] - mx);
-    const float l = (mx + log2f(s)) * kLn2;
-    lse[tok] = l;
-    logp[tok] = zt[p] - l;
+  const int64_t p = (int64_t)blockIdx.x * 32 + threadIdx.x;
+  const int grp = threadIdx.y;
+  float mx = -INFINITY, s = 0.f;
+  if (p < rows) {
+    for (int c = grp; c < n_parts; c += 8) {
+      const float ps = part_s[(size_t)c * T_pad + p];
+      if (ps > 0.f) {                                   // a part without valid columns holds (-inf, 0)
+        const float pm = part_m[(size_t)c * T_pad + p];
+        const float nm = fmaxf(mx, pm);
+        s = s * exp2f(mx - nm) + ps * exp2f(pm - nm);
+        mx = nm;
+      }
+    }
   }
+  s_m[grp][threadIdx.x] = mx, s_s[grp][threadIdx.x] = s;
+  __syncthreads();
+  if (grp != 0 || p >= rows) return;
+  const int tok = tok_of_row[p];
+  if (tok < 0) return;
+  for (int g2 = 1; g2 < 8; ++g2) {
+    const float ps = s_s[g2][threadIdx.x];
+    if (ps > 0.f) {
+      const float pm = s_m[g2][threadIdx.x];
+      const float nm = fmaxf(mx, pm);
+      s = s * exp2f(mx - nm) + ps * exp2f(pm - nm);
+      mx = nm;
+    }
+  }
+  const float l = (mx + log2f(s)) * kLn2;
+  lse[tok] = l;
+  logp[tok] = zt[p] - l;
 }
 
 template <bool kBf16>
@@ -738,9 +760,9 @@ int lm_head_fwd_launch(const LmHeadProblem& p, float* lse, float* logp, void* wo
   g.zt = reinterpret_cast<float*>(ws + pl.zt);
   int rc = launch_gemm<kFwd>(maps, g, (p.T_pad / kPairRows) * pl.n_chunks, p.n_sm, st);
   if (rc != ATGRPO_OK) return rc;
-  const int cgrid = (int)((p.T_pad + 255) / 256 > 0 ? (p.T_pad + 255) / 256 : 1);
-  k_lse_combine<<<cgrid, 256, 0, st>>>(p.sched, p.M, p.tok_of_row, p.T_pad, pl.n_chunks, g.part_m,
-                                       g.part_s, g.zt, lse, logp);
+  const int cgrid = (int)((p.T_pad + 31) / 32 > 0 ? (p.T_pad + 31) / 32 : 1);
+  k_lse_combine<<<cgrid, dim3(32, 8), 0, st>>>(p.sched, p.M, p.tok_of_row, p.T_pad, 2 * pl.n_chunks, g.part_m,
+                                               g.part_s, g.zt, lse, logp);
   return launch_ok();
 }
 
