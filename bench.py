@@ -33,7 +33,7 @@ from paper_2510_11062_b200 import workloads as WL  # noqa: E402
 #       --launch-skip 1 --launch-count 4 python bench.py --steps 1 --warmup 3 --no-cpu-baseline
 # (profiles/k_lm_head_qwen3_1p7b_dram_traffic.txt).  Valid for the kernel as captured; set the entry
 # to None when k_lm_head<kFwd> or its tiling changes.
-FWD_SWEEP_DRAM_BYTES = {"qwen3_1p7b": 1.98e9 + 80.9e6}   # varies 1.3 - 2.0 GB between captures
+FWD_SWEEP_DRAM_BYTES = {"qwen3_1p7b": 1.98e9 + 80.9e6}   # median of three captures (1.34 / 1.98 / 2.64 GB read)
 
 METRIC = "fused AT-GRPO loss fwd+bwd tokens/sec"
 UNIT = "tokens/s"
