@@ -135,3 +135,14 @@ def test_bad_target_is_flagged_not_faulting():
     assert out["status"] == A.ERR_BAD_INDEX
     keep = np.arange(b["T"]) != 17
     assert np.abs(out["logp"].numpy()[keep] - logp[keep]).max() <= 1e-3
+
+
+def test_backward_is_bitwise_repeatable():
+    # no floating-point atomics anywhere on the path: two runs give identical bits (doubles as a race check)
+    b, lse, logp, adv, old = _case("mid_multi", 0.3)
+    case = U.PolicyCase(b, adv, old)
+    lp, ls = torch.from_numpy(logp).float(), torch.from_numpy(lse).float()
+    a, c = case.bwd(lp, ls), case.bwd(lp, ls)
+    assert torch.equal(a["dH"], c["dH"])
+    for x, y in zip(a["dW"], c["dW"]):
+        assert torch.equal(x, y)
