@@ -37,7 +37,8 @@ FWD_SWEEP_DRAM_BYTES = {"qwen3_1p7b": 1.98e9 + 80.9e6}   # median of three captu
 
 METRIC = "fused AT-GRPO loss fwd+bwd tokens/sec"
 UNIT = "tokens/s"
-CPU_SAMPLE_TOKENS = 2048
+CPU_SAMPLE_TOKENS = 2048          # cpu_baseline leg of the GPU arm: about 10 s of oracle work
+REFERENCE_SAMPLE_TOKENS = 1024    # --impl reference: each step about 5 s, so 20 + 3 steps stay near two minutes
 
 
 def measured_peaks():
@@ -91,7 +92,7 @@ def run_reference(args):
         return
     spec = WL.SPECS[args.workload]
     batch = WL.make_rollout(spec)
-    n = min(CPU_SAMPLE_TOKENS, batch["T"])
+    n = min(REFERENCE_SAMPLE_TOKENS, batch["T"])
     times = []
     for i in range(args.warmup + args.steps):
         dt = oracle_sample_seconds(batch, n)
