@@ -150,3 +150,18 @@ def test_random_shapes(seed):
         for m in range(heads):
             if np.linalg.norm(dW[m]) > 0:
                 assert U.rel_fro(gr["dW"][m].numpy(), dW[m]) <= 5e-3
+
+
+def test_all_advantages_zero_gives_zero_gradients():
+    # every group ties: no token carries a gradient, the backward GEMMs get no rows at all
+    b = WL.make_rollout(WL.SPECS["mid_multi"])
+    adv = torch.zeros(b["R"], dtype=torch.float64)
+    lse, logp = U.oracle_logprobs(b)
+    old = WL.make_old_logp(torch.from_numpy(logp), 3, 0.3)
+    case = U.PolicyCase(b, adv, old)
+    out = case.fwd()
+    assert (out["loss"] == 0).all() and out["status"] == 0
+    g = case.bwd(torch.from_numpy(logp).float(), torch.from_numpy(lse).float())
+    assert g["status"] == 0 and (g["dH"] == 0).all()
+    for w in g["dW"]:
+        assert (w == 0).all()
