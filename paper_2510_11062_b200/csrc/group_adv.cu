@@ -6,11 +6,13 @@
 //     passes over the candidates plus one over the groups.  Everything that is accumulated with
 //     atomics is an integer, so the result does not depend on the order of arrival:
 //       minmax  : g, per-group count, min and max reward (order-preserving integer encoding)
-//       moments : x = round((r - min)/(max - min) * 2^30); sum of x and of x^2 in 64-bit integers
+//       moments : x = round((r - min)/(max - min) * 2^25); sum of x and of x^2 in 64-bit integers
+//                 (2^30 and a second word for x^2 in groups of 4096 members or more)
 //       finalize: exact integer K*sum(x^2) - sum(x)^2 (128-bit) -> mean, 1/(std + eps) per group
 //       apply   : adv = (r - mean) * 1/(std + eps)
-//     Quantising to 2^-30 of the group's range moves mean and std by < 1e-9 of the range; a group
-//     with max == min gets exact zeros.  Random access touches only the per-group table.
+//     Quantising to 2^-25 of the group's range moves mean and std by < 3e-8 of the range; a group
+//     with max == min gets exact zeros.  Random access touches only the per-group table, two
+//     16-byte entries per group.
 //
 // (B) Bucketing requested (group_offsets / group_perm): counting sort + ordered statistics:
 //   key_count  : g = (e*n_role + i)*n_turn + t, per-group histogram; the atomic's return value is
@@ -161,7 +163,9 @@ k_scatter(const int32_t* __restrict__ gid, const int32_t* __restrict__ slot,
 
 
 // ------------------------------------------------------------------ (A) sort-free aggregate
-constexpr double kQuant = 1073741824.0;   // 2^30 steps across a group's reward range
+constexpr double kQuantSmall = 33554432.0;     // 2^25 steps across a group's reward range (< 4096 members)
+constexpr double kQuantBig = 1073741824.0;     // 2^30 steps for larger groups (x^2 sum split in two words)
+constexpr unsigned kBigGroup = 4096;           // 4096 * (2^25)^2 = 2^62 still fits one 64-bit sum
 
 // Order-preserving map float -> uint32 (and back), so integer atomicMax orders rewards.
 __device__ __forceinline__ uint32_t enc_ordered(float f) {
@@ -172,21 +176,32 @@ __device__ __forceinline__ float dec_ordered(uint32_t e) {
   return __uint_as_float((e & 0x80000000u) ? (e ^ 0x80000000u) : ~e);
 }
 
-struct GroupTable {            // struct of arrays over the G slots; one memset zeroes all of it
-  uint32_t* cnt;               // members
-  uint32_t* nmin;              // ~enc(min): atomicMax from 0 tracks the minimum
-  uint32_t* emax;              // enc(max)
-  unsigned long long* sum;     // sum of x;        after finalize: mean as double
-  unsigned long long* sqlo;    // sum of x^2 mod 2^32 parts; after finalize: 1/(std+eps) as double
-  unsigned long long* sqhi;    // sum of x^2 >> 32
+// Two 16-byte entries per group slot, in separate arrays: the first pass and the last touch one
+// array each, so a table larger than L2 costs them half the traffic.  One memset zeroes both.
+struct alignas(16) GroupHead {
+  uint32_t cnt;                // members
+  uint32_t nmin;               // ~enc(min): atomicMax from 0 tracks the minimum
+  uint32_t emax;               // enc(max)
+  uint32_t pad;
+};
+struct alignas(16) GroupMoments {
+  unsigned long long sum;      // sum of x;   after finalize: mean as double
+  unsigned long long sq;       // sum of x^2 (low 32-bit parts for big groups); after finalize: 1/(std+eps)
+};
+
+struct GroupTable {
+  GroupHead* h;
+  GroupMoments* m;
+  unsigned long long* sqhi;    // sum of x^2 >> 32, touched by groups of kBigGroup members or more only
   unsigned long long* best;    // optional: max of (enc(reward) << 32 | ~candidate): argmax, ties to the lowest index
 };
 
 __device__ __forceinline__ void minmax_one(int g, float r, int c, const GroupTable& t) {
   const uint32_t e = enc_ordered(r);
-  atomicAdd(&t.cnt[g], 1u);
-  atomicMax(&t.nmin[g], ~e);
-  atomicMax(&t.emax[g], e);
+  GroupHead* ge = t.h + g;
+  atomicAdd(&ge->cnt, 1u);
+  atomicMax(&ge->nmin, ~e);
+  atomicMax(&ge->emax, e);
   if (t.best) atomicMax(&t.best[g], ((unsigned long long)e << 32) | (0xFFFFFFFFu - (uint32_t)c));
 }
 
@@ -238,14 +253,22 @@ k_hash_minmax(const int32_t* __restrict__ env, const int32_t* __restrict__ role,
 }
 
 __device__ __forceinline__ void moments_one(int g, float r, const GroupTable& t) {
-  const double lo = (double)dec_ordered(~t.nmin[g]);
-  const double range = (double)dec_ordered(t.emax[g]) - lo;
+  GroupMoments* ge = t.m + g;
+  const uint4 head = *reinterpret_cast<const uint4*>(t.h + g);     // cnt, nmin, emax in one 16-byte load
+  const double lo = (double)dec_ordered(~head.y);
+  const double range = (double)dec_ordered(head.z) - lo;
   if (!(range > 0.0)) return;                       // single member or all equal: nothing to add
-  const unsigned long long x = (unsigned long long)__double2ll_rn(((double)r - lo) * (kQuant / range));
-  const unsigned long long x2 = x * x;              // < 2^60
-  atomicAdd(&t.sum[g], x);
-  atomicAdd(&t.sqlo[g], x2 & 0xFFFFFFFFull);
-  atomicAdd(&t.sqhi[g], x2 >> 32);
+  const bool big = head.x >= kBigGroup;
+  const unsigned long long x = (unsigned long long)__double2ll_rn(
+      ((double)r - lo) * ((big ? kQuantBig : kQuantSmall) / range));
+  const unsigned long long x2 = x * x;
+  atomicAdd(&ge->sum, x);
+  if (big) {
+    atomicAdd(&ge->sq, x2 & 0xFFFFFFFFull);
+    atomicAdd(&t.sqhi[g], x2 >> 32);
+  } else {
+    atomicAdd(&ge->sq, x2);
+  }
 }
 
 template <bool kVec>
@@ -277,17 +300,21 @@ k_hash_finalize(GroupTable t, int G, float std_eps, int ddof, float* __restrict_
                 float* __restrict__ group_std, int32_t* __restrict__ group_best) {
   const int g = blockIdx.x * blockDim.x + threadIdx.x;
   if (g >= G) return;
-  const unsigned K = t.cnt[g];
+  GroupMoments* ge = t.m + g;
+  const GroupHead hd = t.h[g];
+  const unsigned K = hd.cnt;
   double mu = 0.0, sd = 0.0, inv = 0.0;
   if (K > 0) {
-    const double lo = (double)dec_ordered(~t.nmin[g]);
-    const double range = (double)dec_ordered(t.emax[g]) - lo;
+    const double lo = (double)dec_ordered(~hd.nmin);
+    const double range = (double)dec_ordered(hd.emax) - lo;
     mu = lo;
     if (range > 0.0) {
-      const unsigned long long sx = t.sum[g];
-      const unsigned __int128 sxx = ((unsigned __int128)t.sqhi[g] << 32) + t.sqlo[g];
+      const bool big = K >= kBigGroup;
+      const unsigned long long sx = ge->sum;
+      const unsigned __int128 sxx =
+          big ? (((unsigned __int128)t.sqhi[g] << 32) + ge->sq) : (unsigned __int128)ge->sq;
       const unsigned __int128 num = (unsigned __int128)K * sxx - (unsigned __int128)sx * sx;   // exact, >= 0
-      const double step = range / kQuant;
+      const double step = range / (big ? kQuantBig : kQuantSmall);
       mu = lo + ((double)sx / (double)K) * step;
       const int dof = (int)K - ddof;
       if (dof > 0) {
@@ -298,8 +325,8 @@ k_hash_finalize(GroupTable t, int G, float std_eps, int ddof, float* __restrict_
     }
     if (K > 1) inv = 1.0 / (sd + (double)std_eps);
   }
-  t.sum[g] = (unsigned long long)__double_as_longlong(mu);
-  t.sqlo[g] = (unsigned long long)__double_as_longlong(inv);
+  ge->sum = (unsigned long long)__double_as_longlong(mu);
+  ge->sq = (unsigned long long)__double_as_longlong(inv);
   if (group_mean) group_mean[g] = (float)mu;
   if (group_std) group_std[g] = (float)sd;
   if (group_best) group_best[g] = K > 0 ? (int32_t)(0xFFFFFFFFu - (uint32_t)(t.best[g] & 0xFFFFFFFFull)) : -1;
@@ -314,9 +341,8 @@ k_mix_rewards(const float* __restrict__ team, const float* __restrict__ loc, flo
 }
 
 __device__ __forceinline__ float apply_one(int g, float r, const GroupTable& t) {
-  const double mu = __longlong_as_double((long long)t.sum[g]);
-  const double inv = __longlong_as_double((long long)t.sqlo[g]);
-  return (float)(((double)r - mu) * inv);
+  const double2 mi = *reinterpret_cast<const double2*>(t.m + g);      // mean, 1/(std+eps): one 16-byte load
+  return (float)(((double)r - mi.x) * mi.y);
 }
 
 template <bool kVec>
@@ -516,7 +542,7 @@ __global__ void __launch_bounds__(kThreads) k_group_stats(StatsArgs a) {
 
 struct Plan {
   size_t count, slot, gid, offsets, perm, block_sum;   // pipeline (B)
-  size_t h_gid, h_table;                               // pipeline (A): gid[n], then 36 bytes per slot
+  size_t h_gid, h_table;                               // pipeline (A): gid[n], then 40 bytes per slot
   size_t total;
 };
 Plan make_plan(int64_t n, int64_t G) {
@@ -530,7 +556,7 @@ Plan make_plan(int64_t n, int64_t G) {
   p.block_sum = c.off; c.take<int32_t>((size_t)((G + kScanBlock - 1) / kScanBlock) + 1);
   Carver h(nullptr);                                   // the two pipelines never run together:
   p.h_gid = h.off; h.take<int32_t>((size_t)n);         // they share the same bytes
-  p.h_table = h.off; h.take<unsigned long long>((size_t)G * 9 / 2 + 8);
+  p.h_table = h.off; h.take<unsigned long long>((size_t)G * 5 + 8);   // two 16-byte entries + one overflow word per slot
   p.total = c.off > h.off ? c.off : h.off;
   return p;
 }
@@ -592,14 +618,11 @@ int group_adv_launch(const float* rewards, const int32_t* env_id, const int32_t*
     int32_t* hgid = group_of_cand ? group_of_cand : reinterpret_cast<int32_t*>(ws + pl.h_gid);
     char* tb = ws + pl.h_table;
     GroupTable t;
-    t.sum = reinterpret_cast<unsigned long long*>(tb);
-    t.sqlo = t.sum + G;
-    t.sqhi = t.sqlo + G;
-    t.cnt = reinterpret_cast<uint32_t*>(t.sqhi + G);
-    t.nmin = t.cnt + G;
-    t.emax = t.nmin + G;
+    t.h = reinterpret_cast<GroupHead*>(tb);
+    t.m = reinterpret_cast<GroupMoments*>(tb + (size_t)G * 16);
+    t.sqhi = reinterpret_cast<unsigned long long*>(tb + (size_t)G * 32);
     t.best = best;
-    ATGRPO_CUDA_OK(cudaMemsetAsync(tb, 0, (size_t)G * 36, st));
+    ATGRPO_CUDA_OK(cudaMemsetAsync(tb, 0, (size_t)G * 40, st));
     const bool v1 = aligned16(env_id) && aligned16(role_id) && aligned16(turn_id) &&
                     aligned16(rewards) && aligned16(hgid);
     const bool v2 = aligned16(rewards) && aligned16(hgid);
