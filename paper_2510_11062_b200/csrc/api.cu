@@ -47,7 +47,7 @@ PolicyPlan policy_plan(int64_t T, int d, int V, int M, bool is_bwd, bool dH_dire
   p.coef = c.off;
   if (is_bwd) c.take<float>((size_t)T + 1);
   p.gemm = c.off;
-  c.off += align_up(is_bwd ? lm_head_bwd_workspace_bytes(p.T_pad, d, V, M, n_sm, dH_direct)
+  c.off += align_up(is_bwd ? lm_head_bwd_workspace_bytes(p.T_pad, d, V, dH_direct)
                            : lm_head_fwd_workspace_bytes(p.T_pad, d, V, n_sm), 256);
   p.loss = c.off;
   c.off += align_up(loss_reduce_workspace_bytes(T), 256);
@@ -174,8 +174,8 @@ int32_t atgrpo_policy_loss_launch_count(int64_t T, int32_t d, int32_t V, int32_t
   const int route = M == 1 ? 1 : 3;                  // single-head table, or histogram + scan + scatter
   if (!is_bwd) return route + (M > 1 ? 1 : 0) + 3;   // (+ row gather) + GEMM sweep, logsumexp combine, Eq. 2 reduction
   // routing for the counts, coef, routing of the gradient-carrying tokens, row gather,
-  // three GEMMs per vocabulary chunk, dH cast
-  return route + 1 + 3 + 1 + 3 * lm_head_bwd_chunks(padded_rows(T, M), d, V, M, sm_count_or_default()) + 1;
+  // one GEMM launch per vocabulary chunk plus one, dH cast
+  return route + 1 + 3 + 1 + lm_head_bwd_chunks(padded_rows(T, M), V) + 1 + 1;
 }
 
 int atgrpo_policy_loss_fwd(const void* H, int64_t ldH, const void* const* W, int32_t M,

@@ -90,13 +90,12 @@ size_t lm_head_fwd_workspace_bytes(int64_t T_pad, int32_t d, int32_t V, int32_t 
 // lse[T], logp[T] in token order.
 int lm_head_fwd_launch(const LmHeadProblem& p, float* lse, float* logp, void* workspace,
                        cudaStream_t st);
-size_t lm_head_bwd_workspace_bytes(int64_t T_pad, int32_t d, int32_t V, int32_t M, int32_t n_sm,
-                                   bool dH_direct);
+size_t lm_head_bwd_workspace_bytes(int64_t T_pad, int32_t d, int32_t V, bool dH_direct);
 // coef[T] in token order (0 for tokens that pass no gradient); dH / dW as the C ABI documents.
 int lm_head_bwd_launch(const LmHeadProblem& p, const float* lse, const float* coef,
                        const int32_t* row_of_token, const atgrpo_params& prm, void* dH,
                        void* const* dW, void* workspace, cudaStream_t st);
 int device_sm_count(int* n_sm, int* cc_major);
-int lm_head_bwd_chunks(int64_t T_pad, int32_t d, int32_t V, int32_t M, int32_t n_sm);   // vocabulary chunks of one backward call
+int lm_head_bwd_chunks(int64_t T_pad, int32_t V);   // vocabulary chunks of one backward call (it makes one GEMM launch more)
 
 }  // namespace atgrpo

@@ -1,5 +1,5 @@
 // LM-head contractions of the policy loss (pi_theta of Eq. 2 and the gradient of Eq. 2) on the
-// sm_100a tensor cores.  One warp-specialised persistent kernel template serves four modes:
+// sm_100a tensor cores.  One warp-specialised persistent kernel serves four kinds of work item:
 //
 //   kFwd : z = H W_m^T tile by tile, streaming logsumexp and target-logit gather in the epilogue;
 //          the logits only ever exist in tensor memory.
@@ -7,6 +7,11 @@
 //          dZ = coef*(softmax - onehot) and writes them as bf16 into the chunk buffer.
 //   kDh  : dH_rows += dZ_chunk * W_m[chunk, :]          (A K-major, B MN-major)
 //   kDw  : dW_m[chunk, :] = dZ_chunk^T * H_rows          (A and B MN-major)
+//
+// The forward call is one kFwd launch.  The backward call is one kBwd launch per vocabulary chunk
+// plus one: launch c holds the long dH and dW tiles of chunk c-1 and the short dZ tiles of chunk c
+// (two chunk buffers, used alternately), ordered long-first with the short tiles topping up the
+// pairs that got one long tile fewer, so a launch ends within about one short tile on every pair.
 //
 // The kernel runs on CTA pairs (clusters of two, cta_group::2): a pair owns a 256 x 256 output
 // tile, each CTA stages its own 128 rows of A and half of B (32 KiB per k-step of 64) through TMA
@@ -41,11 +46,15 @@ constexpr int kSmemBytes = kStages * kStageBytes + 1024 /* alignment slack */ + 
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 
-enum Mode { kFwd = 0, kDz = 1, kDh = 2, kDw = 3 };
+enum Mode { kFwd = 0, kDz = 1, kDh = 2, kDw = 3, kBwd = 4 /* a launch mixing kDz, kDh and kDw items */ };
 
 struct Maps {
-  CUtensorMap a;
-  CUtensorMap b[ATGRPO_MAX_HEADS];
+  CUtensorMap a_z;                       // rows of H (or their gathered copy): K-major boxes of BK x BM
+  CUtensorMap a_h;                       // dZ chunk read by kDh: K-major boxes of BK x BM
+  CUtensorMap a_w;                       // dZ chunk read by kDw as dZ^T: 64 x 64 boxes
+  CUtensorMap b_w;                       // rows of H read by kDw: 64 x 64 boxes
+  CUtensorMap b_z[ATGRPO_MAX_HEADS];     // W_m for the logits: K-major boxes of BK x BN/2
+  CUtensorMap b_h[ATGRPO_MAX_HEADS];     // W_m read by kDh: 64 x 64 boxes
 };
 
 struct GemmArgs {
@@ -56,8 +65,9 @@ struct GemmArgs {
   int V, d, M;
   int64_t T_pad;
   // kFwd / kDz: vocabulary tiling
-  int v_begin;            // first vocabulary row of this launch (0 for kFwd)
-  int n_vtiles;           // 256-wide vocabulary tiles in this launch
+  int has_z;              // kBwd: the launch holds kDz items
+  int v_begin;            // first vocabulary row of the logits items (0 for kFwd)
+  int n_vtiles;           // 256-wide vocabulary tiles of the logits items
   int tiles_per_chunk;    // kFwd: tiles one work item sweeps (1 for kDz)
   int n_chunks;
   int m_block;            // kFwd / kDz: row tiles swept together so their rows of H stay in L2
@@ -66,9 +76,12 @@ struct GemmArgs {
   float* zt;              // kFwd out: target logit              [T_pad]
   const float* lse;       // kDz in, token order
   const float* coef;      // kDz in, token order
-  __nv_bfloat16* dz;      // kDz out / kDh, kDw in: [T_pad, vc]
+  __nv_bfloat16* dz;      // kDz out: [T_pad, vc]
   int vc;                 // chunk buffer width (multiple of 256)
-  int vc_valid;           // vocabulary rows of this chunk that exist (<= vc)
+  // kDh / kDw: the chunk whose dZ an earlier launch wrote (the maps a_h / a_w point at its buffer)
+  int has_g;              // kBwd: the launch holds kDh and kDw items
+  int g_begin;            // first vocabulary row of that chunk
+  int vc_valid;           // vocabulary rows of that chunk that exist (<= vc)
   // kDh
   float* dh_acc;          // [T_pad, d] fp32
   int first_chunk;
@@ -116,21 +129,11 @@ __device__ __forceinline__ int head_of_tile(const Schedule* s, int M, int mt) {
 }
 
 // Work items are tiles of a CTA pair: 256 rows x 256 columns.  `rank` selects this CTA's half.
-template <int kMode>
-__device__ __forceinline__ int total_items(const GemmArgs& g, const Schedule* sched) {
-  const int n_pt = sched->tile_begin[g.M] / 2;          // heads start on even 128-row tiles
-  const int n_dt = (g.d + BN - 1) / BN;
-  if (kMode == kFwd || kMode == kDz) return n_pt * g.n_chunks;
-  if (kMode == kDh) return n_pt * n_dt;
-  return g.M * ((g.vc_valid + kPairRows - 1) / kPairRows) * n_dt;
-}
-
-template <int kMode>
-__device__ __forceinline__ Tile decode_item(const GemmArgs& g, const Schedule* s, int it, int rank) {
+__device__ __forceinline__ Tile decode_item(int mode, const GemmArgs& g, const Schedule* s, int it, int rank) {
   Tile t;
   const int n_dt = (g.d + BN - 1) / BN;
   t.v0 = 0, t.chunk = 0, t.nt_begin = 0, t.nt_end = 1;
-  if (kMode == kFwd || kMode == kDz) {
+  if (mode == kFwd || mode == kDz) {
     // Row tiles come in blocks of m_block pairs; inside a block the row tile runs fastest, then
     // the vocabulary chunk: co-resident pairs share W tiles, and a block's rows of H stay in L2.
     const int n_pt = s->tile_begin[g.M] / 2;
@@ -147,7 +150,7 @@ __device__ __forceinline__ Tile decode_item(const GemmArgs& g, const Schedule* s
     t.nt_end = min(t.nt_begin + g.tiles_per_chunk, g.n_vtiles);
     t.n0 = g.v_begin + t.nt_begin * BN;
     t.k_steps = (g.d + BK - 1) / BK;
-  } else if (kMode == kDh) {
+  } else if (mode == kDh) {
     const int pt = it / n_dt, dt = it - pt * n_dt;     // d tiles fastest: they share the dZ tile
     const int mt = 2 * pt + rank;
     t.head = head_of_tile(s, g.M, 2 * pt);
@@ -169,7 +172,79 @@ __device__ __forceinline__ Tile decode_item(const GemmArgs& g, const Schedule* s
   return t;
 }
 
-template <int kMode>
+// The work items of one CTA pair, in the order the pair runs them.  A forward launch deals its
+// items round-robin.  A backward launch holds long items (dH and dW tiles of one chunk: hundreds
+// of k-steps) and short ones (dZ tiles of the next chunk: d/64 k-steps): the long items are dealt
+// round-robin first, then the pairs that got one long item fewer receive `ratio` short items each
+// (ratio = long/short k-steps), and what is left is dealt round-robin again.  Every role of both
+// CTAs of a pair walks the same sequence.
+struct ItemSeq {
+  int pair, n_pairs;
+  int n_h, n_big, n_small, small_mode;
+  int lead, n_short, pre;
+  int phase, k;
+
+  __device__ __forceinline__ void init(int kMode, const GemmArgs& g, const Schedule* s, int pair_, int n_pairs_) {
+    pair = pair_, n_pairs = n_pairs_;
+    phase = 0, k = 0;
+    const int n_pt = s->tile_begin[g.M] / 2;            // heads start on even 128-row tiles
+    const int n_dt = (g.d + BN - 1) / BN;
+    n_h = 0, n_big = 0, lead = 0, n_short = 0, pre = 0;
+    if (kMode == kFwd) {
+      small_mode = kFwd;
+      n_small = n_pt * g.n_chunks;
+      return;
+    }
+    small_mode = kDz;
+    n_small = g.has_z ? n_pt * g.n_chunks : 0;
+    if (g.has_g) {
+      const int n_vt = (g.vc_valid + kPairRows - 1) / kPairRows;
+      n_h = n_pt * n_dt;
+      n_big = n_h + g.M * n_vt * n_dt;
+      lead = n_big % n_pairs;
+      if (lead > 0 && n_small > 0) {
+        const int k_long = ((g.vc_valid + BK - 1) / BK + (2 * n_pt * (BM / BK) + g.M - 1) / g.M) / 2;
+        const int k_short = (g.d + BK - 1) / BK;
+        const int ratio = max(1, (k_long + k_short / 2) / k_short);
+        n_short = n_pairs - lead;
+        pre = min(n_small, n_short * ratio);
+      }
+    }
+  }
+
+  __device__ __forceinline__ bool next(int& mode, int& it) {
+    if (phase == 0) {
+      const int b = pair + k * n_pairs;
+      if (b < n_big) {
+        ++k;
+        mode = b < n_h ? kDh : kDw;
+        it = b < n_h ? b : b - n_h;
+        return true;
+      }
+      phase = 1, k = 0;
+    }
+    if (phase == 1) {
+      if (pre > 0 && pair >= lead) {
+        const int j = (pair - lead) + k * n_short;
+        if (j < pre) {
+          ++k;
+          mode = small_mode, it = j;
+          return true;
+        }
+      }
+      phase = 2, k = 0;
+    }
+    const int j = pre + pair + k * n_pairs;
+    if (j < n_small) {
+      ++k;
+      mode = small_mode, it = j;
+      return true;
+    }
+    return false;
+  }
+};
+
+template <int kMode>    // kFwd or kBwd
 __global__ void __launch_bounds__(kGemmThreads, 1)
 k_lm_head(const __grid_constant__ Maps maps, const GemmArgs g) {
   extern __shared__ uint8_t smem_raw[];
@@ -210,7 +285,8 @@ k_lm_head(const __grid_constant__ Maps maps, const GemmArgs g) {
     }
     *s_abort = 0;
     fence_mbar_init();
-    prefetch_tmap(&maps.a);
+    prefetch_tmap(&maps.a_z);
+    if (kMode == kBwd && g.has_g) prefetch_tmap(&maps.a_h), prefetch_tmap(&maps.a_w), prefetch_tmap(&maps.b_w);
   }
   if (warp == 1) {
     tmem_alloc_pair(smem_u32(const_cast<uint32_t*>(s_tmem)), kTmemCols);
@@ -221,7 +297,9 @@ k_lm_head(const __grid_constant__ Maps maps, const GemmArgs g) {
   cluster_sync_all();                                 // peer barriers initialised, TMEM allocated
   tc_fence_after();
   const uint32_t tmem_base = *s_tmem;
-  const int n_items = total_items<kMode>(g, sched);
+  ItemSeq seq;
+  seq.init(kMode, g, sched, pair, n_pairs);
+  int item_mode = kFwd, it = 0;
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
@@ -230,8 +308,9 @@ k_lm_head(const __grid_constant__ Maps maps, const GemmArgs g) {
       uint32_t phase = 0;
       bool ok = true;
       const uint64_t keep = l2_policy_evict_last();
-      for (int it = pair; ok && it < n_items; it += n_pairs) {
-        const Tile t = decode_item<kMode>(g, sched, it, rank);
+      while (ok && seq.next(item_mode, it)) {
+        const int mode = kMode == kFwd ? (int)kFwd : item_mode;
+        const Tile t = decode_item(mode, g, sched, it, rank);
         for (int nt = t.nt_begin; ok && nt < t.nt_end; ++nt) {
           const int n0 = t.n0 + (nt - t.nt_begin) * BN + rank * (BN / 2);   // this CTA's half of B
           for (int ks = 0; ks < t.k_steps; ++ks) {
@@ -239,21 +318,21 @@ k_lm_head(const __grid_constant__ Maps maps, const GemmArgs g) {
             const uint32_t sa = smem_base + stage * kStageBytes, sb = sa + kABytes;
             const uint32_t fb = mapa_shared(full_bar(stage), 0);             // the leader's barrier
             if (rank == 0) mbar_expect_tx(full_bar(stage), 2 * kStageBytes);
-            if (kMode == kFwd || kMode == kDz) {
-              tma_load_2d_pair_hint(sa, &maps.a, ks * BK, t.row0, fb, keep);          // rows of H: re-read per W tile
-              tma_load_2d_pair(sb, &maps.b[t.head], ks * BK, n0, fb);
-            } else if (kMode == kDh) {
-              tma_load_2d_pair(sa, &maps.a, ks * BK, t.row0, fb);                      // dZ: shared by the d tiles
+            if (mode == kFwd || mode == kDz) {
+              tma_load_2d_pair_hint(sa, &maps.a_z, ks * BK, t.row0, fb, keep);        // rows of H: re-read per W tile
+              tma_load_2d_pair(sb, &maps.b_z[t.head], ks * BK, n0, fb);
+            } else if (mode == kDh) {
+              tma_load_2d_pair(sa, &maps.a_h, ks * BK, t.row0, fb);                    // dZ: shared by the d tiles
 #pragma unroll
               for (int b = 0; b < 2; ++b)                                             // W chunk: re-read per wave
-                tma_load_2d_pair_hint(sb + b * kBoxBytes, &maps.b[t.head], n0 + 64 * b, g.v_begin + ks * BK, fb, keep);
+                tma_load_2d_pair_hint(sb + b * kBoxBytes, &maps.b_h[t.head], n0 + 64 * b, g.g_begin + ks * BK, fb, keep);
             } else {
 #pragma unroll
               for (int b = 0; b < 2; ++b)
-                tma_load_2d_pair(sa + b * kBoxBytes, &maps.a, t.v0 + 64 * b, t.row0 + ks * BK, fb);
+                tma_load_2d_pair(sa + b * kBoxBytes, &maps.a_w, t.v0 + 64 * b, t.row0 + ks * BK, fb);
 #pragma unroll
               for (int b = 0; b < 2; ++b)                                             // H: re-read per wave
-                tma_load_2d_pair_hint(sb + b * kBoxBytes, &maps.b[0], n0 + 64 * b, t.row0 + ks * BK, fb, keep);
+                tma_load_2d_pair_hint(sb + b * kBoxBytes, &maps.b_w, n0 + 64 * b, t.row0 + ks * BK, fb, keep);
             }
             if (++stage == kStages) stage = 0, phase ^= 1u;
           }
@@ -263,13 +342,21 @@ k_lm_head(const __grid_constant__ Maps maps, const GemmArgs g) {
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0 && rank == 0) {
-      constexpr bool a_mn = (kMode == kDw), b_mn = (kMode == kDh || kMode == kDw);
-      constexpr uint32_t idesc = idesc_bf16(kPairRows, BN, a_mn, b_mn);
       int stage = 0, acc = 0;
       uint32_t phase = 0, acc_phase = 0;
       bool ok = true;
-      for (int it = pair; ok && it < n_items; it += n_pairs) {
-        const Tile t = decode_item<kMode>(g, sched, it, rank);
+      while (ok && seq.next(item_mode, it)) {
+        const int mode = kMode == kFwd ? (int)kFwd : item_mode;
+        // Everything that depends on the item's kind is settled here, once per item: the single
+        // issuing thread has about 128 cycles per MMA, so the inner loop only adds offsets.
+        const bool a_mn = (mode == kDw), b_mn = (mode == kDh || mode == kDw);
+        const uint32_t idesc = mode == kDw   ? idesc_bf16(kPairRows, BN, true, true)
+                               : mode == kDh ? idesc_bf16(kPairRows, BN, false, true)
+                                             : idesc_bf16(kPairRows, BN, false, false);
+        const uint64_t a_desc0 = a_mn ? smem_desc(0, kBoxBytes, 1024) : smem_desc(0, 16, 1024);
+        const uint64_t b_desc0 = b_mn ? smem_desc(0, kBoxBytes, 1024) : smem_desc(0, 16, 1024);
+        const uint64_t a_kk = (a_mn ? 2048u : 32u) >> 4, b_kk = (b_mn ? 2048u : 32u) >> 4;   // K step of 16 elements
+        const Tile t = decode_item(mode, g, sched, it, rank);
         if (t.k_steps == 0) continue;
         for (int nt = t.nt_begin; ok && nt < t.nt_end; ++nt) {
           if (!(ok = mbar_wait(tempty_bar(acc), acc_phase ^ 1u, s_abort, g.status))) break;
@@ -278,15 +365,13 @@ k_lm_head(const __grid_constant__ Maps maps, const GemmArgs g) {
           for (int ks = 0; ks < t.k_steps; ++ks) {
             if (!(ok = mbar_wait(full_bar(stage), phase, s_abort, g.status))) break;
             tc_fence_after();
+            // the start-address field holds (address >> 4) in 14 bits: shared memory stays below
+            // 2^18 bytes, so adding the offsets never carries into the next field
             const uint32_t sa = smem_base + stage * kStageBytes, sb = sa + kABytes;
+            const uint64_t ad = a_desc0 + (sa >> 4), bd = b_desc0 + (sb >> 4);
 #pragma unroll
-            for (int kk = 0; kk < BK / 16; ++kk) {
-              const uint64_t ad = a_mn ? smem_desc(sa + kk * 2048, kBoxBytes, 1024)
-                                       : smem_desc(sa + kk * 32, 16, 1024);
-              const uint64_t bd = b_mn ? smem_desc(sb + kk * 2048, kBoxBytes, 1024)
-                                       : smem_desc(sb + kk * 32, 16, 1024);
-              umma_bf16_pair(d_tmem, ad, bd, idesc, (ks | kk) != 0 ? 1u : 0u);
-            }
+            for (int kk = 0; kk < BK / 16; ++kk)
+              umma_bf16_pair(d_tmem, ad + kk * a_kk, bd + kk * b_kk, idesc, (ks | kk) != 0 ? 1u : 0u);
             umma_commit_pair(empty_bar(stage), 3);   // frees the stage in both CTAs
             if (++stage == kStages) stage = 0, phase ^= 1u;
           }
@@ -310,11 +395,12 @@ k_lm_head(const __grid_constant__ Maps maps, const GemmArgs g) {
     uint32_t acc_phase = 0;
     bool ok = true;
     const uint32_t tempty_leader0 = mapa_shared(tempty_bar(0), 0), tempty_leader1 = mapa_shared(tempty_bar(1), 0);
-    for (int it = pair; ok && it < n_items; it += n_pairs) {
-      const Tile t = decode_item<kMode>(g, sched, it, rank);
+    while (ok && seq.next(item_mode, it)) {
+      const int mode = kMode == kFwd ? (int)kFwd : item_mode;
+      const Tile t = decode_item(mode, g, sched, it, rank);
       uint32_t r[32];
 
-      if (kMode == kFwd || kMode == kDz) {
+      if (mode == kFwd || mode == kDz) {
         const int row = t.row0 + r_in_tile;
         const bool valid = r_in_tile < t.rows_valid;
         const int tok = valid ? g.tok_of_row[row] : -1;
@@ -329,18 +415,18 @@ k_lm_head(const __grid_constant__ Maps maps, const GemmArgs g) {
         float m2 = -INFINITY, ssum = 0.f, zt = 0.f;
         bool have_zt = false;
         float lse2 = 0.f, cf = 0.f;
-        if (kMode == kDz && tok >= 0) lse2 = g.lse[tok] * kLog2e, cf = g.coef[tok];
+        if (mode == kDz && tok >= 0) lse2 = g.lse[tok] * kLog2e, cf = g.coef[tok];
         for (int nt = t.nt_begin; ok && nt < t.nt_end; ++nt) {
           const int n0 = t.n0 + (nt - t.nt_begin) * BN;
           if (!(ok = mbar_wait_backoff(tfull_bar(acc), acc_phase, s_abort, g.status))) break;
           tc_fence_after();
           for (int c = c_begin; c < c_end; ++c) {
             const int col0 = n0 + c * 32;
-            if (kMode == kFwd && col0 >= g.V) break;
+            if (mode == kFwd && col0 >= g.V) break;
             __syncwarp();
             tmem_ld32(lane_addr + acc * BN + c * 32, r);
             tmem_ld_wait();
-            if (kMode == kFwd) {
+            if (mode == kFwd) {
               if (y >= col0 && y < col0 + 32) {
 #pragma unroll
                 for (int i = 0; i < 32; ++i)
@@ -397,7 +483,7 @@ k_lm_head(const __grid_constant__ Maps maps, const GemmArgs g) {
           mbar_arrive_cluster(acc ? tempty_leader1 : tempty_leader0);
           if (++acc == 2) acc = 0, acc_phase ^= 1u;
         }
-        if (kMode == kFwd && ok && tok >= 0) {
+        if (mode == kFwd && ok && tok >= 0) {
           g.part_m[(size_t)(2 * t.chunk + half) * g.T_pad + row] = m2;
           g.part_s[(size_t)(2 * t.chunk + half) * g.T_pad + row] = ssum;
           if (have_zt) g.zt[row] = zt;
@@ -411,11 +497,11 @@ k_lm_head(const __grid_constant__ Maps maps, const GemmArgs g) {
         }
         bool valid;
         size_t out_row;
-        if (kMode == kDh) {
+        if (mode == kDh) {
           valid = r_in_tile < t.rows_valid;
           out_row = (size_t)(t.row0 + r_in_tile);
         } else {
-          const int v = g.v_begin + t.v0 + r_in_tile;
+          const int v = g.g_begin + t.v0 + r_in_tile;
           valid = (t.v0 + r_in_tile < g.vc_valid) && v < g.V;
           out_row = (size_t)v;
         }
@@ -431,10 +517,10 @@ k_lm_head(const __grid_constant__ Maps maps, const GemmArgs g) {
             for (int i = 0; i < 32; ++i) r[i] = 0u;
           }
           if (!valid) continue;
-          if (kMode == kDh || !g.dw_bf16) {
-            float* dst = (kMode == kDh ? g.dh_acc : static_cast<float*>(g.dW[t.head])) +
+          if (mode == kDh || !g.dw_bf16) {
+            float* dst = (mode == kDh ? g.dh_acc : static_cast<float*>(g.dW[t.head])) +
                          out_row * g.d + col0;
-            const bool add = kMode == kDh ? !g.first_chunk : (g.dw_accumulate != 0);
+            const bool add = mode == kDh ? !g.first_chunk : (g.dw_accumulate != 0);
             // 32 bytes per lane and instruction (d is a multiple of 8, rows are 32-byte aligned)
 #pragma unroll
             for (int q8 = 0; q8 < 4; ++q8) {
@@ -632,33 +718,20 @@ int row_block_tiles(int64_t n_pt, int d) {
   return (int)gm;
 }
 
-// Width of the dZ chunk buffer (a multiple of 256 columns, buffer <= 512 MiB): the width that
-// minimises the modelled time of the three GEMM launches per chunk, counted in k-steps of one
-// 256x256x64 pair tile per wave of CTA pairs plus a fixed cost per launch.  Wave quantisation of the dW GEMM
-// (few, long tiles) is what this mostly avoids.
-int bwd_chunk_width(int64_t T_pad, int d, int V, int M, int n_sm) {
+// Width of one dZ chunk buffer (a multiple of 256 columns, each of the two buffers <= 512 MiB).
+// A backward launch mixes the long tiles of one chunk with the short ones of the next, so wave
+// quantisation does not depend on the width; wide chunks mean fewer launches and fewer
+// read-modify-write passes over the dH accumulator.  The vocabulary is cut into equal chunks.
+int bwd_chunk_width(int64_t T_pad, int V) {
   const int64_t budget = 512ll << 20;
   if (T_pad < kPairRows) T_pad = kPairRows;            // T = 0: keep the arithmetic below defined
   const int64_t vmax = (int64_t)(V + BN - 1) / BN * BN;
   int64_t cap = budget / (T_pad * 2) / BN * BN;
   if (cap < BN) cap = BN;
   if (cap > vmax) cap = vmax;
-  const int64_t n_pt = T_pad / kPairRows, n_dt = (d + BN - 1) / BN, ksd = (d + BK - 1) / BK;
-  const int64_t n_pairs = n_sm / 2 > 0 ? n_sm / 2 : 1;
-  auto waves = [&](int64_t tiles) { return (tiles + n_pairs - 1) / n_pairs; };
-  auto chunk_cost = [&](int64_t w) {
-    const int64_t z = waves(n_pt * ((w + BN - 1) / BN)) * ksd;
-    const int64_t h = waves(n_pt * n_dt) * ((w + BK - 1) / BK);
-    const int64_t dw = waves((int64_t)M * ((w + kPairRows - 1) / kPairRows) * n_dt) * ((4 * n_pt + M - 1) / M);
-    return z + h + dw + 3 * 24;
-  };
-  int64_t best = cap, best_cost = -1;
-  for (int64_t vc = BN; vc <= cap; vc += BN) {
-    const int64_t full = V / vc, tail = V - full * vc;
-    const int64_t cost = full * chunk_cost(vc) + (tail > 0 ? chunk_cost(tail) : 0);
-    if (best_cost < 0 || cost <= best_cost) best_cost = cost, best = vc;
-  }
-  return (int)best;
+  const int64_t n_chunks = (V + cap - 1) / cap;
+  const int64_t vc = ((V + n_chunks - 1) / n_chunks + BN - 1) / BN * BN;
+  return (int)vc;
 }
 
 struct FwdPlan { size_t part_m, part_s, zt, total; int n_chunks, tiles_per_chunk, n_vt; };
@@ -676,19 +749,23 @@ FwdPlan fwd_plan(int64_t T_pad, int V, int n_sm) {
   return p;
 }
 
-struct BwdPlan { size_t dz, dh_acc, total; int vc; };
-BwdPlan bwd_plan(int64_t T_pad, int d, int V, int M, int n_sm, bool dH_direct) {
+struct BwdPlan { size_t dz[2], dh_acc, total; int vc; };
+BwdPlan bwd_plan(int64_t T_pad, int d, int V, bool dH_direct) {
   BwdPlan p;
-  p.vc = bwd_chunk_width(T_pad, d, V, M, n_sm);
+  p.vc = bwd_chunk_width(T_pad, V);
   Carver c(nullptr);
-  p.dz = c.off; c.take<__nv_bfloat16>((size_t)T_pad * p.vc);
+  for (int i = 0; i < 2; ++i) {
+    p.dz[i] = c.off;
+    if (i == 0 || V > p.vc) c.take<__nv_bfloat16>((size_t)T_pad * p.vc);   // one chunk: one buffer
+  }
   p.dh_acc = c.off;
   if (!dH_direct) c.take<float>((size_t)T_pad * d);
   p.total = c.off;
   return p;
 }
 
-// Launches `pairs` clusters of two CTAs (never more than can be resident at once).
+// Launches `pairs` clusters of two CTAs (never more than can be resident at once); `items` is an
+// upper bound of the launch's work items.
 template <int kMode>
 int launch_gemm(const Maps& maps, const GemmArgs& g, int64_t items, int n_sm, cudaStream_t st) {
   if (cudaFuncSetAttribute(k_lm_head<kMode>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -734,8 +811,8 @@ int device_sm_count(int* n_sm, int* cc_major) {
   return ATGRPO_OK;
 }
 
-int lm_head_bwd_chunks(int64_t T_pad, int32_t d, int32_t V, int32_t M, int32_t n_sm) {
-  const int vc = bwd_chunk_width(T_pad, d, V, M, n_sm);
+int lm_head_bwd_chunks(int64_t T_pad, int32_t V) {
+  const int vc = bwd_chunk_width(T_pad, V);
   return (V + vc - 1) / vc;
 }
 
@@ -749,9 +826,10 @@ int lm_head_fwd_launch(const LmHeadProblem& p, float* lse, float* logp, void* wo
   const FwdPlan pl = fwd_plan(p.T_pad, p.V, p.n_sm);
   char* ws = static_cast<char*>(workspace);
   Maps maps;
-  if (!make_map(&maps.a, p.A_rows, p.d, p.rows_bound, p.ldA, BK, BM)) return ATGRPO_ERR_CUDA;
+  memset(&maps, 0, sizeof(maps));
+  if (!make_map(&maps.a_z, p.A_rows, p.d, p.rows_bound, p.ldA, BK, BM)) return ATGRPO_ERR_CUDA;
   for (int m = 0; m < p.M; ++m)
-    if (!make_map(&maps.b[m], p.W[m], p.d, p.V, p.d, BK, BN / 2)) return ATGRPO_ERR_CUDA;
+    if (!make_map(&maps.b_z[m], p.W[m], p.d, p.V, p.d, BK, BN / 2)) return ATGRPO_ERR_CUDA;
   GemmArgs g = base_args(p);
   g.v_begin = 0, g.n_vtiles = pl.n_vt, g.tiles_per_chunk = pl.tiles_per_chunk, g.n_chunks = pl.n_chunks;
   g.m_block = row_block_tiles(p.T_pad / kPairRows, p.d);
@@ -766,50 +844,69 @@ int lm_head_fwd_launch(const LmHeadProblem& p, float* lse, float* logp, void* wo
   return launch_ok();
 }
 
-size_t lm_head_bwd_workspace_bytes(int64_t T_pad, int32_t d, int32_t V, int32_t M, int32_t n_sm,
-                                   bool dH_direct) {
-  return bwd_plan(T_pad, d, V, M, n_sm, dH_direct).total;
+size_t lm_head_bwd_workspace_bytes(int64_t T_pad, int32_t d, int32_t V, bool dH_direct) {
+  return bwd_plan(T_pad, d, V, dH_direct).total;
 }
 
 int lm_head_bwd_launch(const LmHeadProblem& p, const float* lse, const float* coef,
                        const int32_t* row_of_token, const atgrpo_params& prm, void* dH,
                        void* const* dW, void* workspace, cudaStream_t st) {
   const bool dH_direct = false;   // rows are compacted: dH always goes through the accumulator
-  const BwdPlan pl = bwd_plan(p.T_pad, p.d, p.V, p.M, p.n_sm, dH_direct);
+  const BwdPlan pl = bwd_plan(p.T_pad, p.d, p.V, dH_direct);
   char* ws = static_cast<char*>(workspace);
-  __nv_bfloat16* dz = reinterpret_cast<__nv_bfloat16*>(ws + pl.dz);
+  __nv_bfloat16* dz[2] = {reinterpret_cast<__nv_bfloat16*>(ws + pl.dz[0]),
+                          reinterpret_cast<__nv_bfloat16*>(ws + pl.dz[1])};
   float* dh_acc = dH_direct ? static_cast<float*>(dH) : reinterpret_cast<float*>(ws + pl.dh_acc);
 
-  Maps m_dz, m_dh, m_dw;
-  if (!make_map(&m_dz.a, p.A_rows, p.d, p.rows_bound, p.ldA, BK, BM)) return ATGRPO_ERR_CUDA;
-  if (!make_map(&m_dh.a, dz, pl.vc, p.T_pad, pl.vc, BK, BM)) return ATGRPO_ERR_CUDA;
-  if (!make_map(&m_dw.a, dz, pl.vc, p.T_pad, pl.vc, 64, 64)) return ATGRPO_ERR_CUDA;
-  if (!make_map(&m_dw.b[0], p.A_rows, p.d, p.rows_bound, p.ldA, 64, 64)) return ATGRPO_ERR_CUDA;
+  // Maps that do not depend on the chunk buffer, then one pair (K-major / transposed view) per buffer.
+  Maps base;
+  memset(&base, 0, sizeof(base));
+  if (!make_map(&base.a_z, p.A_rows, p.d, p.rows_bound, p.ldA, BK, BM)) return ATGRPO_ERR_CUDA;
+  if (!make_map(&base.b_w, p.A_rows, p.d, p.rows_bound, p.ldA, 64, 64)) return ATGRPO_ERR_CUDA;
   for (int m = 0; m < p.M; ++m) {
-    if (!make_map(&m_dz.b[m], p.W[m], p.d, p.V, p.d, BK, BN / 2)) return ATGRPO_ERR_CUDA;
-    if (!make_map(&m_dh.b[m], p.W[m], p.d, p.V, p.d, 64, 64)) return ATGRPO_ERR_CUDA;
+    if (!make_map(&base.b_z[m], p.W[m], p.d, p.V, p.d, BK, BN / 2)) return ATGRPO_ERR_CUDA;
+    if (!make_map(&base.b_h[m], p.W[m], p.d, p.V, p.d, 64, 64)) return ATGRPO_ERR_CUDA;
+  }
+  const int n_chunks = (p.V + pl.vc - 1) / pl.vc;
+  const int n_buf = n_chunks > 1 ? 2 : 1;
+  CUtensorMap a_h[2], a_w[2];
+  for (int i = 0; i < n_buf; ++i) {
+    if (!make_map(&a_h[i], dz[i], pl.vc, p.T_pad, pl.vc, BK, BM)) return ATGRPO_ERR_CUDA;
+    if (!make_map(&a_w[i], dz[i], pl.vc, p.T_pad, pl.vc, 64, 64)) return ATGRPO_ERR_CUDA;
   }
   const int64_t n_pt = p.T_pad / kPairRows;
   const int n_dt = (p.d + BN - 1) / BN;
-  int chunk = 0;
-  for (int v_begin = 0; v_begin < p.V; v_begin += pl.vc, ++chunk) {
+  // Launch c: dZ of chunk c (if there is one) into buffer c % 2, dH and dW of chunk c - 1.
+  for (int c = 0; c <= n_chunks; ++c) {
     GemmArgs g = base_args(p);
-    g.v_begin = v_begin;
+    Maps maps = base;
+    int64_t items = 0;
     g.vc = pl.vc;
-    g.vc_valid = p.V - v_begin < pl.vc ? p.V - v_begin : pl.vc;
-    g.n_vtiles = (g.vc_valid + BN - 1) / BN;
-    g.tiles_per_chunk = 1;
-    g.m_block = row_block_tiles(n_pt, p.d);
-    g.n_chunks = g.n_vtiles;
-    g.lse = lse, g.coef = coef, g.dz = dz;
-    g.dh_acc = dh_acc, g.first_chunk = chunk == 0;
+    g.lse = lse, g.coef = coef;
+    g.dh_acc = dh_acc;
     for (int m = 0; m < p.M; ++m) g.dW[m] = dW[m];
     g.dw_bf16 = prm.dW_dtype == ATGRPO_BF16, g.dw_accumulate = prm.accumulate_dW;
-    int rc = launch_gemm<kDz>(m_dz, g, n_pt * g.n_vtiles, p.n_sm, st);
-    if (rc != ATGRPO_OK) return rc;
-    rc = launch_gemm<kDh>(m_dh, g, n_pt * n_dt, p.n_sm, st);
-    if (rc != ATGRPO_OK) return rc;
-    rc = launch_gemm<kDw>(m_dw, g, (int64_t)p.M * ((g.vc_valid + kPairRows - 1) / kPairRows) * n_dt, p.n_sm, st);
+    if (c < n_chunks) {
+      g.has_z = 1;
+      g.v_begin = c * pl.vc;
+      const int valid = p.V - g.v_begin < pl.vc ? p.V - g.v_begin : pl.vc;
+      g.n_vtiles = (valid + BN - 1) / BN;
+      g.tiles_per_chunk = 1;
+      g.n_chunks = g.n_vtiles;
+      g.m_block = row_block_tiles(n_pt, p.d);
+      g.dz = dz[c % n_buf];
+      items += n_pt * g.n_vtiles;
+    }
+    if (c > 0) {
+      g.has_g = 1;
+      g.g_begin = (c - 1) * pl.vc;
+      g.vc_valid = p.V - g.g_begin < pl.vc ? p.V - g.g_begin : pl.vc;
+      g.first_chunk = c == 1;
+      maps.a_h = a_h[(c - 1) % n_buf];
+      maps.a_w = a_w[(c - 1) % n_buf];
+      items += n_pt * n_dt + (int64_t)p.M * ((g.vc_valid + kPairRows - 1) / kPairRows) * n_dt;
+    }
+    const int rc = launch_gemm<kBwd>(maps, g, items, p.n_sm, st);
     if (rc != ATGRPO_OK) return rc;
   }
   if (!dH_direct) {
