@@ -30,10 +30,10 @@ from paper_2510_11062_b200 import workloads as WL  # noqa: E402
 
 # DRAM bytes (read + write) of ONE forward-sweep launch, from a 1-pass ncu capture of
 #   ncu --metrics dram__bytes_read.sum,dram__bytes_write.sum --clock-control none -k regex:k_lm_head
-#       --launch-skip 1 --launch-count 4 python bench.py --steps 1 --warmup 3 --no-cpu-baseline
+#       --launch-skip 1 --launch-count 12 python bench.py --steps 1 --warmup 3 --no-cpu-baseline
 # (profiles/k_lm_head_qwen3_1p7b_dram_traffic.txt).  Valid for the kernel as captured; set the entry
 # to None when k_lm_head<kFwd> or its tiling changes.
-FWD_SWEEP_DRAM_BYTES = {"qwen3_1p7b": 1.98e9 + 80.9e6}   # median of three captures (1.34 / 1.98 / 2.64 GB read)
+FWD_SWEEP_DRAM_BYTES = {"qwen3_1p7b": 2.08e9 + 79.5e6}   # capture of the current kernel (earlier builds: 1.34 - 2.64 GB read, timing dependent)
 
 METRIC = "fused AT-GRPO loss fwd+bwd tokens/sec"
 UNIT = "tokens/s"
@@ -372,13 +372,16 @@ def run_ours(args):
 def run_stress(args):
     """Memory-bound workload: grouped advantages over 262144 (env, role, turn) slots and the Eq. 2
     reduction over 4 Mi tokens (x scale).  L2 is flushed before every timed call (outside the
-    timed events), so the GB/s are HBM figures: 20 B per candidate, 12 B per token."""
+    timed events), so the GB/s are HBM figures: 20 B per candidate; 12 B per token plus 4 B per
+    response for the reduction.  The *_grouped variants keep the candidates in rollout order (the
+    members of a group adjacent) and set params.candidates_grouped."""
     from paper_2510_11062_b200 import atgrpo as A
     A.lib()
     dev = torch.device("cuda", int(os.environ.get("LOCAL_RANK", "0")))
     torch.cuda.set_device(dev)
-    scale = 16 if args.workload == "stress16" else 1
-    s = WL.make_stress(n_env=16384 * scale, n_tokens=4_194_304 * scale)
+    scale = 16 if args.workload.startswith("stress16") else 1
+    grouped = args.workload.endswith("_grouped")     # rollout order: the members of a group adjacent
+    s = WL.make_stress(n_env=16384 * scale, n_tokens=4_194_304 * scale, shuffle=not grouped)
     R, G, T = s["R"], s["G"], s["T"]
     d = {k: s[k].to(dev) for k in ("rewards", "env_id", "role_id", "turn_id", "resp_of_token", "logp", "old_logp")}
     adv = torch.empty(R, device=dev)
@@ -387,7 +390,7 @@ def run_stress(args):
     ws_a = A.workspace(A.atgrpo_group_advantages_workspace_bytes(R, G), dev)
     ws_l = A.workspace(A.atgrpo_clipped_loss_workspace_bytes(T), dev)
     flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
-    prm = A.Params()
+    prm = A.Params(candidates_grouped=1 if grouped else 0)
 
     def f_adv():
         A.atgrpo_group_advantages(d["rewards"], d["env_id"], d["role_id"], d["turn_id"], s["n_env"], s["n_role"],
@@ -416,17 +419,21 @@ def run_stress(args):
         raise SystemExit("device status %d" % int(status.item()))
     peaks = measured_peaks()
     adv_gbs = 20.0 * R / (adv_ms * 1e-3) / 1e9
-    loss_gbs = 12.0 * T / (loss_ms * 1e-3) / 1e9
+    loss_bytes = 12.0 * T + 4.0 * R                 # logp, old_logp, response index per token; each advantage once
+    loss_gbs = loss_bytes / (loss_ms * 1e-3) / 1e9
     line = dict(metric="grouped advantage HBM GB/s (20 B per candidate)", value=adv_gbs, unit="GB/s", n_gpus=1,
                 steps=args.steps, warmup=max(args.warmup, 3), ms_per_step=adv_ms, higher_is_better=True,
                 scaling="weak", vs_baseline=None, dtype="f32", data="synthetic",
                 config=dict(workload=args.workload, candidates=R, group_slots=G, tokens=T,
+                            candidate_order="rollout order (groups adjacent)" if grouped else "shuffled",
                             l2="flushed before every timed call"),
-                gpu_launches=4 * args.steps,
-                roofline=dict(bound="hbm", kernel="grouped-advantage pipeline (5 launches)", achieved=adv_gbs,
+                gpu_launches=(1 if grouped else 4) * args.steps,
+                roofline=dict(bound="hbm", kernel="k_run_advantages (one pass)" if grouped else
+                              "grouped-advantage pipeline (4 launches)", achieved=adv_gbs,
                               peak=peaks["hbm_gbs"], unit="GB/s", frac=adv_gbs / peaks["hbm_gbs"], traffic=None,
                               peak_source=peaks["source"] + " copy bandwidth"),
-                loss_reduction=dict(ms=loss_ms, gbs=loss_gbs, frac=loss_gbs / peaks["hbm_gbs"], bytes_per_token=12),
+                loss_reduction=dict(ms=loss_ms, gbs=loss_gbs, frac=loss_gbs / peaks["hbm_gbs"],
+                                    bytes="12 per token + 4 per response"),
                 best_ms=dict(advantages=adv_best, loss_reduction=loss_best), clocks=clocks)
     print(json.dumps(line), flush=True)
 
@@ -482,7 +489,7 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--workload", default="qwen3_1p7b", choices=sorted(WL.SPECS) + ["stress", "stress16", "adamw"])
+    ap.add_argument("--workload", default="qwen3_1p7b", choices=sorted(WL.SPECS) + ["stress", "stress16", "stress_grouped", "stress16_grouped", "adamw"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

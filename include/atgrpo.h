@@ -44,7 +44,9 @@ typedef enum atgrpo_status {
   ATGRPO_ERR_WORKSPACE = 3,   /* workspace NULL, misaligned or too small                      */
   ATGRPO_ERR_BAD_INDEX = 4,   /* device-detected: an id / token / role outside its range      */
   ATGRPO_ERR_TIMEOUT = 5,     /* device-detected: a bounded wait inside a kernel expired      */
-  ATGRPO_ERR_CUDA = 6         /* a CUDA runtime or driver call failed on the host             */
+  ATGRPO_ERR_CUDA = 6,        /* a CUDA runtime or driver call failed on the host             */
+  ATGRPO_ERR_LAYOUT = 7       /* device-detected: params->candidates_grouped was set, but the  */
+                              /* members of some group are not adjacent                       */
 } atgrpo_status;
 
 enum { ATGRPO_BF16 = 0, ATGRPO_F32 = 1 };
@@ -64,6 +66,14 @@ typedef struct atgrpo_params {
   int32_t dW_dtype;      /* ATGRPO_F32 (default) or ATGRPO_BF16: element type of every dW_m    */
   int32_t accumulate_dW; /* 0: dW_m is overwritten; 1: dW_m += gradient (gradient accumulation)*/
   int32_t reduction;     /* ATGRPO_REDUCE_TOKEN_MEAN (default) or ATGRPO_REDUCE_SEQUENCE           */
+  int32_t candidates_grouped; /* atgrpo_group_advantages only.  0 (default): candidates in any order.
+                               * 1: the caller promises that the members of every group are adjacent,
+                               * the order Algorithm 1 appends them in (the K samples of one
+                               * (environment, agent, turn) together); groups may follow one another
+                               * in any order.  The advantages are then computed in one streaming
+                               * pass.  The promise is checked on the device: a group that shows up in
+                               * two places raises ATGRPO_ERR_LAYOUT, and its members get the statistics
+                               * of their own stretch.  Ignored when bucketing outputs are requested. */
 } atgrpo_params;
 
 /* Readings of the expectation in Eq. 2.
@@ -88,8 +98,9 @@ const char* atgrpo_status_string(int status);
  * paper's hash(e,i,t); G = n_env*n_role*n_turn slots, empty slots allowed, G < 2^31.
  * For each non-empty group of K members: mu = mean, sigma = std (params->ddof), and
  *   adv[c] = (rewards[c] - mu) / (sigma + params->std_eps);   K = 1 gives adv = 0.
- * Sums run in fp64 in ascending candidate order, so the result is bit-reproducible and a group
- * of identical rewards yields exact zeros.
+ * The result is bit-reproducible and a group of identical rewards yields exact zeros (fp64 sums
+ * in ascending candidate order when bucketing outputs are requested or candidates_grouped is set;
+ * exact integer accumulation of rewards quantised to 2^-25 of the group's range otherwise).
  *
  * Outputs: adv[n_cand] (required).  Optional (NULL to skip): group_of_cand[n_cand] = g;
  * group_offsets[G+1] and group_perm[n_cand], the stable bucketing (slot s owns

@@ -16,7 +16,7 @@ import torch
 _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "libatgrpo.so")
 
-OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_BAD_INDEX, ERR_TIMEOUT, ERR_CUDA = range(7)
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_BAD_INDEX, ERR_TIMEOUT, ERR_CUDA, ERR_LAYOUT = range(8)
 BF16, F32 = 0, 1
 REDUCE_TOKEN_MEAN, REDUCE_SEQUENCE = 0, 1
 MAX_HEADS = 8
@@ -41,7 +41,8 @@ class _Params(ctypes.Structure):
     _fields_ = [("clip_eps_low", ctypes.c_float), ("clip_eps_high", ctypes.c_float),
                 ("std_eps", ctypes.c_float), ("ddof", ctypes.c_int32),
                 ("dH_dtype", ctypes.c_int32), ("dW_dtype", ctypes.c_int32),
-                ("accumulate_dW", ctypes.c_int32), ("reduction", ctypes.c_int32)]
+                ("accumulate_dW", ctypes.c_int32), ("reduction", ctypes.c_int32),
+                ("candidates_grouped", ctypes.c_int32)]
 
 
 class _AdamWParams(ctypes.Structure):
@@ -75,10 +76,12 @@ class Params:
     dW_dtype: int = F32
     accumulate_dW: int = 0
     reduction: int = 0          # REDUCE_TOKEN_MEAN or REDUCE_SEQUENCE
+    candidates_grouped: int = 0  # 1: the members of every group are adjacent (checked on the device)
 
     def c(self) -> _Params:
         return _Params(self.clip_eps_low, self.clip_eps_high, self.std_eps, self.ddof,
-                       self.dH_dtype, self.dW_dtype, self.accumulate_dW, self.reduction)
+                       self.dH_dtype, self.dW_dtype, self.accumulate_dW, self.reduction,
+                       self.candidates_grouped)
 
 
 _lib = None

@@ -14,6 +14,7 @@ bool params_ok(const atgrpo_params* p) {
   if (p->dH_dtype != ATGRPO_BF16 && p->dH_dtype != ATGRPO_F32) return false;
   if (p->dW_dtype != ATGRPO_BF16 && p->dW_dtype != ATGRPO_F32) return false;
   if (p->reduction != ATGRPO_REDUCE_TOKEN_MEAN && p->reduction != ATGRPO_REDUCE_SEQUENCE) return false;
+  if (p->candidates_grouped != 0 && p->candidates_grouped != 1) return false;
   return true;
 }
 
@@ -91,6 +92,7 @@ const char* atgrpo_status_string(int status) {
     case ATGRPO_ERR_BAD_INDEX: return "index out of range (detected on the device)";
     case ATGRPO_ERR_TIMEOUT: return "bounded wait expired inside a kernel";
     case ATGRPO_ERR_CUDA: return "CUDA call failed";
+    case ATGRPO_ERR_LAYOUT: return "candidates_grouped was set but a group's members are not adjacent";
     default: return "unknown status";
   }
 }

@@ -21,6 +21,15 @@
 //   scatter    : unordered bucket fill, perm_u[offsets[g] + slot] = c
 //   stats      : one thread per group sorts its few members by candidate index (which makes the
 //                permutation stable and the fp64 sums order-fixed), then mean / std / advantage.
+// (C) Adjacent groups (params.candidates_grouped): the caller promises that the members of every
+//     group are adjacent, which is the order Algorithm 1 appends them in (the K samples of one
+//     (environment, agent, turn) together).  One streaming pass: a block stages a tile of
+//     candidates in shared memory, the thread that holds the first member of a run of equal keys
+//     sums the run in fp64 in ascending order and writes the advantages back into the tile, and the
+//     tile leaves with coalesced stores; a run that outgrows the staged window is reduced by the
+//     whole block.  One integer atomic per RUN checks the promise (a key that starts two runs
+//     raises ATGRPO_ERR_LAYOUT).
+//
 // Groups of the paper hold K = 4 .. 16 candidates, far fewer than a warp, so a thread per group
 // with block-cooperative coalesced staging keeps every lane busy; blocks that meet a large group
 // switch to a block-per-group path (shared-memory bitonic sort or an ordered rescan) with a
@@ -540,6 +549,301 @@ __global__ void __launch_bounds__(kThreads) k_group_stats(StatsArgs a) {
   }
 }
 
+// ------------------------------------------------------------------ (C) adjacent groups
+constexpr int kRunTile = 2048;                       // candidates a block owns per step: 8 per thread
+constexpr int kRunHalo = 256;                        // look-ahead for runs that cross the end of a tile
+constexpr int kRunWin = kRunTile + kRunHalo;
+
+struct RunArgs {
+  const float* rewards;
+  const int32_t* env;
+  const int32_t* role;
+  const int32_t* turn;
+  int n, n_env, n_role, n_turn;
+  float* adv;
+  int32_t* gid_out;        // optional
+  int32_t* seen;           // [G], zeroed: runs started per group
+  float* group_mean;       // optional, zeroed
+  float* group_std;        // optional, zeroed
+  float std_eps;
+  int ddof;
+  int32_t* status;
+};
+
+// `earlier` = runs of group g seen before this one (the value the atomic on seen[g] returned).
+__device__ __forceinline__ void run_publish(const RunArgs& a, int g, int earlier, double mu, double sd) {
+  if (earlier != 0) raise_status(a.status, ATGRPO_ERR_LAYOUT);
+  if (a.group_mean) a.group_mean[g] = (float)mu;
+  if (a.group_std) a.group_std[g] = (float)sd;
+}
+
+constexpr int kRunWarpK = 64;                        // runs longer than this are summed by a whole warp
+constexpr int kRunPad = 4;                           // g_s[kRunPad + i] = key of staged candidate i (16-byte aligned quads)
+
+// 1/k (correctly rounded by the compiler) for the divisions by a run's size in the thread-per-run
+// path (k <= kRunWarpK = 64).
+__constant__ double c_inv_k[kRunWarpK + 1] = {
+    0.0, 1.0 / 1, 1.0 / 2, 1.0 / 3, 1.0 / 4, 1.0 / 5, 1.0 / 6, 1.0 / 7,
+    1.0 / 8, 1.0 / 9, 1.0 / 10, 1.0 / 11, 1.0 / 12, 1.0 / 13, 1.0 / 14, 1.0 / 15,
+    1.0 / 16, 1.0 / 17, 1.0 / 18, 1.0 / 19, 1.0 / 20, 1.0 / 21, 1.0 / 22, 1.0 / 23,
+    1.0 / 24, 1.0 / 25, 1.0 / 26, 1.0 / 27, 1.0 / 28, 1.0 / 29, 1.0 / 30, 1.0 / 31,
+    1.0 / 32, 1.0 / 33, 1.0 / 34, 1.0 / 35, 1.0 / 36, 1.0 / 37, 1.0 / 38, 1.0 / 39,
+    1.0 / 40, 1.0 / 41, 1.0 / 42, 1.0 / 43, 1.0 / 44, 1.0 / 45, 1.0 / 46, 1.0 / 47,
+    1.0 / 48, 1.0 / 49, 1.0 / 50, 1.0 / 51, 1.0 / 52, 1.0 / 53, 1.0 / 54, 1.0 / 55,
+    1.0 / 56, 1.0 / 57, 1.0 / 58, 1.0 / 59, 1.0 / 60, 1.0 / 61, 1.0 / 62, 1.0 / 63,
+    1.0 / 64,
+};
+
+// Std and 1/(std + eps) of one run of K members from its sum of squared deviations.
+__device__ __forceinline__ void run_stats(double ss, int K, int ddof, float std_eps, double& sd, double& inv) {
+  const int dof = K - ddof;
+  sd = dof > 0 ? sqrt(K <= kRunWarpK ? ss * c_inv_k[dof] : ss / (double)dof) : 0.0;
+  inv = K > 1 ? 1.0 / (sd + (double)std_eps) : 0.0;
+}
+
+template <bool kVec>   // kVec: all five arrays are 16-byte aligned
+__global__ void __launch_bounds__(kThreads) k_run_advantages(RunArgs a) {
+  __shared__ __align__(16) int g_s[kRunPad + kRunWin];     // g_s[kRunPad - 1] = key of the candidate before the tile
+  __shared__ __align__(16) double d_s[kRunWin];            // rewards, widened once
+  __shared__ __align__(16) float a_s[kRunWin];             // advantages
+  __shared__ unsigned short head_s[kRunTile];              // first members of the runs that start in the tile
+  __shared__ unsigned short big_s[kRunTile / kRunWarpK + 1];   // those with more than kRunWarpK members
+  __shared__ double red[kThreads];
+  __shared__ int s_heads, s_big, s_lead, s_cross, s_long, s_end;
+
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int n_tiles = (a.n + kRunTile - 1) / kRunTile;
+  for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
+    const int t0 = tile * kRunTile;
+    const int own = min(kRunTile, a.n - t0);          // candidates whose runs this block owns
+    const int cnt = min(kRunWin, a.n - t0);           // candidates staged
+    // ---- stage keys and rewards
+    const int n_quads = kVec ? cnt >> 2 : 0;
+    if (kVec) {
+#pragma unroll
+      for (int e = 0; e < (kRunWin / 4 + kThreads - 1) / kThreads; ++e) {
+        const int q = e * kThreads + threadIdx.x;
+        if (q < n_quads) {
+          const int c4 = (t0 >> 2) + q;
+          const int4 ev = reinterpret_cast<const int4*>(a.env)[c4];
+          const int4 rv = reinterpret_cast<const int4*>(a.role)[c4];
+          const int4 tv = reinterpret_cast<const int4*>(a.turn)[c4];
+          const float4 w = reinterpret_cast<const float4*>(a.rewards)[c4];
+          int4 g;
+          g.x = group_of(ev.x, rv.x, tv.x, a.n_env, a.n_role, a.n_turn);
+          g.y = group_of(ev.y, rv.y, tv.y, a.n_env, a.n_role, a.n_turn);
+          g.z = group_of(ev.z, rv.z, tv.z, a.n_env, a.n_role, a.n_turn);
+          g.w = group_of(ev.w, rv.w, tv.w, a.n_env, a.n_role, a.n_turn);
+          *reinterpret_cast<int4*>(&g_s[kRunPad + 4 * q]) = g;
+          *reinterpret_cast<double2*>(&d_s[4 * q]) = make_double2((double)w.x, (double)w.y);
+          *reinterpret_cast<double2*>(&d_s[4 * q + 2]) = make_double2((double)w.z, (double)w.w);
+          if (a.gid_out && 4 * q < own) *reinterpret_cast<int4*>(&a.gid_out[t0 + 4 * q]) = g;   // own % 4 == 0 here or the tail below
+        }
+      }
+    }
+    for (int i = 4 * n_quads + threadIdx.x; i < cnt; i += kThreads) {
+      const int c = t0 + i;
+      const int g = group_of(a.env[c], a.role[c], a.turn[c], a.n_env, a.n_role, a.n_turn);
+      g_s[kRunPad + i] = g;
+      d_s[i] = (double)a.rewards[c];
+      if (a.gid_out && i < own) a.gid_out[c] = g;
+    }
+    if (threadIdx.x == 0) {
+      g_s[kRunPad - 1] =
+          t0 > 0 ? group_of(a.env[t0 - 1], a.role[t0 - 1], a.turn[t0 - 1], a.n_env, a.n_role, a.n_turn) : -1;
+      s_long = -1, s_heads = 0, s_big = 0;
+    }
+    __syncthreads();
+    const int* gk = g_s + kRunPad;                    // gk[i] = key of staged candidate i, gk[-1] = the one before
+
+    // Thread 0: how many leading candidates continue a run the previous tile owns, and where the
+    // run that crosses the end of this tile stops.  Everyone: list the runs that start here.
+    if (threadIdx.x == 0) {
+      int lead = 0;
+      const int gp = gk[-1];
+      if (gp >= 0)
+        while (lead < cnt && gk[lead] == gp) ++lead;
+      s_lead = lead;
+      int ce = own;
+      if (own < cnt) {
+        const int gl = gk[own - 1];                   // key of the tile's last candidate
+        if (gl >= 0)
+          while (ce < cnt && gk[ce] == gl) ++ce;
+      }
+      s_cross = ce;
+    }
+    unsigned head_bits = 0;                           // bit 4*e + j: candidate 4*(e*kThreads + threadIdx.x) + j starts a run
+#pragma unroll
+    for (int e = 0; e < kRunTile / 4 / kThreads; ++e) {
+      const int i0 = 4 * (e * kThreads + threadIdx.x);
+      if (i0 < own) {
+        const int4 g = *reinterpret_cast<const int4*>(&gk[i0]);
+        const int prev = gk[i0 - 1];
+        const int gg[5] = {prev, g.x, g.y, g.z, g.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          if (i0 + j < own) {
+            if (gg[j + 1] < 0) {
+              a_s[i0 + j] = 0.f;
+              raise_status(a.status, ATGRPO_ERR_BAD_INDEX);
+            } else if (gg[j + 1] != gg[j]) {
+              head_bits |= 1u << (4 * e + j);
+            }
+          }
+        }
+      }
+    }
+    {
+      // one shared-memory atomic per warp reserves the warp's slots in the run list
+      const int mine = __popc(head_bits);
+      int incl = mine;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int u = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += u;
+      }
+      int base = 0;
+      if (lane == 31) base = atomicAdd(&s_heads, incl);
+      base = __shfl_sync(0xffffffffu, base, 31);
+      int pos = base + incl - mine;
+      while (head_bits) {
+        const int bit = __ffs(head_bits) - 1;
+        head_bits &= head_bits - 1;
+        head_s[pos++] = (unsigned short)(4 * ((bit >> 2) * kThreads + threadIdx.x) + (bit & 3));
+      }
+    }
+    __syncthreads();
+
+    // ---- one thread per run (the list is dense, so every lane works): fp64 sums in ascending order
+    const int n_heads = s_heads;
+    for (int h = threadIdx.x; h < n_heads; h += kThreads) {
+      const int i = head_s[h];
+      const int g = gk[i];
+      const double first = d_s[i];
+      double sum = first;
+      bool all_eq = true;
+      int K = 1;
+      while (i + K < cnt && gk[i + K] == g) {         // members and their sum in one sweep
+        const double v = d_s[i + K];
+        sum += v;
+        all_eq = all_eq && (v == first);
+        ++K;
+      }
+      if (i + K == cnt && t0 + cnt < a.n) {           // may go on beyond the staged window
+        s_long = i;
+        continue;
+      }
+      if (K > kRunWarpK) {
+        big_s[atomicAdd(&s_big, 1)] = (unsigned short)i;
+        continue;
+      }
+      const int earlier = atomicAdd(&a.seen[g], 1);   // issued early: its round trip overlaps the arithmetic
+      double mu = first, sd = 0.0;
+      if (all_eq) {                                   // identical rewards: exact zeros, no rounding of the mean
+        for (int k = 0; k < K; ++k) a_s[i + k] = 0.f;
+      } else {
+        mu = sum * c_inv_k[K];
+        double ss = 0.0;
+        for (int k = 0; k < K; ++k) {
+          const double dlt = d_s[i + k] - mu;
+          ss = fma(dlt, dlt, ss);
+        }
+        double inv;
+        run_stats(ss, K, a.ddof, a.std_eps, sd, inv);
+        for (int k = 0; k < K; ++k) a_s[i + k] = (float)((d_s[i + k] - mu) * inv);
+      }
+      run_publish(a, g, earlier, mu, sd);
+    }
+    __syncthreads();
+
+    // ---- runs of more than kRunWarpK members inside the window: one warp each, lane-strided
+    // partial sums in ascending order and a fixed shuffle tree
+    const int n_big = s_big;
+    for (int b = warp; b < n_big; b += kThreads / 32) {
+      const int i = big_s[b];
+      const int g = gk[i];
+      int K = 0;                                      // lanes count their strided members
+      for (int k = lane; i + k < cnt && gk[i + k] == g; k += 32) ++K;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) K += __shfl_xor_sync(0xffffffffu, K, o);
+      double part = 0.0;
+      for (int k = lane; k < K; k += 32) part += d_s[i + k];
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
+      const double mu = part / (double)K;
+      part = 0.0;
+      for (int k = lane; k < K; k += 32) {
+        const double dlt = d_s[i + k] - mu;
+        part += dlt * dlt;
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
+      double sd, inv;
+      run_stats(part, K, a.ddof, a.std_eps, sd, inv);
+      for (int k = lane; k < K; k += 32) a_s[i + k] = (float)((d_s[i + k] - mu) * inv);
+      if (lane == 0) run_publish(a, g, atomicAdd(&a.seen[g], 1), mu, sd);
+    }
+    __syncthreads();
+
+    // ---- the tile leaves with coalesced stores
+    const int lh = s_long;
+    const int lo = s_lead, hi = lh >= 0 ? lh : s_cross;   // the long run is written by the block path below
+    if (kVec) {
+      const int q_lo = (lo + 3) >> 2, q_hi = hi >> 2;      // whole quads inside [lo, hi)
+      for (int q = q_lo + threadIdx.x; q < q_hi; q += kThreads)
+        reinterpret_cast<float4*>(a.adv + t0)[q] = *reinterpret_cast<const float4*>(&a_s[4 * q]);
+      if (q_lo < q_hi) {
+        if ((int)threadIdx.x < 4 * q_lo - lo) a.adv[t0 + lo + threadIdx.x] = a_s[lo + threadIdx.x];
+        if ((int)threadIdx.x < hi - 4 * q_hi) a.adv[t0 + 4 * q_hi + threadIdx.x] = a_s[4 * q_hi + threadIdx.x];
+      } else {
+        for (int i = lo + threadIdx.x; i < hi; i += kThreads) a.adv[t0 + i] = a_s[i];
+      }
+    } else {
+      for (int i = lo + threadIdx.x; i < hi; i += kThreads) a.adv[t0 + i] = a_s[i];
+    }
+
+    if (lh >= 0) {
+      // ---- a run that outgrew the window: the whole block reduces it from global memory
+      const int g = gk[lh];
+      const int beg = t0 + lh;
+      int end = t0 + cnt;                             // equal up to here
+      for (;;) {
+        const int c = end + threadIdx.x;
+        const bool same = c < a.n &&
+                          group_of(a.env[c], a.role[c], a.turn[c], a.n_env, a.n_role, a.n_turn) == g;
+        const int n_same = __syncthreads_count(same);
+        if (n_same == kThreads) {
+          end += kThreads;
+          continue;
+        }
+        // first mismatch inside this chunk: members are the threads before it
+        if (threadIdx.x == 0) s_end = a.n;
+        __syncthreads();
+        if (!same) atomicMin(&s_end, c);
+        __syncthreads();
+        end = min(s_end, a.n);
+        break;
+      }
+      const int K = end - beg;                        // > kRunHalo
+      double part = 0.0;
+      for (int c = beg + threadIdx.x; c < end; c += kThreads) part += (double)a.rewards[c];
+      const double mu = block_sum_fixed(part, red) / (double)K;
+      part = 0.0;
+      for (int c = beg + threadIdx.x; c < end; c += kThreads) {
+        const double dlt = (double)a.rewards[c] - mu;
+        part += dlt * dlt;
+      }
+      const double ss = block_sum_fixed(part, red);
+      double sd, inv;
+      run_stats(ss, K, a.ddof, a.std_eps, sd, inv);
+      for (int c = beg + threadIdx.x; c < end; c += kThreads)
+        a.adv[c] = (float)(((double)a.rewards[c] - mu) * inv);
+      if (threadIdx.x == 0) run_publish(a, g, atomicAdd(&a.seen[g], 1), mu, sd);
+    }
+    __syncthreads();                                  // the tile's shared memory is reused
+  }
+}
+
 struct Plan {
   size_t count, slot, gid, offsets, perm, block_sum;   // pipeline (B)
   size_t h_gid, h_table;                               // pipeline (A): gid[n], then 40 bytes per slot
@@ -613,6 +917,21 @@ int group_adv_launch(const float* rewards, const int32_t* env_id, const int32_t*
   int32_t* perm = group_perm ? group_perm : reinterpret_cast<int32_t*>(ws + pl.perm);
   int32_t* block_sum = reinterpret_cast<int32_t*>(ws + pl.block_sum);
 
+  if (n > 0 && group_offsets == nullptr && group_perm == nullptr && ex == nullptr && prm.candidates_grouped) {
+    // (C) adjacent groups: one streaming pass
+    ATGRPO_CUDA_OK(cudaMemsetAsync(count, 0, (size_t)G * sizeof(int32_t), st));
+    if (group_mean) ATGRPO_CUDA_OK(cudaMemsetAsync(group_mean, 0, (size_t)G * sizeof(float), st));
+    if (group_std) ATGRPO_CUDA_OK(cudaMemsetAsync(group_std, 0, (size_t)G * sizeof(float), st));
+    RunArgs a{rewards, env_id, role_id, turn_id, n, n_env, n_role, n_turn, adv, group_of_cand, count,
+              group_mean, group_std, prm.std_eps, prm.ddof, device_status};
+    const int n_tiles = (n + kRunTile - 1) / kRunTile;
+    const int grid = n_tiles < 148 * 8 ? n_tiles : 148 * 8;
+    const bool vec = aligned16(env_id) && aligned16(role_id) && aligned16(turn_id) && aligned16(rewards) &&
+                     aligned16(adv) && (group_of_cand == nullptr || aligned16(group_of_cand));
+    if (vec) k_run_advantages<true><<<grid, kThreads, 0, st>>>(a);
+    else k_run_advantages<false><<<grid, kThreads, 0, st>>>(a);
+    return launch_ok();
+  }
   if (n > 0 && group_offsets == nullptr && group_perm == nullptr) {
     // (A) advantages only
     int32_t* hgid = group_of_cand ? group_of_cand : reinterpret_cast<int32_t*>(ws + pl.h_gid);

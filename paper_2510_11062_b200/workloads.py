@@ -131,12 +131,13 @@ def make_old_logp(logp: torch.Tensor, seed: int, sigma: float = 0.05) -> torch.T
 
 def make_stress(n_env: int = 16384, n_role: int = 4, n_turn: int = 4, k_max: int = 16,
                 n_tokens: int = 4_194_304, seed: int = 1239, frac_const: float = 0.01,
-                exact_R: int | None = None) -> dict:
+                exact_R: int | None = None, shuffle: bool = True) -> dict:
     """Memory-bound grouping + loss-reduction stress input.
 
     G = n_env*n_role*n_turn group slots, group sizes K_g ~ U{1..k_max} (K=1 groups occur
     naturally), candidates globally shuffled, at least frac_const of the groups given
-    identical rewards.  With exact_R the groups are filled in slot order until exactly
+    identical rewards.  With shuffle=False the candidates stay in rollout order instead (the
+    members of a group adjacent, as Algorithm 1 appends them).  With exact_R the groups are filled in slot order until exactly
     exact_R candidates exist (later slots stay empty).  Tokens: n_tokens response tokens,
     resp_of_token = sorted U{0..R-1} (responses of length 0 allowed), logp ~ U[-12,-0.1],
     old_logp = logp + N(0, 0.05)."""
@@ -157,8 +158,9 @@ def make_stress(n_env: int = 16384, n_role: int = 4, n_turn: int = 4, k_max: int
     is_const = torch.zeros(G, dtype=torch.bool)
     is_const[const_groups] = True
     rewards = torch.where(is_const[slot], const_vals[slot], rewards)
-    shuffle = torch.randperm(R, generator=g)
-    slot, rewards = slot[shuffle], rewards[shuffle].contiguous()
+    order = torch.randperm(R, generator=g)
+    if shuffle:
+        slot, rewards = slot[order], rewards[order].contiguous()
     turn_id = (slot % n_turn).to(torch.int32)
     role_id = ((slot // n_turn) % n_role).to(torch.int32)
     env_id = (slot // (n_turn * n_role)).to(torch.int32)

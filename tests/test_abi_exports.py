@@ -33,8 +33,8 @@ def test_every_declared_symbol_is_exported(lib):
 
 
 def test_status_strings(lib):
-    texts = {A.status_string(c) for c in range(7)}
-    assert len(texts) == 7 and A.status_string(99) == "unknown status"
+    texts = {A.status_string(c) for c in range(8)}
+    assert len(texts) == 8 and A.status_string(99) == "unknown status"
 
 
 def test_workspace_queries_are_monotone_and_aligned(lib):
