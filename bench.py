@@ -207,12 +207,19 @@ class Runner:
                                       d["resp_of_token"], self.adv, self.old_logp, self.prm, self.loss, self.logp,
                                       self.lse, device_status=self.status, workspace=self.ws_fwd)
 
-    def backward(self):
+    def backward(self, comm_stream=None):
+        """comm_stream (multi-GPU runs): the sum of dW over the ranks runs there, chunk by chunk,
+        while the main stream computes the next vocabulary chunk."""
         d = self.d
-        self.A.atgrpo_policy_loss_bwd(d["H"], self.W, d["target"], self.role_of_token, self.head_of_role,
-                                      d["resp_of_token"], self.adv, self.old_logp, self.logp, self.lse,
-                                      self.grad_loss, self.prm, self.dH, self.dW, device_status=self.status,
-                                      workspace=self.ws_bwd)
+        kw = dict(H=d["H"], W=self.W, target=d["target"], role_of_token=self.role_of_token,
+                  head_of_role=self.head_of_role, resp_of_token=d["resp_of_token"], adv=self.adv,
+                  old_logp=self.old_logp, logp=self.logp, lse=self.lse, grad_loss=self.grad_loss,
+                  params=self.prm, dH=self.dH, dW=self.dW, device_status=self.status, workspace=self.ws_bwd)
+        if comm_stream is None:
+            self.A.atgrpo_policy_loss_bwd(**kw)
+        else:
+            from paper_2510_11062_b200 import data_parallel as DP
+            DP.backward_overlapped(self.A, kw, comm_stream)
 
     def make_old_logp(self):
         """Perf-only: old_logp = the library's own logp + N(0, 0.05) (parity runs use the oracle's)."""
@@ -265,12 +272,12 @@ def run_ours(args):
         counts = torch.bincount(heads, minlength=r.M).to(dev)
         r.grad_loss, _ = DP.token_mean_scale(counts)
 
+    comm = torch.cuda.Stream() if world > 1 else None
+
     def step():
         r.advantages()
         r.forward()
-        r.backward()
-        if world > 1:
-            DP.allreduce_gradients(r.dW)
+        r.backward(comm)
 
     ev = lambda: torch.cuda.Event(enable_timing=True)
     for _ in range(max(args.warmup, 3)):
@@ -291,9 +298,7 @@ def run_ours(args):
         marks[k][1].record()
         r.forward()
         marks[k][2].record()
-        r.backward()
-        if world > 1:
-            DP.allreduce_gradients(r.dW)
+        r.backward(comm)
         marks[k][3].record()
     t_end.record()
     torch.cuda.synchronize()

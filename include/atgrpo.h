@@ -258,6 +258,33 @@ int atgrpo_policy_loss_bwd(
     int32_t* device_status, void* workspace, size_t workspace_bytes, void* stream);
 
 /* ------------------------------------------------------------------------------------------
+ * The backward call with a notification per vocabulary chunk, for data-parallel training: the
+ * update of Sec. 3 uses the gradient of the whole batch B_m, so ranks that hold different
+ * environments sum their dW_m, and that sum can start on the rows that are final while the rest
+ * is still being computed.
+ *
+ * atgrpo_policy_loss_bwd_chunks: the backward call walks the vocabulary in *n_chunks pieces of
+ * *rows_per_chunk rows (the last one shorter); a function of (T, M, V) only.
+ * atgrpo_policy_loss_bwd_notify: as atgrpo_policy_loss_bwd; in addition chunk_events is a HOST
+ * array of n_events CUDA events (cudaEvent_t, created by the caller; n_events must equal
+ * n_chunks), and event c is recorded on `stream` as soon as the rows
+ * [c*rows_per_chunk, min(V, (c+1)*rows_per_chunk)) of every dW_m are final.  dH is final when the
+ * call's last kernel has run, as usual.  With T = 0 all events are recorded after the zero fill.
+ * ------------------------------------------------------------------------------------------ */
+int atgrpo_policy_loss_bwd_chunks(int64_t T, int32_t M, int32_t V, int32_t* n_chunks, int32_t* rows_per_chunk);
+
+int atgrpo_policy_loss_bwd_notify(
+    const void* H, int64_t ldH, const void* const* W /* host array */, int32_t M,
+    const int32_t* target,
+    const int32_t* role_of_token, const int32_t* head_of_role, int32_t n_role,
+    const int32_t* resp_of_token, const float* adv, int64_t n_resp,
+    const float* old_logp, const float* logp, const float* lse, const float* grad_loss,
+    int64_t T, int32_t d, int32_t V, const atgrpo_params* params /* host */,
+    void* dH, void* const* dW /* host array */,
+    void* const* chunk_events /* host array of cudaEvent_t */, int32_t n_events,
+    int32_t* device_status, void* workspace, size_t workspace_bytes, void* stream);
+
+/* ------------------------------------------------------------------------------------------
  * Parameter update of one policy's LM head -- theta_m <- theta_m - eta * grad L(theta_m) (Sec. 3)
  * with the optimiser settings of App. "Training Details": gradient clipping at a global L2 norm,
  * Adam with weight decay (read as AdamW: decoupled decay, bias-corrected moments).

@@ -29,6 +29,7 @@ EXPORTS = (
     "atgrpo_clipped_loss_workspace_bytes", "atgrpo_clipped_loss",
     "atgrpo_policy_loss_workspace_bytes", "atgrpo_policy_loss_launch_count",
     "atgrpo_policy_loss_fwd", "atgrpo_policy_loss_bwd",
+    "atgrpo_policy_loss_bwd_chunks", "atgrpo_policy_loss_bwd_notify",
     "atgrpo_grad_sumsq_workspace_bytes", "atgrpo_grad_sumsq", "atgrpo_adamw_step",
 )
 
@@ -127,6 +128,12 @@ def lib() -> ctypes.CDLL:
         L.atgrpo_policy_loss_bwd.argtypes = [vp, i64, ctypes.POINTER(vp), i32, vp, vp, vp, i32, vp, vp,
                                              i64, vp, vp, vp, vp, i64, i32, i32, pp, vp,
                                              ctypes.POINTER(vp), vp, vp, sz, vp]
+        L.atgrpo_policy_loss_bwd_chunks.restype = ctypes.c_int
+        L.atgrpo_policy_loss_bwd_chunks.argtypes = [i64, i32, i32, ctypes.POINTER(i32), ctypes.POINTER(i32)]
+        L.atgrpo_policy_loss_bwd_notify.restype = ctypes.c_int
+        L.atgrpo_policy_loss_bwd_notify.argtypes = [vp, i64, ctypes.POINTER(vp), i32, vp, vp, vp, i32, vp, vp,
+                                                    i64, vp, vp, vp, vp, i64, i32, i32, pp, vp,
+                                                    ctypes.POINTER(vp), ctypes.POINTER(vp), i32, vp, vp, sz, vp]
         L.atgrpo_grad_sumsq_workspace_bytes.restype = sz
         L.atgrpo_grad_sumsq_workspace_bytes.argtypes = []
         L.atgrpo_grad_sumsq.restype = ctypes.c_int
@@ -278,24 +285,44 @@ def atgrpo_policy_loss_fwd(H, W, target, role_of_token, head_of_role, resp_of_to
     _check(rc, "atgrpo_policy_loss_fwd")
 
 
+def atgrpo_policy_loss_bwd_chunks(T: int, M: int, V: int):
+    """(n_chunks, rows_per_chunk) of the vocabulary walk of one backward call; see include/atgrpo.h."""
+    n, rows = ctypes.c_int32(0), ctypes.c_int32(0)
+    _check(lib().atgrpo_policy_loss_bwd_chunks(T, M, V, ctypes.byref(n), ctypes.byref(rows)),
+           "atgrpo_policy_loss_bwd_chunks")
+    return n.value, rows.value
+
+
 def atgrpo_policy_loss_bwd(H, W, target, role_of_token, head_of_role, resp_of_token, adv, old_logp,
                            logp, lse, grad_loss, params: Params, dH, dW, device_status=None,
-                           workspace=None):
-    """Gradient of sum_m grad_loss[m]*loss[m] w.r.t. H and every W_m; see include/atgrpo.h."""
+                           workspace=None, chunk_events=None):
+    """Gradient of sum_m grad_loss[m]*loss[m] w.r.t. H and every W_m; see include/atgrpo.h.
+    With chunk_events (a list of torch.cuda.Event, one per vocabulary chunk) the call goes through
+    atgrpo_policy_loss_bwd_notify: event c is recorded when the dW rows of chunk c are final."""
     i32, f32, bf = torch.int32, torch.float32, torch.bfloat16
     T, d = H.shape
     V = W[0].shape[0]
     n_role = 0 if head_of_role is None else head_of_role.numel()
     dh_t = bf if params.dH_dtype == BF16 else f32
     dw_t = bf if params.dW_dtype == BF16 else f32
-    rc = lib().atgrpo_policy_loss_bwd(
-        ctypes.c_void_p(H.data_ptr()), H.stride(0) if T > 1 else d, _ptr_array(W, bf), len(W),
-        _ptr(target, i32), _ptr(role_of_token, i32), _ptr(head_of_role, i32), n_role,
-        _ptr(resp_of_token, i32), _ptr(adv, f32), adv.numel(), _ptr(old_logp, f32),
-        _ptr(logp, f32), _ptr(lse, f32), _ptr(grad_loss, f32), T, d, V, ctypes.byref(params.c()),
-        _ptr(dH, dh_t), _ptr_array(dW, dw_t), _ptr(device_status, i32), _ptr(workspace),
-        workspace.numel(), _stream())
-    _check(rc, "atgrpo_policy_loss_bwd")
+    head = (ctypes.c_void_p(H.data_ptr()), H.stride(0) if T > 1 else d, _ptr_array(W, bf), len(W),
+            _ptr(target, i32), _ptr(role_of_token, i32), _ptr(head_of_role, i32), n_role,
+            _ptr(resp_of_token, i32), _ptr(adv, f32), adv.numel(), _ptr(old_logp, f32),
+            _ptr(logp, f32), _ptr(lse, f32), _ptr(grad_loss, f32), T, d, V, ctypes.byref(params.c()),
+            _ptr(dH, dh_t), _ptr_array(dW, dw_t))
+    tail = (_ptr(device_status, i32), _ptr(workspace), workspace.numel(), _stream())
+    if chunk_events is None:
+        rc = lib().atgrpo_policy_loss_bwd(*head, *tail)
+        _check(rc, "atgrpo_policy_loss_bwd")
+        return
+    handles = []
+    for ev in chunk_events:
+        if not ev.cuda_event:            # torch creates the CUDA event on its first record
+            ev.record()
+        handles.append(ev.cuda_event)
+    arr = (ctypes.c_void_p * len(handles))(*handles)
+    rc = lib().atgrpo_policy_loss_bwd_notify(*head, arr, len(handles), *tail)
+    _check(rc, "atgrpo_policy_loss_bwd_notify")
 
 
 def atgrpo_grad_sumsq_workspace_bytes() -> int:

@@ -79,6 +79,18 @@ int policy_common_checks(const void* H, int64_t ldH, const void* const* W, int32
   return ATGRPO_OK;
 }
 
+// Shared body of atgrpo_policy_loss_bwd and atgrpo_policy_loss_bwd_notify (defined further down).
+int policy_loss_bwd_impl(const void* H, int64_t ldH, const void* const* W, int32_t M,
+                         const int32_t* target, const int32_t* role_of_token,
+                         const int32_t* head_of_role, int32_t n_role,
+                         const int32_t* resp_of_token, const float* adv, int64_t n_resp,
+                         const float* old_logp, const float* logp, const float* lse,
+                         const float* grad_loss, int64_t T, int32_t d, int32_t V,
+                         const atgrpo_params* params, void* dH, void* const* dW,
+                         void* const* chunk_events, int32_t n_events, bool notify,
+                         int32_t* device_status, void* workspace, size_t workspace_bytes,
+                         void* stream);
+
 }  // namespace
 
 extern "C" {
@@ -239,10 +251,55 @@ int atgrpo_policy_loss_bwd(const void* H, int64_t ldH, const void* const* W, int
                            const atgrpo_params* params, void* dH, void* const* dW,
                            int32_t* device_status, void* workspace, size_t workspace_bytes,
                            void* stream) {
+  return policy_loss_bwd_impl(H, ldH, W, M, target, role_of_token, head_of_role, n_role, resp_of_token, adv,
+                              n_resp, old_logp, logp, lse, grad_loss, T, d, V, params, dH, dW, nullptr, 0,
+                              false, device_status, workspace, workspace_bytes, stream);
+}
+
+int atgrpo_policy_loss_bwd_chunks(int64_t T, int32_t M, int32_t V, int32_t* n_chunks, int32_t* rows_per_chunk) {
+  if (T < 0 || M < 1 || V < 1 || n_chunks == nullptr || rows_per_chunk == nullptr) return ATGRPO_ERR_INVALID_ARG;
+  const int64_t T_pad = padded_rows(T, M);
+  *n_chunks = lm_head_bwd_chunks(T_pad, V);
+  *rows_per_chunk = lm_head_bwd_chunk_rows(T_pad, V);
+  return ATGRPO_OK;
+}
+
+int atgrpo_policy_loss_bwd_notify(const void* H, int64_t ldH, const void* const* W, int32_t M,
+                                  const int32_t* target, const int32_t* role_of_token,
+                                  const int32_t* head_of_role, int32_t n_role,
+                                  const int32_t* resp_of_token, const float* adv, int64_t n_resp,
+                                  const float* old_logp, const float* logp, const float* lse,
+                                  const float* grad_loss, int64_t T, int32_t d, int32_t V,
+                                  const atgrpo_params* params, void* dH, void* const* dW,
+                                  void* const* chunk_events, int32_t n_events, int32_t* device_status,
+                                  void* workspace, size_t workspace_bytes, void* stream) {
+  return policy_loss_bwd_impl(H, ldH, W, M, target, role_of_token, head_of_role, n_role, resp_of_token, adv,
+                              n_resp, old_logp, logp, lse, grad_loss, T, d, V, params, dH, dW, chunk_events,
+                              n_events, true, device_status, workspace, workspace_bytes, stream);
+}
+
+}  // extern "C"
+
+namespace {
+int policy_loss_bwd_impl(const void* H, int64_t ldH, const void* const* W, int32_t M,
+                         const int32_t* target, const int32_t* role_of_token,
+                         const int32_t* head_of_role, int32_t n_role,
+                         const int32_t* resp_of_token, const float* adv, int64_t n_resp,
+                         const float* old_logp, const float* logp, const float* lse,
+                         const float* grad_loss, int64_t T, int32_t d, int32_t V,
+                         const atgrpo_params* params, void* dH, void* const* dW,
+                         void* const* chunk_events, int32_t n_events, bool notify,
+                         int32_t* device_status, void* workspace, size_t workspace_bytes,
+                         void* stream) {
   int rc = policy_common_checks(H, ldH, W, M, target, role_of_token, head_of_role, n_role,
                                 resp_of_token, adv, n_resp, old_logp, T, d, V, params, workspace);
   if (rc != ATGRPO_OK) return rc;
   if (dW == nullptr) return ATGRPO_ERR_INVALID_ARG;
+  if (notify) {
+    if (chunk_events == nullptr || n_events != lm_head_bwd_chunks(padded_rows(T, M), V)) return ATGRPO_ERR_INVALID_ARG;
+    for (int c = 0; c < n_events; ++c)
+      if (chunk_events[c] == nullptr) return ATGRPO_ERR_INVALID_ARG;
+  }
   for (int m = 0; m < M; ++m)
     if (dW[m] == nullptr || !aligned(dW[m], 32)) return ATGRPO_ERR_INVALID_ARG;
   if (T > 0 && (logp == nullptr || lse == nullptr || dH == nullptr || !aligned(dH, 32)))
@@ -259,6 +316,8 @@ int atgrpo_policy_loss_bwd(const void* H, int64_t ldH, const void* const* W, int
     if (!params->accumulate_dW)
       for (int m = 0; m < M; ++m)
         ATGRPO_CUDA_OK(cudaMemsetAsync(dW[m], 0, (size_t)V * d * dw_elem, st));
+    for (int c = 0; notify && c < n_events; ++c)
+      ATGRPO_CUDA_OK(cudaEventRecord(static_cast<cudaEvent_t>(chunk_events[c]), st));
     return ATGRPO_OK;
   }
   Schedule* sched = reinterpret_cast<Schedule*>(ws + pl.sched);
@@ -290,8 +349,12 @@ int atgrpo_policy_loss_bwd(const void* H, int64_t ldH, const void* const* W, int
   p.M = M, p.d = d, p.V = V, p.T = T, p.T_pad = pl.T_pad;
   p.sched = sched, p.tok_of_row = tok_of_row, p.target = target, p.device_status = device_status;
   p.n_sm = n_sm;
-  return lm_head_bwd_launch(p, lse, coef, row_of_token, *params, dH, dW, ws + pl.gemm, st);
+  return lm_head_bwd_launch(p, lse, coef, row_of_token, *params, dH, dW, ws + pl.gemm, st,
+                            notify ? chunk_events : nullptr);
 }
+}  // namespace
+
+extern "C" {
 
 size_t atgrpo_grad_sumsq_workspace_bytes(void) { return grad_sumsq_workspace_bytes(); }
 

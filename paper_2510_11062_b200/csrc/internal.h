@@ -92,9 +92,13 @@ int lm_head_fwd_launch(const LmHeadProblem& p, float* lse, float* logp, void* wo
                        cudaStream_t st);
 size_t lm_head_bwd_workspace_bytes(int64_t T_pad, int32_t d, int32_t V, bool dH_direct);
 // coef[T] in token order (0 for tokens that pass no gradient); dH / dW as the C ABI documents.
+// chunk_events (optional, lm_head_bwd_chunks() entries): event c is recorded once the dW rows of
+// vocabulary chunk c are final.
 int lm_head_bwd_launch(const LmHeadProblem& p, const float* lse, const float* coef,
                        const int32_t* row_of_token, const atgrpo_params& prm, void* dH,
-                       void* const* dW, void* workspace, cudaStream_t st);
+                       void* const* dW, void* workspace, cudaStream_t st,
+                       void* const* chunk_events = nullptr);
+int lm_head_bwd_chunk_rows(int64_t T_pad, int32_t V);   // vocabulary rows per chunk
 int device_sm_count(int* n_sm, int* cc_major);
 int lm_head_bwd_chunks(int64_t T_pad, int32_t V);   // vocabulary chunks of one backward call (it makes one GEMM launch more)
 

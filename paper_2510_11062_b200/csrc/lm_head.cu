@@ -818,6 +818,8 @@ int lm_head_bwd_chunks(int64_t T_pad, int32_t V) {
   return (V + vc - 1) / vc;
 }
 
+int lm_head_bwd_chunk_rows(int64_t T_pad, int32_t V) { return bwd_chunk_width(T_pad, V); }
+
 size_t lm_head_fwd_workspace_bytes(int64_t T_pad, int32_t d, int32_t V, int32_t n_sm) {
   (void)d;
   return fwd_plan(T_pad, V, n_sm).total;
@@ -852,7 +854,7 @@ size_t lm_head_bwd_workspace_bytes(int64_t T_pad, int32_t d, int32_t V, bool dH_
 
 int lm_head_bwd_launch(const LmHeadProblem& p, const float* lse, const float* coef,
                        const int32_t* row_of_token, const atgrpo_params& prm, void* dH,
-                       void* const* dW, void* workspace, cudaStream_t st) {
+                       void* const* dW, void* workspace, cudaStream_t st, void* const* chunk_events) {
   const bool dH_direct = false;   // rows are compacted: dH always goes through the accumulator
   const BwdPlan pl = bwd_plan(p.T_pad, p.d, p.V, dH_direct);
   char* ws = static_cast<char*>(workspace);
@@ -910,6 +912,8 @@ int lm_head_bwd_launch(const LmHeadProblem& p, const float* lse, const float* co
     }
     const int rc = launch_gemm<kBwd>(maps, g, items, p.n_sm, st);
     if (rc != ATGRPO_OK) return rc;
+    if (chunk_events != nullptr && c > 0)             // the dW rows of chunk c - 1 are final
+      ATGRPO_CUDA_OK(cudaEventRecord(static_cast<cudaEvent_t>(chunk_events[c - 1]), st));
   }
   if (!dH_direct) {
     const int64_t total = p.T * (p.d / 4);

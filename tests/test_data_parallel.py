@@ -41,7 +41,14 @@ def _worker(rank, world, port, q):
     wl = torch.from_numpy(loss) * scale.double()
     dist.all_reduce(wl)
     dWt = [torch.from_numpy(w) for w in dW]
+    by_rows = [w.clone() for w in dWt]
     DP.allreduce_gradients(dWt)
+    # the same sum taken row range by row range (what the overlapped backward does chunk by chunk)
+    ranges = DP.chunk_row_ranges(spec.V, 4, 16)
+    assert ranges == [(0, 16), (16, 32), (32, 48), (48, 50)]
+    for lo, hi in ranges:
+        DP.allreduce_gradient_rows(by_rows, lo, hi)
+    assert all(torch.equal(a, b) for a, b in zip(by_rows, dWt))
     q.put((rank, adv, sh["token_index"].numpy(), dH, wl.numpy(), [w.numpy() for w in dWt], total.numpy(),
            np.nonzero(((full["env_id"] % world) == rank).numpy())[0]))
     dist.barrier()
