@@ -169,16 +169,33 @@ __global__ void __launch_bounds__(kThreads) k_clipped_loss(LossArgs a) {
   const int64_t stride = (int64_t)gridDim.x * kThreads;
   const int64_t tid = (int64_t)blockIdx.x * kThreads + threadIdx.x;
   const float inv_T = a.T > 0 ? 1.f / (float)a.T : 0.f;
-  // four consecutive tokens per thread and iteration (16-byte loads) when the arrays allow it
+  // Four consecutive tokens per thread and iteration (16-byte loads) when the arrays allow it.  The
+  // loads of the next iteration are issued before the current one is worked on, so a warp's
+  // streaming loads overlap its advantage gathers and arithmetic (all warps start in step, and
+  // without this every round of loads waited for the previous round's arithmetic).
   const int64_t n4 = a.vec ? a.T >> 2 : 0;
-  for (int64_t q = tid; q < n4; q += stride) {
-    const float4 lp = reinterpret_cast<const float4*>(a.logp)[q];
-    const float4 lo = reinterpret_cast<const float4*>(a.old_logp)[q];
-    const int4 rs = reinterpret_cast<const int4*>(a.resp)[q];
+  int64_t q = tid;
+  float4 lp = make_float4(0.f, 0.f, 0.f, 0.f), lo = lp;
+  int4 rs = make_int4(0, 0, 0, 0);
+  if (q < n4) {
+    lp = reinterpret_cast<const float4*>(a.logp)[q];
+    lo = reinterpret_cast<const float4*>(a.old_logp)[q];
+    rs = reinterpret_cast<const int4*>(a.resp)[q];
+  }
+  while (q < n4) {
+    const int64_t qn = q + stride;
+    float4 lp_n = lp, lo_n = lo;
+    int4 rs_n = rs;
+    if (qn < n4) {
+      lp_n = reinterpret_cast<const float4*>(a.logp)[qn];
+      lo_n = reinterpret_cast<const float4*>(a.old_logp)[qn];
+      rs_n = reinterpret_cast<const int4*>(a.resp)[qn];
+    }
     loss_token<kHeads>(a, 4 * q + 0, lp.x, lo.x, rs.x, inv_T, acc);
     loss_token<kHeads>(a, 4 * q + 1, lp.y, lo.y, rs.y, inv_T, acc);
     loss_token<kHeads>(a, 4 * q + 2, lp.z, lo.z, rs.z, inv_T, acc);
     loss_token<kHeads>(a, 4 * q + 3, lp.w, lo.w, rs.w, inv_T, acc);
+    q = qn, lp = lp_n, lo = lo_n, rs = rs_n;
   }
   for (int64_t j = 4 * n4 + tid; j < a.T; j += stride)
     loss_token<kHeads>(a, j, a.logp[j], a.old_logp[j], a.resp[j], inv_T, acc);
@@ -524,8 +541,16 @@ int loss_reduce_launch(const float* logp, const float* old_logp, const int32_t* 
       k_seq_scale<<<g, kThreads, 0, st>>>(coef, role_of_token, head_of_role, n_role, M, T, grad_loss, head_cnt);
     return launch_ok();
   }
-  if (M == 1) k_clipped_loss<1><<<g, kThreads, 0, st>>>(a);
-  else k_clipped_loss<0><<<g, kThreads, 0, st>>>(a);
+  // one resident wave: the grid-stride loop then keeps every thread's next loads in flight
+  // (a second wave of blocks would start cold behind the first)
+  int n_sm = 148, cc = 0, per_sm = 0, grid = g;
+  if (device_sm_count(&n_sm, &cc) != ATGRPO_OK || n_sm <= 0) n_sm = 148;
+  const cudaError_t oe = M == 1
+      ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_clipped_loss<1>, kThreads, 0)
+      : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_clipped_loss<0>, kThreads, 0);
+  if (oe == cudaSuccess && per_sm > 0 && grid > per_sm * n_sm) grid = per_sm * n_sm;
+  if (M == 1) k_clipped_loss<1><<<grid, kThreads, 0, st>>>(a);
+  else k_clipped_loss<0><<<grid, kThreads, 0, st>>>(a);
   return launch_ok();
 }
 
