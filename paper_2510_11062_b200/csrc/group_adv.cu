@@ -925,9 +925,17 @@ int group_adv_launch(const float* rewards, const int32_t* env_id, const int32_t*
     RunArgs a{rewards, env_id, role_id, turn_id, n, n_env, n_role, n_turn, adv, group_of_cand, count,
               group_mean, group_std, prm.std_eps, prm.ddof, device_status};
     const int n_tiles = (n + kRunTile - 1) / kRunTile;
-    const int grid = n_tiles < 148 * 8 ? n_tiles : 148 * 8;
     const bool vec = aligned16(env_id) && aligned16(role_id) && aligned16(turn_id) && aligned16(rewards) &&
                      aligned16(adv) && (group_of_cand == nullptr || aligned16(group_of_cand));
+    // one resident wave of blocks; each walks its tiles with a grid stride
+    int dev = 0, n_sm = 148, per_sm = 0;
+    ATGRPO_CUDA_OK(cudaGetDevice(&dev));
+    if (cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n_sm <= 0) n_sm = 148;
+    const cudaError_t oe = vec
+        ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_run_advantages<true>, kThreads, 0)
+        : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_run_advantages<false>, kThreads, 0);
+    if (oe != cudaSuccess || per_sm <= 0) per_sm = 4;
+    const int grid = n_tiles < per_sm * n_sm ? n_tiles : per_sm * n_sm;
     if (vec) k_run_advantages<true><<<grid, kThreads, 0, st>>>(a);
     else k_run_advantages<false><<<grid, kThreads, 0, st>>>(a);
     return launch_ok();
