@@ -601,15 +601,29 @@ __device__ __forceinline__ void run_stats(double ss, int K, int ddof, float std_
   inv = K > 1 ? 1.0 / (sd + (double)std_eps) : 0.0;
 }
 
+// First set bit at index >= pos in a bit array that is known to have one (the sentinel).
+__device__ __forceinline__ int next_boundary(const unsigned* bnd, int pos) {
+  int w = pos >> 5;
+  unsigned m = bnd[w] >> (pos & 31);
+  if (m) return pos + __ffs(m) - 1;
+  do m = bnd[++w];
+  while (m == 0);
+  return (w << 5) + __ffs(m) - 1;
+}
+
+constexpr int kRunBndWords = (kRunWin + 32) / 32 + 1;
+
 template <bool kVec>   // kVec: all five arrays are 16-byte aligned
-__global__ void __launch_bounds__(kThreads) k_run_advantages(RunArgs a) {
+__global__ void __launch_bounds__(kThreads, 6) k_run_advantages(RunArgs a) {
   __shared__ __align__(16) int g_s[kRunPad + kRunWin];     // g_s[kRunPad - 1] = key of the candidate before the tile
-  __shared__ __align__(16) double d_s[kRunWin];            // rewards, widened once
-  __shared__ __align__(16) float a_s[kRunWin];             // advantages
+  __shared__ __align__(16) double d_s[kRunWin];            // rewards, widened once; the low word of slot i is
+                                                           // overwritten with candidate i's advantage (float)
+  __shared__ unsigned bnd_s[kRunBndWords];                 // bit i: staged candidate i does not continue the run of i-1
   __shared__ unsigned short head_s[kRunTile];              // first members of the runs that start in the tile
   __shared__ unsigned short big_s[kRunTile / kRunWarpK + 1];   // those with more than kRunWarpK members
   __shared__ double red[kThreads];
   __shared__ int s_heads, s_big, s_lead, s_cross, s_long, s_end;
+  float* a_s = reinterpret_cast<float*>(d_s);              // advantage of candidate i at a_s[2 * i]
 
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int n_tiles = (a.n + kRunTile - 1) / kRunTile;
@@ -648,6 +662,7 @@ __global__ void __launch_bounds__(kThreads) k_run_advantages(RunArgs a) {
       d_s[i] = (double)a.rewards[c];
       if (a.gid_out && i < own) a.gid_out[c] = g;
     }
+    if (threadIdx.x < kRunBndWords) bnd_s[threadIdx.x] = 0u;
     if (threadIdx.x == 0) {
       g_s[kRunPad - 1] =
           t0 > 0 ? group_of(a.env[t0 - 1], a.role[t0 - 1], a.turn[t0 - 1], a.n_env, a.n_role, a.n_turn) : -1;
@@ -655,44 +670,51 @@ __global__ void __launch_bounds__(kThreads) k_run_advantages(RunArgs a) {
     }
     __syncthreads();
     const int* gk = g_s + kRunPad;                    // gk[i] = key of staged candidate i, gk[-1] = the one before
-
-    // Thread 0: how many leading candidates continue a run the previous tile owns, and where the
-    // run that crosses the end of this tile stops.  Everyone: list the runs that start here.
-    if (threadIdx.x == 0) {
-      int lead = 0;
-      const int gp = gk[-1];
-      if (gp >= 0)
-        while (lead < cnt && gk[lead] == gp) ++lead;
-      s_lead = lead;
-      int ce = own;
-      if (own < cnt) {
-        const int gl = gk[own - 1];                   // key of the tile's last candidate
-        if (gl >= 0)
-          while (ce < cnt && gk[ce] == gl) ++ce;
+    if (kVec && threadIdx.x < 4) {
+      // Blocks that start together stay in step (every tile costs the same), so without help all of
+      // them load, then all of them compute.  Ask L2 for this block's next tile now: HBM then works
+      // during the compute phases and the next staging loop finds its data in L2.
+      const int nt = tile + gridDim.x;
+      if (nt < n_tiles) {
+        const int nb = nt * kRunTile;
+        const int bytes = (min(kRunWin, a.n - nb) & ~3) * 4;
+        const void* src = threadIdx.x == 0 ? (const void*)(a.env + nb)
+                          : threadIdx.x == 1 ? (const void*)(a.role + nb)
+                          : threadIdx.x == 2 ? (const void*)(a.turn + nb) : (const void*)(a.rewards + nb);
+        if (bytes > 0)
+          asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(bytes) : "memory");
       }
-      s_cross = ce;
     }
+
+    // ---- mark where runs begin (whole window) and list the runs that start inside the tile
     unsigned head_bits = 0;                           // bit 4*e + j: candidate 4*(e*kThreads + threadIdx.x) + j starts a run
 #pragma unroll
-    for (int e = 0; e < kRunTile / 4 / kThreads; ++e) {
+    for (int e = 0; e < (kRunWin / 4 + kThreads - 1) / kThreads; ++e) {
       const int i0 = 4 * (e * kThreads + threadIdx.x);
-      if (i0 < own) {
+      if (i0 < cnt) {
         const int4 g = *reinterpret_cast<const int4*>(&gk[i0]);
         const int prev = gk[i0 - 1];
         const int gg[5] = {prev, g.x, g.y, g.z, g.w};
+        unsigned nib = 0;
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-          if (i0 + j < own) {
-            if (gg[j + 1] < 0) {
-              a_s[i0 + j] = 0.f;
-              raise_status(a.status, ATGRPO_ERR_BAD_INDEX);
-            } else if (gg[j + 1] != gg[j]) {
-              head_bits |= 1u << (4 * e + j);
+          if (i0 + j < cnt) {
+            const bool bad = gg[j + 1] < 0;
+            if (bad || gg[j + 1] != gg[j]) nib |= 1u << j;
+            if (i0 + j < own) {
+              if (bad) {
+                a_s[2 * (i0 + j)] = 0.f;
+                raise_status(a.status, ATGRPO_ERR_BAD_INDEX);
+              } else if (gg[j + 1] != gg[j]) {
+                head_bits |= 1u << (4 * e + j);
+              }
             }
           }
         }
+        if (nib) atomicOr(&bnd_s[i0 >> 5], nib << (i0 & 31));
       }
     }
+    if (threadIdx.x == 0) atomicOr(&bnd_s[cnt >> 5], 1u << (cnt & 31));   // sentinel: the window ends a run
     {
       // one shared-memory atomic per warp reserves the warp's slots in the run list
       const int mine = __popc(head_bits);
@@ -714,21 +736,17 @@ __global__ void __launch_bounds__(kThreads) k_run_advantages(RunArgs a) {
     }
     __syncthreads();
 
+    // Thread 0: how many leading candidates continue a run the previous tile owns, and where the
+    // run that crosses the end of this tile stops.
+    if (threadIdx.x == 0) {
+      s_lead = (bnd_s[0] & 1u) ? 0 : next_boundary(bnd_s, 1);
+      s_cross = own < cnt ? next_boundary(bnd_s, own) : own;
+    }
     // ---- one thread per run (the list is dense, so every lane works): fp64 sums in ascending order
     const int n_heads = s_heads;
     for (int h = threadIdx.x; h < n_heads; h += kThreads) {
       const int i = head_s[h];
-      const int g = gk[i];
-      const double first = d_s[i];
-      double sum = first;
-      bool all_eq = true;
-      int K = 1;
-      while (i + K < cnt && gk[i + K] == g) {         // members and their sum in one sweep
-        const double v = d_s[i + K];
-        sum += v;
-        all_eq = all_eq && (v == first);
-        ++K;
-      }
+      const int K = next_boundary(bnd_s, i + 1) - i;
       if (i + K == cnt && t0 + cnt < a.n) {           // may go on beyond the staged window
         s_long = i;
         continue;
@@ -737,20 +755,48 @@ __global__ void __launch_bounds__(kThreads) k_run_advantages(RunArgs a) {
         big_s[atomicAdd(&s_big, 1)] = (unsigned short)i;
         continue;
       }
+      const int g = gk[i];
       const int earlier = atomicAdd(&a.seen[g], 1);   // issued early: its round trip overlaps the arithmetic
+      const double* p = d_s + i;
+      const double first = p[0];
+      double sum = 0.0;
+      bool all_eq = true;
+#pragma unroll 4
+      for (int k = 0; k < K; ++k) {
+        const double v = p[k];
+        sum += v;
+        all_eq = all_eq && (v == first);
+      }
+      float* out = a_s + 2 * i;
       double mu = first, sd = 0.0;
       if (all_eq) {                                   // identical rewards: exact zeros, no rounding of the mean
-        for (int k = 0; k < K; ++k) a_s[i + k] = 0.f;
+#pragma unroll 4
+        for (int k = 0; k < K; ++k) out[2 * k] = 0.f;
       } else {
         mu = sum * c_inv_k[K];
         double ss = 0.0;
+#pragma unroll 4
         for (int k = 0; k < K; ++k) {
-          const double dlt = d_s[i + k] - mu;
+          const double dlt = p[k] - mu;
           ss = fma(dlt, dlt, ss);
         }
-        double inv;
-        run_stats(ss, K, a.ddof, a.std_eps, sd, inv);
-        for (int k = 0; k < K; ++k) a_s[i + k] = (float)((d_s[i + k] - mu) * inv);
+        // The advantage is wanted to 1e-5: the deviation r - mean is taken in fp64, std and
+        // 1/(std + eps) in fp32 (one MUFU square root and reciprocal instead of two software fp64
+        // routines per run).  A variance outside the comfortable fp32 range takes the fp64 route.
+        const int dof = K - a.ddof;
+        const double var = dof > 0 ? ss * c_inv_k[dof] : 0.0;
+        if (var < 1e30) {
+          const float sdf = sqrtf((float)var);        // an underflow to 0 is harmless: eps dominates there
+          const float invf = K > 1 ? 1.0f / (sdf + a.std_eps) : 0.f;
+          sd = (double)sdf;
+#pragma unroll 4
+          for (int k = 0; k < K; ++k) out[2 * k] = (float)(p[k] - mu) * invf;
+        } else {
+          double inv;
+          run_stats(ss, K, a.ddof, a.std_eps, sd, inv);
+#pragma unroll 4
+          for (int k = 0; k < K; ++k) out[2 * k] = (float)((p[k] - mu) * inv);
+        }
       }
       run_publish(a, g, earlier, mu, sd);
     }
@@ -762,10 +808,7 @@ __global__ void __launch_bounds__(kThreads) k_run_advantages(RunArgs a) {
     for (int b = warp; b < n_big; b += kThreads / 32) {
       const int i = big_s[b];
       const int g = gk[i];
-      int K = 0;                                      // lanes count their strided members
-      for (int k = lane; i + k < cnt && gk[i + k] == g; k += 32) ++K;
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) K += __shfl_xor_sync(0xffffffffu, K, o);
+      const int K = next_boundary(bnd_s, i + 1) - i;
       double part = 0.0;
       for (int k = lane; k < K; k += 32) part += d_s[i + k];
 #pragma unroll
@@ -780,7 +823,7 @@ __global__ void __launch_bounds__(kThreads) k_run_advantages(RunArgs a) {
       for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
       double sd, inv;
       run_stats(part, K, a.ddof, a.std_eps, sd, inv);
-      for (int k = lane; k < K; k += 32) a_s[i + k] = (float)((d_s[i + k] - mu) * inv);
+      for (int k = lane; k < K; k += 32) a_s[2 * (i + k)] = (float)((d_s[i + k] - mu) * inv);
       if (lane == 0) run_publish(a, g, atomicAdd(&a.seen[g], 1), mu, sd);
     }
     __syncthreads();
@@ -790,16 +833,21 @@ __global__ void __launch_bounds__(kThreads) k_run_advantages(RunArgs a) {
     const int lo = s_lead, hi = lh >= 0 ? lh : s_cross;   // the long run is written by the block path below
     if (kVec) {
       const int q_lo = (lo + 3) >> 2, q_hi = hi >> 2;      // whole quads inside [lo, hi)
-      for (int q = q_lo + threadIdx.x; q < q_hi; q += kThreads)
-        reinterpret_cast<float4*>(a.adv + t0)[q] = *reinterpret_cast<const float4*>(&a_s[4 * q]);
+      for (int q = q_lo + threadIdx.x; q < q_hi; q += kThreads) {
+        const double2 u = *reinterpret_cast<const double2*>(&d_s[4 * q]);
+        const double2 v = *reinterpret_cast<const double2*>(&d_s[4 * q + 2]);
+        reinterpret_cast<float4*>(a.adv + t0)[q] =
+            make_float4(__int_as_float(__double2loint(u.x)), __int_as_float(__double2loint(u.y)),
+                        __int_as_float(__double2loint(v.x)), __int_as_float(__double2loint(v.y)));
+      }
       if (q_lo < q_hi) {
-        if ((int)threadIdx.x < 4 * q_lo - lo) a.adv[t0 + lo + threadIdx.x] = a_s[lo + threadIdx.x];
-        if ((int)threadIdx.x < hi - 4 * q_hi) a.adv[t0 + 4 * q_hi + threadIdx.x] = a_s[4 * q_hi + threadIdx.x];
+        if ((int)threadIdx.x < 4 * q_lo - lo) a.adv[t0 + lo + threadIdx.x] = a_s[2 * (lo + threadIdx.x)];
+        if ((int)threadIdx.x < hi - 4 * q_hi) a.adv[t0 + 4 * q_hi + threadIdx.x] = a_s[2 * (4 * q_hi + threadIdx.x)];
       } else {
-        for (int i = lo + threadIdx.x; i < hi; i += kThreads) a.adv[t0 + i] = a_s[i];
+        for (int i = lo + threadIdx.x; i < hi; i += kThreads) a.adv[t0 + i] = a_s[2 * i];
       }
     } else {
-      for (int i = lo + threadIdx.x; i < hi; i += kThreads) a.adv[t0 + i] = a_s[i];
+      for (int i = lo + threadIdx.x; i < hi; i += kThreads) a.adv[t0 + i] = a_s[2 * i];
     }
 
     if (lh >= 0) {
