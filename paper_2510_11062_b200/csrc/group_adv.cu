@@ -578,6 +578,7 @@ __device__ __forceinline__ void run_publish(const RunArgs& a, int g, int earlier
 }
 
 constexpr int kRunWarpK = 64;                        // runs longer than this are summed by a whole warp
+constexpr int kRunRegK = 16;                         // runs up to this size are held in registers by their thread
 constexpr int kRunPad = 4;                           // g_s[kRunPad + i] = key of staged candidate i (16-byte aligned quads)
 
 // 1/k (correctly rounded by the compiler) for the divisions by a run's size in the thread-per-run
@@ -614,16 +615,14 @@ __device__ __forceinline__ int next_boundary(const unsigned* bnd, int pos) {
 constexpr int kRunBndWords = (kRunWin + 32) / 32 + 1;
 
 template <bool kVec>   // kVec: all five arrays are 16-byte aligned
-__global__ void __launch_bounds__(kThreads, 6) k_run_advantages(RunArgs a) {
+__global__ void __launch_bounds__(kThreads, 4) k_run_advantages(RunArgs a) {
   __shared__ __align__(16) int g_s[kRunPad + kRunWin];     // g_s[kRunPad - 1] = key of the candidate before the tile
-  __shared__ __align__(16) double d_s[kRunWin];            // rewards, widened once; the low word of slot i is
-                                                           // overwritten with candidate i's advantage (float)
+  __shared__ __align__(16) float r_s[kRunWin];             // rewards in; candidate i's advantage replaces its reward
   __shared__ unsigned bnd_s[kRunBndWords];                 // bit i: staged candidate i does not continue the run of i-1
   __shared__ unsigned short head_s[kRunTile];              // first members of the runs that start in the tile
   __shared__ unsigned short big_s[kRunTile / kRunWarpK + 1];   // those with more than kRunWarpK members
   __shared__ double red[kThreads];
   __shared__ int s_heads, s_big, s_lead, s_cross, s_long, s_end;
-  float* a_s = reinterpret_cast<float*>(d_s);              // advantage of candidate i at a_s[2 * i]
 
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int n_tiles = (a.n + kRunTile - 1) / kRunTile;
@@ -649,8 +648,7 @@ __global__ void __launch_bounds__(kThreads, 6) k_run_advantages(RunArgs a) {
           g.z = group_of(ev.z, rv.z, tv.z, a.n_env, a.n_role, a.n_turn);
           g.w = group_of(ev.w, rv.w, tv.w, a.n_env, a.n_role, a.n_turn);
           *reinterpret_cast<int4*>(&g_s[kRunPad + 4 * q]) = g;
-          *reinterpret_cast<double2*>(&d_s[4 * q]) = make_double2((double)w.x, (double)w.y);
-          *reinterpret_cast<double2*>(&d_s[4 * q + 2]) = make_double2((double)w.z, (double)w.w);
+          *reinterpret_cast<float4*>(&r_s[4 * q]) = w;
           if (a.gid_out && 4 * q < own) *reinterpret_cast<int4*>(&a.gid_out[t0 + 4 * q]) = g;   // own % 4 == 0 here or the tail below
         }
       }
@@ -659,7 +657,7 @@ __global__ void __launch_bounds__(kThreads, 6) k_run_advantages(RunArgs a) {
       const int c = t0 + i;
       const int g = group_of(a.env[c], a.role[c], a.turn[c], a.n_env, a.n_role, a.n_turn);
       g_s[kRunPad + i] = g;
-      d_s[i] = (double)a.rewards[c];
+      r_s[i] = a.rewards[c];
       if (a.gid_out && i < own) a.gid_out[c] = g;
     }
     if (threadIdx.x < kRunBndWords) bnd_s[threadIdx.x] = 0u;
@@ -703,7 +701,7 @@ __global__ void __launch_bounds__(kThreads, 6) k_run_advantages(RunArgs a) {
             if (bad || gg[j + 1] != gg[j]) nib |= 1u << j;
             if (i0 + j < own) {
               if (bad) {
-                a_s[2 * (i0 + j)] = 0.f;
+                r_s[i0 + j] = 0.f;
                 raise_status(a.status, ATGRPO_ERR_BAD_INDEX);
               } else if (gg[j + 1] != gg[j]) {
                 head_bits |= 1u << (4 * e + j);
@@ -757,45 +755,77 @@ __global__ void __launch_bounds__(kThreads, 6) k_run_advantages(RunArgs a) {
       }
       const int g = gk[i];
       const int earlier = atomicAdd(&a.seen[g], 1);   // issued early: its round trip overlaps the arithmetic
-      const double* p = d_s + i;
-      const double first = p[0];
-      double sum = 0.0;
-      bool all_eq = true;
-#pragma unroll 4
-      for (int k = 0; k < K; ++k) {
-        const double v = p[k];
-        sum += v;
-        all_eq = all_eq && (v == first);
-      }
-      float* out = a_s + 2 * i;
-      double mu = first, sd = 0.0;
-      if (all_eq) {                                   // identical rewards: exact zeros, no rounding of the mean
-#pragma unroll 4
-        for (int k = 0; k < K; ++k) out[2 * k] = 0.f;
-      } else {
-        mu = sum * c_inv_k[K];
-        double ss = 0.0;
-#pragma unroll 4
-        for (int k = 0; k < K; ++k) {
-          const double dlt = p[k] - mu;
-          ss = fma(dlt, dlt, ss);
+      // Shared memory is read at 32 unrelated offsets per warp (bank conflicts), so the members are
+      // fetched ONCE into registers; everything after that is register arithmetic.
+      float* p = r_s + i;
+      double mu, sd = 0.0;
+      if (K <= kRunRegK) {
+        double v[kRunRegK];
+#pragma unroll
+        for (int k = 0; k < kRunRegK; ++k) v[k] = k < K ? (double)p[k] : 0.0;
+        const double first = v[0];
+        double sum = 0.0;
+        bool all_eq = true;
+#pragma unroll
+        for (int k = 0; k < kRunRegK; ++k) {
+          sum += v[k];                                // ascending order; the padding adds exact zeros
+          all_eq = all_eq && (k >= K || v[k] == first);
         }
-        // The advantage is wanted to 1e-5: the deviation r - mean is taken in fp64, std and
-        // 1/(std + eps) in fp32 (one MUFU square root and reciprocal instead of two software fp64
-        // routines per run).  A variance outside the comfortable fp32 range takes the fp64 route.
-        const int dof = K - a.ddof;
-        const double var = dof > 0 ? ss * c_inv_k[dof] : 0.0;
-        if (var < 1e30) {
-          const float sdf = sqrtf((float)var);        // an underflow to 0 is harmless: eps dominates there
-          const float invf = K > 1 ? 1.0f / (sdf + a.std_eps) : 0.f;
-          sd = (double)sdf;
-#pragma unroll 4
-          for (int k = 0; k < K; ++k) out[2 * k] = (float)(p[k] - mu) * invf;
+        mu = first;
+        if (all_eq) {                                 // identical rewards: exact zeros, no rounding of the mean
+#pragma unroll
+          for (int k = 0; k < kRunRegK; ++k)
+            if (k < K) p[k] = 0.f;
         } else {
+          mu = sum * c_inv_k[K];
+          double ss = 0.0;
+#pragma unroll
+          for (int k = 0; k < kRunRegK; ++k) {
+            const double dlt = k < K ? v[k] - mu : 0.0;
+            ss = fma(dlt, dlt, ss);
+          }
+          // The advantage is wanted to 1e-5: the deviation r - mean is taken in fp64, std and
+          // 1/(std + eps) in fp32 (one MUFU square root and reciprocal instead of two software
+          // fp64 routines per run).  A variance outside the comfortable fp32 range takes the fp64 route.
+          const int dof = K - a.ddof;
+          const double var = dof > 0 ? ss * c_inv_k[dof] : 0.0;
+          if (var < 1e30) {
+            const float sdf = sqrtf((float)var);      // an underflow to 0 is harmless: eps dominates there
+            const float invf = 1.0f / (sdf + a.std_eps);
+            sd = (double)sdf;
+#pragma unroll
+            for (int k = 0; k < kRunRegK; ++k)
+              if (k < K) p[k] = (float)(v[k] - mu) * invf;
+          } else {
+            double inv;
+            run_stats(ss, K, a.ddof, a.std_eps, sd, inv);
+#pragma unroll
+            for (int k = 0; k < kRunRegK; ++k)
+              if (k < K) p[k] = (float)((v[k] - mu) * inv);
+          }
+        }
+      } else {
+        const double first = (double)p[0];
+        double sum = 0.0;
+        bool all_eq = true;
+        for (int k = 0; k < K; ++k) {
+          const double v = (double)p[k];
+          sum += v;
+          all_eq = all_eq && (v == first);
+        }
+        mu = first;
+        if (all_eq) {
+          for (int k = 0; k < K; ++k) p[k] = 0.f;
+        } else {
+          mu = sum * c_inv_k[K];
+          double ss = 0.0;
+          for (int k = 0; k < K; ++k) {
+            const double dlt = (double)p[k] - mu;
+            ss = fma(dlt, dlt, ss);
+          }
           double inv;
           run_stats(ss, K, a.ddof, a.std_eps, sd, inv);
-#pragma unroll 4
-          for (int k = 0; k < K; ++k) out[2 * k] = (float)((p[k] - mu) * inv);
+          for (int k = 0; k < K; ++k) p[k] = (float)(((double)p[k] - mu) * inv);
         }
       }
       run_publish(a, g, earlier, mu, sd);
@@ -810,20 +840,20 @@ __global__ void __launch_bounds__(kThreads, 6) k_run_advantages(RunArgs a) {
       const int g = gk[i];
       const int K = next_boundary(bnd_s, i + 1) - i;
       double part = 0.0;
-      for (int k = lane; k < K; k += 32) part += d_s[i + k];
+      for (int k = lane; k < K; k += 32) part += (double)r_s[i + k];
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
       const double mu = part / (double)K;
       part = 0.0;
       for (int k = lane; k < K; k += 32) {
-        const double dlt = d_s[i + k] - mu;
+        const double dlt = (double)r_s[i + k] - mu;
         part += dlt * dlt;
       }
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
       double sd, inv;
       run_stats(part, K, a.ddof, a.std_eps, sd, inv);
-      for (int k = lane; k < K; k += 32) a_s[2 * (i + k)] = (float)((d_s[i + k] - mu) * inv);
+      for (int k = lane; k < K; k += 32) r_s[i + k] = (float)(((double)r_s[i + k] - mu) * inv);
       if (lane == 0) run_publish(a, g, atomicAdd(&a.seen[g], 1), mu, sd);
     }
     __syncthreads();
@@ -833,21 +863,16 @@ __global__ void __launch_bounds__(kThreads, 6) k_run_advantages(RunArgs a) {
     const int lo = s_lead, hi = lh >= 0 ? lh : s_cross;   // the long run is written by the block path below
     if (kVec) {
       const int q_lo = (lo + 3) >> 2, q_hi = hi >> 2;      // whole quads inside [lo, hi)
-      for (int q = q_lo + threadIdx.x; q < q_hi; q += kThreads) {
-        const double2 u = *reinterpret_cast<const double2*>(&d_s[4 * q]);
-        const double2 v = *reinterpret_cast<const double2*>(&d_s[4 * q + 2]);
-        reinterpret_cast<float4*>(a.adv + t0)[q] =
-            make_float4(__int_as_float(__double2loint(u.x)), __int_as_float(__double2loint(u.y)),
-                        __int_as_float(__double2loint(v.x)), __int_as_float(__double2loint(v.y)));
-      }
+      for (int q = q_lo + threadIdx.x; q < q_hi; q += kThreads)
+        reinterpret_cast<float4*>(a.adv + t0)[q] = *reinterpret_cast<const float4*>(&r_s[4 * q]);
       if (q_lo < q_hi) {
-        if ((int)threadIdx.x < 4 * q_lo - lo) a.adv[t0 + lo + threadIdx.x] = a_s[2 * (lo + threadIdx.x)];
-        if ((int)threadIdx.x < hi - 4 * q_hi) a.adv[t0 + 4 * q_hi + threadIdx.x] = a_s[2 * (4 * q_hi + threadIdx.x)];
+        if ((int)threadIdx.x < 4 * q_lo - lo) a.adv[t0 + lo + threadIdx.x] = r_s[lo + threadIdx.x];
+        if ((int)threadIdx.x < hi - 4 * q_hi) a.adv[t0 + 4 * q_hi + threadIdx.x] = r_s[4 * q_hi + threadIdx.x];
       } else {
-        for (int i = lo + threadIdx.x; i < hi; i += kThreads) a.adv[t0 + i] = a_s[2 * i];
+        for (int i = lo + threadIdx.x; i < hi; i += kThreads) a.adv[t0 + i] = r_s[i];
       }
     } else {
-      for (int i = lo + threadIdx.x; i < hi; i += kThreads) a.adv[t0 + i] = a_s[2 * i];
+      for (int i = lo + threadIdx.x; i < hi; i += kThreads) a.adv[t0 + i] = r_s[i];
     }
 
     if (lh >= 0) {
