@@ -1,6 +1,6 @@
 // Agent- and turn-wise grouped advantage (Eq. 1 over the groups of Algorithm 1).
 //
-// Two pipelines, both on the caller's stream with no host synchronisation.
+// Three pipelines, all on the caller's stream with no host synchronisation.
 //
 // (A) Advantages only (no bucketing output requested): a sort-free group aggregate in three
 //     passes over the candidates plus one over the groups.  Everything that is accumulated with
@@ -21,14 +21,16 @@
 //   scatter    : unordered bucket fill, perm_u[offsets[g] + slot] = c
 //   stats      : one thread per group sorts its few members by candidate index (which makes the
 //                permutation stable and the fp64 sums order-fixed), then mean / std / advantage.
+//
 // (C) Adjacent groups (params.candidates_grouped): the caller promises that the members of every
 //     group are adjacent, which is the order Algorithm 1 appends them in (the K samples of one
 //     (environment, agent, turn) together).  One streaming pass: a block stages a tile of
-//     candidates in shared memory, the thread that holds the first member of a run of equal keys
-//     sums the run in fp64 in ascending order and writes the advantages back into the tile, and the
-//     tile leaves with coalesced stores; a run that outgrows the staged window is reduced by the
-//     whole block.  One integer atomic per RUN checks the promise (a key that starts two runs
-//     raises ATGRPO_ERR_LAYOUT).
+//     candidates in shared memory and marks where runs of equal keys begin; one thread per run
+//     fetches the run's members once into registers, sums them in fp64 in ascending order and
+//     writes the advantages back over the staged rewards, and the tile leaves with coalesced
+//     stores; longer runs loop over shared memory, are summed by a warp, or (beyond the staged
+//     window) by the whole block.  One integer atomic per RUN checks the promise (a key that
+//     starts two runs raises ATGRPO_ERR_LAYOUT).
 //
 // Groups of the paper hold K = 4 .. 16 candidates, far fewer than a warp, so a thread per group
 // with block-cooperative coalesced staging keeps every lane busy; blocks that meet a large group
