@@ -66,6 +66,23 @@ def test_runs_that_cross_tiles_and_outgrow_the_window(shift):
     _check(rewards, e, r, t, 14, 3, 2, ddof=1)
 
 
+def test_unaligned_pointers_take_the_scalar_staging_path():
+    s = WL.make_stress(n_env=300, n_role=2, n_turn=2, n_tokens=10, seed=8, shuffle=False)
+    R = s["R"]
+    assert R > 2 * 2048
+    pad = lambda t: torch.cat([torch.zeros(1, dtype=t.dtype), t]).to(U.DEV)[1:]   # 4-byte aligned only
+    rewards, e, r, t = pad(s["rewards"]), pad(s["env_id"]), pad(s["role_id"]), pad(s["turn_id"])
+    adv = torch.empty(R + 1, dtype=torch.float32, device=U.DEV)[1:]
+    gid = torch.empty(R + 1, dtype=torch.int32, device=U.DEV)[1:]
+    status = A.new_status(U.DEV)
+    ws = A.workspace(A.atgrpo_group_advantages_workspace_bytes(R, 1200), U.DEV)
+    A.atgrpo_group_advantages(rewards, e, r, t, 300, 2, 2, A.Params(candidates_grouped=1), adv, group_of_cand=gid,
+                              device_status=status, workspace=ws)
+    torch.cuda.synchronize()
+    ref = U.oracle_group_advantages(s["rewards"], s["env_id"], s["role_id"], s["turn_id"], 300, 2, 2)
+    U.check_group_advantages(dict(adv=adv.cpu(), group_of_cand=gid.cpu(), status=int(status.item())), ref)
+
+
 def test_single_candidate_and_constant_long_run():
     one = torch.zeros(1, dtype=torch.int32)
     gpu, _ = _check(torch.tensor([0.7]), one, one, one, 1, 1, 1)
