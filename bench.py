@@ -401,6 +401,8 @@ def run_ours(args):
                       peak_source=peaks["source"] + " sustained cuBLAS bf16",
                       flops_per_launch=pass_flops,
                       backward_dense_equiv_tflops=bwd_tf, backward_frac=bwd_tf / peaks["bf16_sustained"],
+                      backward_algorithmic_tflops=2.0 * pass_flops / (bwd_ms * 1e-3) / 1e12,   # dH + dW only
+                      backward_launches_per_call=r.A.atgrpo_policy_loss_bwd_chunks(r.T, r.M, spec.V)[0] + 1,
                       fwd_bwd_algorithmic_tflops=3.0 * pass_flops / ((fwd_ms + bwd_ms) * 1e-3) / 1e12,
                       fwd_bwd_dense_equiv_8TVd_tflops=4.0 * pass_flops / ((fwd_ms + bwd_ms) * 1e-3) / 1e12,
                       frac_of_nominal_2250=4.0 * pass_flops / ((fwd_ms + bwd_ms) * 1e-3) / 1e12 / 2250.0),
