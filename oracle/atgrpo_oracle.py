@@ -8,16 +8,17 @@ the benchmark's CPU-baseline leg call it.
 Everything is NumPy in float64.  Each function restates one definition of the
 paper (arXiv 2510.11062) in the paper's order and notation:
 
-  group_key            Algorithm 1, "define group key g <- hash(e, i, t)"
+  group_key            Algorithm 1, group-key step: one key per (environment, agent, turn)
   bucket_by_key        Algorithm 1 / Sec. 4.1 "Agent- and Turn-wise Grouping"
   group_advantages     Eq. 1 (group-relative advantage)
   mix_rewards          Eq. 3 (agent-wise credit assignment: team + local reward)
-  group_argmax         Algorithm 1, tree-structured sampling: c* = argmax_c r^(c) inside a group
+  group_argmax         Algorithm 1, greedy selection step of the tree-structured sampling
   route_tokens         Sec. 3 "Role-sharing vs. Role-specialized", B_m = U_{sigma(i)=m} D_i
   token_logprobs       pi_theta in Eq. 2: log-softmax of the LM-head logits at the sampled token
   clipped_objective    Eq. 2, per token (token-level credit, Sec. 4.1 "Reward Mask")
   policy_loss          Eq. 2, one loss per policy m (token-level reading)
-  policy_loss_sequence Eq. 2 as printed: one ratio per response, mean over the responses of B_m
+  policy_loss_sequence Eq. 2 as printed: one ratio per response; mean over the responses of B_m, or
+                       (group_of_resp given) mean over groups of the per-group mean over K candidates
   policy_loss_grads    gradient of Eq. 2 w.r.t. the hidden states H and the head W_m
   grad_sumsq, clip_scale, adamw_step
                        the update theta_m <- theta_m - eta*grad L of Sec. 3 with the optimiser
@@ -250,42 +251,72 @@ def _sequence_terms(logp, old_logp, adv, resp_of_token, head_of_token, eps_low, 
     return ids, head_c, term, r, active
 
 
+def _response_weights(ids, head_c, n_heads, group_of_resp):
+    """Weight of every present response in its policy's expectation, and the item count per policy.
+
+    group_of_resp None: every response of policy m weighs 1/R_m (R_m = its responses with tokens).
+    Otherwise Eq. 2's E_g[(1/K) sum_c .]: response c of group g weighs 1/(K_g * G_m), K_g = the
+    responses of g that have tokens, G_m = the groups of policy m that have such a response."""
+    w = np.zeros(ids.size)
+    count = np.zeros(n_heads, dtype=np.int64)
+    if group_of_resp is None:
+        for m in range(n_heads):
+            sel = head_c == m
+            count[m] = sel.sum()
+            if count[m]:
+                w[sel] = 1.0 / count[m]
+        return w, count
+    grp = _i64(group_of_resp)[ids]
+    for m in range(n_heads):
+        groups = np.unique(grp[head_c == m])
+        count[m] = groups.size
+        for g in groups:
+            members = (grp == g) & (head_c == m)
+            w[members] = 1.0 / (members.sum() * groups.size)
+    return w, count
+
+
 def policy_loss_sequence(logp, old_logp, adv, resp_of_token, head_of_token, n_heads,
-                         eps_low=0.2, eps_high=0.2):
-    """Eq. 2 read literally: L_m = -(1/R_m) sum_{responses c of policy m} min(r_c A_c, clip(r_c) A_c)
-    with the sequence-level ratio r_c; R_m counts the responses of policy m that have tokens.
-    Returns (loss[n_heads], R_m[n_heads], clip_counts[n_heads, 2]) (clip counts per response)."""
+                         eps_low=0.2, eps_high=0.2, group_of_resp=None):
+    """Eq. 2 read literally, with the sequence-level ratio r_c of every response c.
+
+    group_of_resp None: L_m = -(1/R_m) sum_{responses c of policy m} min(r_c A_c, clip(r_c) A_c),
+    R_m = the responses of policy m that have tokens.
+    group_of_resp given (the group g of every response): the expectation exactly as printed,
+    L_m = -(1/G_m) sum_g (1/K_g) sum_{c in g} min(...): every group counts once however many
+    candidates it has (K varies when rollouts end early).
+    Returns (loss[n_heads], count[n_heads] = R_m or G_m, clip_counts[n_heads, 2] per response)."""
     ids, head_c, term, r, _ = _sequence_terms(logp, old_logp, adv, resp_of_token, head_of_token,
                                               eps_low, eps_high)
+    w, count = _response_weights(ids, head_c, n_heads, group_of_resp)
     loss = np.zeros(n_heads)
-    count = np.zeros(n_heads, dtype=np.int64)
     cc = np.zeros((n_heads, 2), dtype=np.int64)
     for m in range(n_heads):
         sel = head_c == m
-        count[m] = sel.sum()
-        if count[m]:
-            loss[m] = -term[sel].sum() / count[m]
+        if sel.any():
+            loss[m] = -(w[sel] * term[sel]).sum()
             cc[m, 0] = (r[sel] < 1.0 - eps_low).sum()
             cc[m, 1] = (r[sel] > 1.0 + eps_high).sum()
     return loss, count, cc
 
 
 def dloss_dlogp_sequence(logp, old_logp, adv, resp_of_token, head_of_token, n_heads, grad_loss=None,
-                         eps_low=0.2, eps_high=0.2):
+                         eps_low=0.2, eps_high=0.2, group_of_resp=None):
     """c_j = d(sum_m grad_loss_m L_m)/d logp_j for the sequence-level loss: every token of response c
-    gets -grad_loss_m * A_c * r_c * active_c / R_m (d r_c / d logp_j = r_c)."""
+    gets -grad_loss_m * w_c * A_c * r_c * active_c (d r_c / d logp_j = r_c), w_c the response's
+    weight in the expectation (1/R_m, or 1/(K_g G_m) with group_of_resp)."""
     ids, head_c, _, r, active = _sequence_terms(logp, old_logp, adv, resp_of_token, head_of_token,
                                                 eps_low, eps_high)
     resp = _i64(resp_of_token)
     A_all = _f64(adv)
     g = np.ones(n_heads) if grad_loss is None else _f64(grad_loss)
-    count = np.bincount(head_c, minlength=n_heads).astype(np.float64)
-    per_resp = {int(c): -(g[h] / count[h]) * A_all[c] * rc * ac for c, h, rc, ac in zip(ids, head_c, r, active)}
+    w, _ = _response_weights(ids, head_c, n_heads, group_of_resp)
+    per_resp = {int(c): -g[h] * wc * A_all[c] * rc * ac for c, h, wc, rc, ac in zip(ids, head_c, w, r, active)}
     return np.array([per_resp[int(c)] for c in resp])
 
 
 def policy_loss_grads(H, W_list, target, old_logp, adv, resp_of_token, head_of_token,
-                      grad_loss=None, eps_low=0.2, eps_high=0.2, reduction="token"):
+                      grad_loss=None, eps_low=0.2, eps_high=0.2, reduction="token", group_of_resp=None):
     """Gradient of sum_m grad_loss_m * L_m (Eq. 2) w.r.t. H and every head W_m.
 
     With c_j = dL/dlogp_j and p_jv = softmax(z_j)_v:
@@ -306,8 +337,11 @@ def policy_loss_grads(H, W_list, target, old_logp, adv, resp_of_token, head_of_t
         lse = np.log(np.exp(z - z.max(axis=1, keepdims=True)).sum(axis=1)) + z.max(axis=1)
         P[m] = np.exp(z - lse[:, None])
         logp[sel] = z[np.arange(sel.size), y[sel]] - lse
-    dl = dloss_dlogp if reduction == "token" else dloss_dlogp_sequence
-    c = dl(logp, old_logp, adv, resp_of_token, head, M, grad_loss, eps_low, eps_high)
+    if reduction == "token":
+        c = dloss_dlogp(logp, old_logp, adv, resp_of_token, head, M, grad_loss, eps_low, eps_high)
+    else:                                       # "sequence"; with group_of_resp the per-group mean
+        c = dloss_dlogp_sequence(logp, old_logp, adv, resp_of_token, head, M, grad_loss, eps_low, eps_high,
+                                 group_of_resp)
     dH = np.zeros_like(Hd)
     dW = []
     for m in range(M):

@@ -440,6 +440,76 @@ def test_sequence_gradients_by_finite_differences_and_autograd():
     assert float((torch.from_numpy(loss) * gl).sum()) == pytest.approx(float(total), rel=1e-12)
 
 
+def test_group_mean_closed_form_with_unequal_group_sizes():
+    # Eq. 2's E_g[(1/K) sum_c .]: group 0 has 3 candidates, group 1 has 1, group 2 (policy 1) has 2 of
+    # which one has no token.  Ratio 1 everywhere, so the term of response c is just A_c.
+    resp = np.array([0, 0, 1, 2, 2, 2, 3, 4, 4])             # response 5 has no token
+    head = np.array([0, 0, 0, 0, 0, 0, 0, 1, 1])
+    group = np.array([0, 0, 0, 1, 2, 2])
+    adv = np.array([3.0, -1.0, 4.0, 10.0, 0.5, 99.0])
+    z = np.zeros(9)
+    loss, count, _ = O.policy_loss_sequence(z, z, adv, resp, head, 2, group_of_resp=group)
+    assert loss[0] == pytest.approx(-((3.0 - 1.0 + 4.0) / 3 + 10.0) / 2, rel=1e-14)     # two groups, equal weight
+    assert loss[1] == pytest.approx(-0.5, rel=1e-14)                                   # K counts responses WITH tokens
+    assert count.tolist() == [2, 1]
+    per_resp, _, _ = O.policy_loss_sequence(z, z, adv, resp, head, 2)
+    assert per_resp[0] == pytest.approx(-(3.0 - 1.0 + 4.0 + 10.0) / 4)                 # differs: every response equal
+    # equal K in every group: the two means coincide
+    resp2, head2 = np.arange(6), np.zeros(6, dtype=int)
+    lp, lo = -rng.random(6), -rng.random(6)
+    a, _, _ = O.policy_loss_sequence(lp, lo, adv, resp2, head2, 1, group_of_resp=np.array([0, 0, 1, 1, 2, 2]))
+    b, _, _ = O.policy_loss_sequence(lp, lo, adv, resp2, head2, 1)
+    np.testing.assert_allclose(a, b, rtol=1e-14)
+    # gradient factor: token j of response c carries -w_c * A_c * r_c (ratio 1, all unclipped)
+    c = O.dloss_dlogp_sequence(z, z, adv, resp, head, 2, group_of_resp=group)
+    want = -np.array([3.0 / 6, 3.0 / 6, -1.0 / 6, 4.0 / 6, 4.0 / 6, 4.0 / 6, 10.0 / 2, 0.5, 0.5])
+    np.testing.assert_allclose(c, want, rtol=1e-14)
+
+
+def test_group_mean_gradients_match_torch_autograd():
+    T, d, V, R, M, G = 44, 6, 30, 9, 2, 4
+    g = torch.Generator().manual_seed(29)
+    H = torch.randn(T, d, dtype=torch.float64, generator=g, requires_grad=True)
+    W = [(torch.randn(V, d, dtype=torch.float64, generator=g) * 0.4).requires_grad_() for _ in range(M)]
+    y = torch.randint(0, V, (T,), generator=g)
+    resp = torch.sort(torch.randint(0, R, (T,), generator=g)).values
+    group = torch.tensor([0, 0, 0, 1, 2, 2, 3, 3, 3])        # group sizes 3, 1, 2, 3
+    head_of_group = torch.tensor([0, 1, 0, 1])
+    head = head_of_group[group][resp]
+    adv = torch.randn(R, dtype=torch.float64, generator=g)
+    gl = torch.tensor([1.0, 0.6], dtype=torch.float64)
+    with torch.no_grad():
+        logp0 = torch.stack([torch.log_softmax(H[j] @ W[head[j]].T, 0)[y[j]] for j in range(T)])
+    old = logp0 + torch.randn(T, dtype=torch.float64, generator=g) * 0.08
+    total = 0.0
+    for m in range(M):
+        per_group = []
+        for q in range(G):
+            if head_of_group[q] != m:
+                continue
+            terms = []
+            for c in (group == q).nonzero().squeeze(1).tolist():
+                sel = (resp == c).nonzero().squeeze(1)
+                if sel.numel() == 0:
+                    continue
+                lp = torch.log_softmax(H[sel] @ W[m].T, 1)[torch.arange(sel.numel()), y[sel]]
+                r = torch.exp((lp - old[sel]).sum())
+                terms.append(torch.minimum(r * adv[c], torch.clamp(r, 0.8, 1.2) * adv[c]))
+            if terms:
+                per_group.append(torch.stack(terms).mean())
+        total = total + gl[m] * (-torch.stack(per_group).mean())
+    total.backward()
+    dH, dW = O.policy_loss_grads(H.detach().numpy(), [w.detach().numpy() for w in W], y.numpy(), old.numpy(),
+                                 adv.numpy(), resp.numpy(), head.numpy(), grad_loss=gl.numpy(),
+                                 reduction="sequence", group_of_resp=group.numpy())
+    np.testing.assert_allclose(dH, H.grad.numpy(), atol=1e-13)
+    for m in range(M):
+        np.testing.assert_allclose(dW[m], W[m].grad.numpy(), atol=1e-13)
+    loss, _, _ = O.policy_loss_sequence(logp0.numpy(), old.numpy(), adv.numpy(), resp.numpy(), head.numpy(), M,
+                                        group_of_resp=group.numpy())
+    assert float((torch.from_numpy(loss) * gl).sum()) == pytest.approx(float(total.detach()), rel=1e-12)
+
+
 # ----------------------------------------------------------------------------- Eq. 3 and greedy selection
 def test_reward_mix_and_group_argmax():
     team = np.array([1.0, 0.0, 1.0, 0.25], dtype=np.float32)
