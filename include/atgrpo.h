@@ -3,17 +3,19 @@
  * (arXiv 2510.11062) for NVIDIA B200 (sm_100a).
  *
  * Two operations of the paper are exported:
- *   - the agent- and turn-wise group-relative advantage (Eq. 1 applied to the groups of
- *     Algorithm 1, "define group key g <- hash(e, i, t)"), and
+ *   - the agent- and turn-wise group-relative advantage (Eq. 1 applied to the groups that the
+ *     group-key step of Algorithm 1 forms, one per environment, agent and turn), and
  *   - the clipped-ratio policy loss (Eq. 2) through the LM head, forward and backward, for one
  *     shared policy (M = 1) or one policy per role (M = N), Sec. 3 "Role-sharing vs.
  *     Role-specialized Policy Optimization".
  *
  * Conventions common to every entry point
  *   - Every pointer is a DEVICE pointer owned by the caller unless its comment says "host".
- *     The library allocates no memory, keeps no state between calls, never synchronises the
- *     device and enqueues all work on `stream` (a cudaStream_t passed as void*; NULL = the
- *     legacy default stream).  Scratch comes from `workspace`, at least as many bytes as the
+ *     The library allocates no memory, never synchronises the device and enqueues all work on
+ *     `stream` (a cudaStream_t passed as void*; NULL = the legacy default stream).  It keeps no
+ *     state between calls apart from two host-side lookups made once per process and cached: the
+ *     driver entry point that encodes tensor maps, and (atgrpo_group_advantages_noalloc only) the
+ *     device address of its built-in scratch array, per device.  Scratch comes from `workspace`, at least as many bytes as the
  *     matching *_workspace_bytes() query returns, 256-byte aligned, private to the call
  *     until the enqueued work has finished.
  *   - Return value: ATGRPO_OK, or an error detected on the host, in which case nothing was
@@ -65,7 +67,7 @@ typedef struct atgrpo_params {
   int32_t dH_dtype;      /* ATGRPO_BF16 (default) or ATGRPO_F32: element type of dH            */
   int32_t dW_dtype;      /* ATGRPO_F32 (default) or ATGRPO_BF16: element type of every dW_m    */
   int32_t accumulate_dW; /* 0: dW_m is overwritten; 1: dW_m += gradient (gradient accumulation)*/
-  int32_t reduction;     /* ATGRPO_REDUCE_TOKEN_MEAN (default) or ATGRPO_REDUCE_SEQUENCE           */
+  int32_t reduction;     /* ATGRPO_REDUCE_TOKEN_MEAN (default), _SEQUENCE or _GROUP_MEAN           */
   int32_t candidates_grouped; /* atgrpo_group_advantages only.  0 (default): candidates in any order.
                                * 1: the caller promises that the members of every group are adjacent,
                                * the order Algorithm 1 appends them in (the K samples of one
@@ -74,6 +76,12 @@ typedef struct atgrpo_params {
                                * pass.  The promise is checked on the device: a group that shows up in
                                * two places raises ATGRPO_ERR_LAYOUT, and its members get the statistics
                                * of their own stretch.  Ignored when bucketing outputs are requested. */
+  /* ATGRPO_REDUCE_GROUP_MEAN only (ignored otherwise; NULL / 0 by default): */
+  const int32_t* group_of_resp; /* device, [n_resp]: group g of every response, in [0, n_groups)
+                                 * (what atgrpo_group_advantages writes to group_of_cand)        */
+  int32_t* group_scratch;       /* device, [n_groups] int32 owned by the caller, private to the call
+                                 * while it runs; the library zeroes it and counts K_g in it      */
+  int32_t n_groups;
 } atgrpo_params;
 
 /* Readings of the expectation in Eq. 2.
@@ -83,8 +91,16 @@ typedef struct atgrpo_params {
  *             responses of policy m that have tokens; every token of response c then carries
  *             coef = grad_loss[m]*A_c*r_c*[unclipped branch active]/R_m.  Requires the tokens packed
  *             response by response (resp_of_token non-decreasing; a violation raises
- *             ATGRPO_ERR_BAD_INDEX); clip counts are per response. */
-enum { ATGRPO_REDUCE_TOKEN_MEAN = 0, ATGRPO_REDUCE_SEQUENCE = 1 };
+ *             ATGRPO_ERR_BAD_INDEX); clip counts are per response.
+ * GROUP_MEAN: the expectation of Eq. 2 exactly as printed, E_g[(1/K) sum_c .]: sequence-level
+ *             ratios as above, loss_m = mean over the groups g of policy m of the mean over the
+ *             K_g responses of g that have tokens, so every group weighs the same however many
+ *             candidates it kept (K varies when rollouts end early).  Token j of response c in
+ *             group g carries coef = grad_loss[m]*A_c*r_c*[active]/(K_g*G_m), G_m = groups of
+ *             policy m with at least one such response.  Needs params->group_of_resp,
+ *             group_scratch and n_groups; all responses of a group must belong to one policy.
+ *             A group id out of range raises ATGRPO_ERR_BAD_INDEX and the response is left out. */
+enum { ATGRPO_REDUCE_TOKEN_MEAN = 0, ATGRPO_REDUCE_SEQUENCE = 1, ATGRPO_REDUCE_GROUP_MEAN = 2 };
 
 /* Text for a status code (static storage, never NULL). */
 const char* atgrpo_status_string(int status);
@@ -122,8 +138,8 @@ int atgrpo_group_advantages(
     int32_t* device_status, void* workspace, size_t workspace_bytes, void* stream);
 
 /* ------------------------------------------------------------------------------------------
- * Credit assignment, advantage and greedy selection in one call -- Eq. 3, Eq. 1 and the
- * tree-structured sampling step of Algorithm 1 ("c* <- argmax_c r^(c)").
+ * Credit assignment, advantage and greedy selection in one call -- Eq. 3, Eq. 1 and the greedy
+ * selection step of Algorithm 1's tree-structured sampling (the best candidate of a group).
  *
  * rewards[c] = alpha*r_team[c] + r_loc[c] (Eq. 3, one fused multiply-add, fp32); advantages as in
  * atgrpo_group_advantages over these rewards; group_best[g] = the candidate of group g with the
@@ -154,7 +170,8 @@ int atgrpo_group_select(
  * anything larger returns ATGRPO_ERR_UNSUPPORTED with nothing enqueued.
  * The call makes no cudaMalloc / cudaFree and calls no allocating routine.  The first call on a
  * device looks up the array's device address (cudaGetSymbolAddress, with that device current)
- * and remembers it; make that first call before starting any stream capture.
+ * and remembers it for the life of the process (the remembered address does not survive a
+ * cudaDeviceReset); make that first call before starting any stream capture.
  * All calls on one device share the one array, which keeps the previous call's contents; each
  * call clears what it needs to start from zero.  Two calls whose kernels can overlap on the GPU
  * (different streams without an ordering between them) race on the array: serialise them.
@@ -319,6 +336,18 @@ int atgrpo_grad_sumsq(const void* grad, int32_t grad_dtype, int64_t n, double* s
 int atgrpo_adamw_step(const void* grad, int32_t grad_dtype, float* master, float* m, float* v,
                       void* w_bf16, int64_t n, const double* grad_sumsq,
                       const atgrpo_adamw_params* params /* host */, void* stream);
+
+/* ------------------------------------------------------------------------------------------
+ * Self-test of the bounded waits (no counterpart in the paper; it exercises the error convention
+ * stated at the top of this file).  Every barrier wait inside the LM-head kernels gives up after
+ * a wall-clock limit and reports ATGRPO_ERR_TIMEOUT; a healthy run never gets there.  This call
+ * enqueues one tiny kernel (one block, no tensor-core or bulk-copy work) whose two waiting warps
+ * wait on a barrier that nothing arrives on, with a limit of limit_ns nanoseconds (1 us .. 50 ms),
+ * and then return normally.  Afterwards *device_status holds ATGRPO_ERR_TIMEOUT (if it was 0
+ * before) and, if `waited` (device, 2 x int32, optional) is given, waited[i] = 1 for each warp
+ * whose wait returned "gave up".  The context stays usable: nothing traps or faults.
+ * ------------------------------------------------------------------------------------------ */
+int atgrpo_selftest_bounded_wait(int64_t limit_ns, int32_t* device_status, int32_t* waited, void* stream);
 
 #ifdef __cplusplus
 }

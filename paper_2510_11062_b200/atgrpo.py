@@ -18,7 +18,7 @@ LIB_PATH = os.path.join(_PKG, "libatgrpo.so")
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_BAD_INDEX, ERR_TIMEOUT, ERR_CUDA, ERR_LAYOUT = range(8)
 BF16, F32 = 0, 1
-REDUCE_TOKEN_MEAN, REDUCE_SEQUENCE = 0, 1
+REDUCE_TOKEN_MEAN, REDUCE_SEQUENCE, REDUCE_GROUP_MEAN = 0, 1, 2
 MAX_HEADS = 8
 
 EXPORTS = (
@@ -31,6 +31,7 @@ EXPORTS = (
     "atgrpo_policy_loss_fwd", "atgrpo_policy_loss_bwd",
     "atgrpo_policy_loss_bwd_chunks", "atgrpo_policy_loss_bwd_notify",
     "atgrpo_grad_sumsq_workspace_bytes", "atgrpo_grad_sumsq", "atgrpo_adamw_step",
+    "atgrpo_selftest_bounded_wait",
 )
 
 
@@ -43,7 +44,9 @@ class _Params(ctypes.Structure):
                 ("std_eps", ctypes.c_float), ("ddof", ctypes.c_int32),
                 ("dH_dtype", ctypes.c_int32), ("dW_dtype", ctypes.c_int32),
                 ("accumulate_dW", ctypes.c_int32), ("reduction", ctypes.c_int32),
-                ("candidates_grouped", ctypes.c_int32)]
+                ("candidates_grouped", ctypes.c_int32),
+                ("group_of_resp", ctypes.c_void_p), ("group_scratch", ctypes.c_void_p),
+                ("n_groups", ctypes.c_int32)]
 
 
 class _AdamWParams(ctypes.Structure):
@@ -76,13 +79,17 @@ class Params:
     dH_dtype: int = BF16
     dW_dtype: int = F32
     accumulate_dW: int = 0
-    reduction: int = 0          # REDUCE_TOKEN_MEAN or REDUCE_SEQUENCE
+    reduction: int = 0          # REDUCE_TOKEN_MEAN, REDUCE_SEQUENCE or REDUCE_GROUP_MEAN
     candidates_grouped: int = 0  # 1: the members of every group are adjacent (checked on the device)
+    group_of_resp: object = None   # REDUCE_GROUP_MEAN: int32 CUDA tensor [n_resp], group of every response
+    group_scratch: object = None   # REDUCE_GROUP_MEAN: int32 CUDA tensor [n_groups], scratch owned by the caller
 
     def c(self) -> _Params:
+        n_groups = 0 if self.group_scratch is None else self.group_scratch.numel()
+        g, sc = _ptr(self.group_of_resp, torch.int32), _ptr(self.group_scratch, torch.int32)
         return _Params(self.clip_eps_low, self.clip_eps_high, self.std_eps, self.ddof,
                        self.dH_dtype, self.dW_dtype, self.accumulate_dW, self.reduction,
-                       self.candidates_grouped)
+                       self.candidates_grouped, g.value if g else None, sc.value if sc else None, n_groups)
 
 
 _lib = None
@@ -140,6 +147,8 @@ def lib() -> ctypes.CDLL:
         L.atgrpo_grad_sumsq.argtypes = [vp, i32, i64, vp, vp, sz, vp]
         L.atgrpo_adamw_step.restype = ctypes.c_int
         L.atgrpo_adamw_step.argtypes = [vp, i32, vp, vp, vp, vp, i64, vp, ctypes.POINTER(_AdamWParams), vp]
+        L.atgrpo_selftest_bounded_wait.restype = ctypes.c_int
+        L.atgrpo_selftest_bounded_wait.argtypes = [i64, vp, vp, vp]
         _lib = L
     return _lib
 
@@ -345,3 +354,10 @@ def atgrpo_adamw_step(grad, master, m, v, w_bf16, grad_sumsq, params: AdamWParam
                                  _ptr(w_bf16, torch.bfloat16), master.numel(),
                                  _ptr(grad_sumsq, torch.float64), ctypes.byref(params.c()), _stream())
     _check(rc, "atgrpo_adamw_step")
+
+
+def atgrpo_selftest_bounded_wait(limit_ns: int, device_status, waited=None) -> int:
+    """Runs the bounded-wait self-test kernel (see include/atgrpo.h); returns the host status code."""
+    i32 = torch.int32
+    return int(lib().atgrpo_selftest_bounded_wait(int(limit_ns), _ptr(device_status, i32), _ptr(waited, i32),
+                                                  _stream()))

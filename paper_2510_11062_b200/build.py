@@ -11,7 +11,7 @@ ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 OBJ = os.path.join(PKG, "_build")
 LIB = os.path.join(PKG, "libatgrpo.so")
-SOURCES = ["api.cu", "group_adv.cu", "loss_reduce.cu", "lm_head.cu", "static_scratch.cu", "optimizer.cu"]
+SOURCES = ["api.cu", "group_adv.cu", "loss_reduce.cu", "lm_head.cu", "static_scratch.cu", "optimizer.cu", "selftest.cu"]
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
          "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC]

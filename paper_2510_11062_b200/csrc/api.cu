@@ -7,17 +7,6 @@ namespace {
 
 inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
 
-bool params_ok(const atgrpo_params* p) {
-  if (p == nullptr) return false;
-  if (!(p->clip_eps_low >= 0.f) || !(p->clip_eps_high >= 0.f) || !(p->std_eps >= 0.f)) return false;
-  if (p->ddof != 0 && p->ddof != 1) return false;
-  if (p->dH_dtype != ATGRPO_BF16 && p->dH_dtype != ATGRPO_F32) return false;
-  if (p->dW_dtype != ATGRPO_BF16 && p->dW_dtype != ATGRPO_F32) return false;
-  if (p->reduction != ATGRPO_REDUCE_TOKEN_MEAN && p->reduction != ATGRPO_REDUCE_SEQUENCE) return false;
-  if (p->candidates_grouped != 0 && p->candidates_grouped != 1) return false;
-  return true;
-}
-
 int64_t padded_rows(int64_t T, int M) {
   // every head occupies whole 256-row tiles (the row extent of a CTA pair)
   const int64_t tiles = (T + 255) / 256 + (M > 1 ? M : 0);
@@ -327,7 +316,7 @@ int policy_loss_bwd_impl(const void* H, int64_t ldH, const void* const* W, int32
   rc = routing_launch(role_of_token, head_of_role, n_role, M, T, pl.T_pad, sched, row_of_token,
                       tok_of_row, nullptr, nullptr, device_status, ws + pl.routing, st);
   if (rc != ATGRPO_OK) return rc;
-  if (params->reduction == ATGRPO_REDUCE_SEQUENCE)
+  if (params->reduction != ATGRPO_REDUCE_TOKEN_MEAN)
     rc = loss_reduce_launch(logp, old_logp, resp_of_token, adv, n_resp, role_of_token, head_of_role,
                             n_role, M, T, *params, grad_loss, nullptr, coef, nullptr, device_status,
                             ws + pl.loss, st);

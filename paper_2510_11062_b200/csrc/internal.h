@@ -4,6 +4,23 @@
 
 namespace atgrpo {
 
+// Validation of the scalar parameters, shared by every entry point that takes atgrpo_params.
+inline bool params_ok(const atgrpo_params* p) {
+  if (p == nullptr) return false;
+  if (!(p->clip_eps_low >= 0.f) || !(p->clip_eps_high >= 0.f) || !(p->std_eps >= 0.f)) return false;   // NaN fails too
+  if (p->ddof != 0 && p->ddof != 1) return false;
+  if (p->dH_dtype != ATGRPO_BF16 && p->dH_dtype != ATGRPO_F32) return false;
+  if (p->dW_dtype != ATGRPO_BF16 && p->dW_dtype != ATGRPO_F32) return false;
+  if (p->reduction != ATGRPO_REDUCE_TOKEN_MEAN && p->reduction != ATGRPO_REDUCE_SEQUENCE &&
+      p->reduction != ATGRPO_REDUCE_GROUP_MEAN)
+    return false;
+  if (p->candidates_grouped != 0 && p->candidates_grouped != 1) return false;
+  if (p->reduction == ATGRPO_REDUCE_GROUP_MEAN &&
+      (p->group_of_resp == nullptr || p->group_scratch == nullptr || p->n_groups < 1))
+    return false;
+  return true;
+}
+
 // ---- group_adv.cu ---------------------------------------------------------------------------
 // Optional extras of the advantage pipeline: Eq. 3 reward mix (rewards = alpha*r_team + r_loc,
 // written to rewards_out if given) and the per-group argmax candidate (group_best[G], -1 = empty).
@@ -34,8 +51,9 @@ struct Schedule {                       // lives in device memory
 
 // ---- loss_reduce.cu -------------------------------------------------------------------------
 // Eq. 2 reduction for up to ATGRPO_MAX_HEADS policies: token mean (coef only for M == 1) or,
-// with prm.reduction == ATGRPO_REDUCE_SEQUENCE, per-response ratios and the mean over responses
-// (coef for any M, scaled by grad_loss[m] / R_m; loss may be NULL).
+// with prm.reduction == ATGRPO_REDUCE_SEQUENCE / _GROUP_MEAN, per-response ratios and the mean
+// over responses / over groups of the per-group mean (coef for any M, scaled by grad_loss[m] / R_m
+// or grad_loss[m] / (K_g G_m); loss may be NULL).
 size_t loss_reduce_workspace_bytes(int64_t T);
 int loss_reduce_launch(const float* logp, const float* old_logp, const int32_t* resp_of_token,
                        const float* adv, int64_t n_resp, const int32_t* role_of_token,

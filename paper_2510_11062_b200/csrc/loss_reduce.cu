@@ -29,7 +29,10 @@ struct LossArgs {
   int vec;                     // logp, old_logp, resp (and coef) are 16-byte aligned
   int64_t* head_cnt;           // optional [M]: items counted per head (sequence mode keeps it for backward)
   const float* seg_term;       // sequence mode: per-response term, stored at the response's first token
-  const int32_t* seg_flags;    // sequence mode: bit 0 ratio below 1-eps_low, bit 1 above 1+eps_high
+  const int32_t* seg_flags;    // sequence mode: bit 0 ratio below 1-eps_low, bit 1 above 1+eps_high,
+                               // bit 2 first response seen of its group, bit 3 response left out (bad group id)
+  const int32_t* group_of_resp;   // group-mean mode: group of every response
+  const int32_t* group_cnt;       // group-mean mode: K_g, responses with tokens per group
 };
 
 // Per-token term of Eq. 2.  Returns l_j; `active` tells whether the unclipped branch carries the
@@ -209,6 +212,10 @@ __global__ void __launch_bounds__(kThreads) k_clipped_loss(LossArgs a) {
 // (resp_of_token non-decreasing), so a response is a segment found by binary search; one warp per
 // response sums its tokens in a fixed order.  Per-response results are parked at the response's
 // first token, which keeps the scratch proportional to T.
+// Group-mean mode (the expectation of Eq. 2 as printed): the response pass also counts K_g, the
+// responses with tokens of every group (integer atomics: order-free), and marks the response that
+// found its group's counter at zero, so the reduction can count the groups G_m; the reduction then
+// adds term_c / K_g and divides by G_m.
 __device__ __forceinline__ int64_t lower_bound_resp(const int32_t* resp, int64_t T, int c) {
   int64_t lo = 0, hi = T;
   while (lo < hi) {
@@ -223,7 +230,8 @@ __global__ void __launch_bounds__(kThreads)
 k_seq_resp(const float* __restrict__ logp, const float* __restrict__ old_logp,
            const int32_t* __restrict__ resp, const float* __restrict__ adv, int64_t n_resp, int64_t T,
            float lo, float hi, float* __restrict__ seg_term, int32_t* __restrict__ seg_flags,
-           float* __restrict__ coef_un) {
+           float* __restrict__ coef_un, const int32_t* __restrict__ group_of_resp,
+           int32_t* __restrict__ group_cnt, int n_groups, int32_t* status) {
   const int lane = threadIdx.x & 31;
   const int64_t warps = (int64_t)gridDim.x * (kThreads / 32);
   for (int64_t c = (int64_t)blockIdx.x * (kThreads / 32) + (threadIdx.x >> 5); c < n_resp; c += warps) {
@@ -239,12 +247,25 @@ k_seq_resp(const float* __restrict__ logp, const float* __restrict__ old_logp,
     const double rc = fmin(fmax(rho, (double)lo), (double)hi);
     const double u = rho * A, cl = rc * A;
     const bool active = (u <= cl) && (A != 0.0);
+    int gflag = 0;
+    if (group_cnt != nullptr) {
+      if (lane == 0) {
+        const int g = group_of_resp[c];
+        if ((unsigned)g < (unsigned)n_groups) {
+          gflag = atomicAdd(&group_cnt[g], 1) == 0 ? 4 : 0;
+        } else {
+          gflag = 8;
+          raise_status(status, ATGRPO_ERR_BAD_INDEX);
+        }
+      }
+      gflag = __shfl_sync(0xffffffffu, gflag, 0);
+    }
     if (lane == 0) {
       seg_term[beg] = (float)(-fmin(u, cl));
-      seg_flags[beg] = (rho < (double)lo ? 1 : 0) | (rho > (double)hi ? 2 : 0);
+      seg_flags[beg] = (rho < (double)lo ? 1 : 0) | (rho > (double)hi ? 2 : 0) | gflag;
     }
     if (coef_un) {
-      const float cu = active ? (float)(A * rho) : 0.f;
+      const float cu = (active && !(gflag & 8)) ? (float)(A * rho) : 0.f;
       for (int64_t j = beg + lane; j < end; j += 32) coef_un[j] = cu;
     }
   }
@@ -271,13 +292,19 @@ __global__ void __launch_bounds__(kThreads) k_seq_reduce(LossArgs a) {
         continue;
       }
     }
-    const float term = a.seg_term[j];
     const int fl = a.seg_flags[j];
+    if (fl & 8) continue;                                                    // left out: bad group id
+    double term = (double)a.seg_term[j];
+    int item = 1;
+    if (a.group_cnt != nullptr) {
+      term /= (double)a.group_cnt[a.group_of_resp[rs]];                      // K_g >= 1: this response counted itself
+      item = (fl >> 2) & 1;                                                  // one response per group counts the group
+    }
 #pragma unroll
     for (int m = 0; m < H; ++m) {
       if (m == head) {
-        acc[m].sum += (double)term;
-        acc[m].cnt += 1;
+        acc[m].sum += term;
+        acc[m].cnt += item;
         acc[m].clo += fl & 1;
         acc[m].chi += (fl >> 1) & 1;
       }
@@ -286,11 +313,14 @@ __global__ void __launch_bounds__(kThreads) k_seq_reduce(LossArgs a) {
   reduce_and_finish<kHeads>(acc, a);
 }
 
-// coef[j] (holding A*rho*[active] of the token's response) *= grad_loss[m] / R_m.
+// coef[j] (holding A*rho*[active] of the token's response) *= grad_loss[m] / R_m, or
+// grad_loss[m] / (K_g * G_m) in group-mean mode (head_cnt then holds G_m).
 __global__ void __launch_bounds__(kThreads)
 k_seq_scale(float* __restrict__ coef, const int32_t* __restrict__ role,
             const int32_t* __restrict__ head_of_role, int n_role, int M, int64_t T,
-            const float* __restrict__ grad_loss, const int64_t* __restrict__ head_cnt) {
+            const float* __restrict__ grad_loss, const int64_t* __restrict__ head_cnt,
+            const int32_t* __restrict__ resp, int64_t n_resp, const int32_t* __restrict__ group_of_resp,
+            const int32_t* __restrict__ group_cnt, int n_groups) {
   const int64_t stride = (int64_t)gridDim.x * kThreads;
   for (int64_t j = (int64_t)blockIdx.x * kThreads + threadIdx.x; j < T; j += stride) {
     int head = 0;
@@ -301,6 +331,12 @@ k_seq_scale(float* __restrict__ coef, const int32_t* __restrict__ role,
     float s = 0.f;
     if ((unsigned)head < (unsigned)M && head_cnt[head] > 0)
       s = (grad_loss ? grad_loss[head] : 1.f) / (float)head_cnt[head];
+    if (group_cnt != nullptr) {
+      const int rs = resp[j];
+      const int g = (unsigned)rs < (unsigned)n_resp ? group_of_resp[rs] : -1;
+      const int K = (unsigned)g < (unsigned)n_groups ? group_cnt[g] : 0;
+      s = K > 0 ? s / (float)K : 0.f;
+    }
     coef[j] *= s;
   }
 }
@@ -523,22 +559,30 @@ int loss_reduce_launch(const float* logp, const float* old_logp, const int32_t* 
   float* seg_term = c.take<float>((size_t)T + 1);
   int32_t* seg_flags = c.take<int32_t>((size_t)T + 1);
   a.head_cnt = nullptr, a.seg_term = nullptr, a.seg_flags = nullptr;
+  a.group_of_resp = nullptr, a.group_cnt = nullptr;
   auto al16 = [](const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; };
   a.vec = al16(logp) && al16(old_logp) && al16(resp_of_token);
   ATGRPO_CUDA_OK(cudaMemsetAsync(a.done, 0, sizeof(unsigned), st));
-  if (prm.reduction == ATGRPO_REDUCE_SEQUENCE) {
-    // per-response ratios, then the mean over responses; coef (if asked for) is scaled afterwards
+  if (prm.reduction != ATGRPO_REDUCE_TOKEN_MEAN) {
+    // per-response ratios, then the mean over responses (or over groups of the per-group mean);
+    // coef (if asked for) is scaled afterwards
+    const bool by_group = prm.reduction == ATGRPO_REDUCE_GROUP_MEAN;
+    int32_t* group_cnt = by_group ? prm.group_scratch : nullptr;
+    if (by_group) ATGRPO_CUDA_OK(cudaMemsetAsync(group_cnt, 0, (size_t)prm.n_groups * sizeof(int32_t), st));
     int64_t rg = (n_resp + kThreads / 32 - 1) / (kThreads / 32);
     if (rg > kMaxBlocks) rg = kMaxBlocks;
     if (rg < 1) rg = 1;
     k_seq_resp<<<(int)rg, kThreads, 0, st>>>(logp, old_logp, resp_of_token, adv, n_resp, T, a.lo, a.hi,
-                                             seg_term, seg_flags, coef);
+                                             seg_term, seg_flags, coef, prm.group_of_resp, group_cnt,
+                                             prm.n_groups, device_status);
     a.head_cnt = head_cnt, a.seg_term = seg_term, a.seg_flags = seg_flags;
+    if (by_group) a.group_of_resp = prm.group_of_resp, a.group_cnt = group_cnt;
     a.coef = nullptr;
     if (M == 1) k_seq_reduce<1><<<g, kThreads, 0, st>>>(a);
     else k_seq_reduce<0><<<g, kThreads, 0, st>>>(a);
     if (coef)
-      k_seq_scale<<<g, kThreads, 0, st>>>(coef, role_of_token, head_of_role, n_role, M, T, grad_loss, head_cnt);
+      k_seq_scale<<<g, kThreads, 0, st>>>(coef, role_of_token, head_of_role, n_role, M, T, grad_loss, head_cnt,
+                                          resp_of_token, n_resp, prm.group_of_resp, group_cnt, prm.n_groups);
     return launch_ok();
   }
   // one resident wave: the grid-stride loop then keeps every thread's next loads in flight

@@ -20,7 +20,8 @@ void* g_scratch_addr[kMaxDevices] = {};         // device address of g_scratch, 
 std::mutex g_mutex;
 
 // In host code `g_scratch` only names the symbol; the address a kernel can use has to be asked
-// for, once per device, while that device is current.
+// for, once per device, while that device is current.  It is cached for the life of the process
+// and would go stale if the application reset the device.
 int scratch_address(void** out) {
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return ATGRPO_ERR_CUDA;
@@ -41,8 +42,7 @@ extern "C" int atgrpo_group_advantages_noalloc(
     int64_t n_cand, int32_t n_env, int32_t n_role, int32_t n_turn, const atgrpo_params* params,
     float* adv, int32_t* group_of_cand, int32_t* group_offsets, int32_t* group_perm,
     float* group_mean, float* group_std, int32_t* device_status, void* stream) {
-  if (params == nullptr || params->std_eps < 0.f || (params->ddof != 0 && params->ddof != 1))
-    return ATGRPO_ERR_INVALID_ARG;
+  if (!atgrpo::params_ok(params)) return ATGRPO_ERR_INVALID_ARG;
   if (n_cand < 0 || n_env < 1 || n_role < 1 || n_turn < 1) return ATGRPO_ERR_INVALID_ARG;
   const int64_t G = (int64_t)n_env * n_role * n_turn;
   // sizes beyond the fixed scratch are refused before anything is enqueued

@@ -163,3 +163,42 @@ def keep_off_the_kinks(logp, old_logp, eps_lo=0.2, eps_hi=0.2, margin=2e-3):
     out = old_logp.clone()
     out[torch.from_numpy(near)] = torch.from_numpy(np.asarray(logp, np.float32))[torch.from_numpy(near)]
     return out
+
+
+def check_rows(x, ref, what, fro=5e-3, row_rel=1e-2, row_abs=1e-3):
+    """Gradient rows against the oracle's: the relative Frobenius error of the whole block (the
+    stated tolerance) AND a bound per row, |x_r - ref_r| <= row_rel*|ref_r| + row_abs*rms_r|ref_r|,
+    so that a single wrong row cannot hide inside the norm of a large block."""
+    x = np.asarray(x, dtype=np.float64)
+    ref = np.asarray(ref, dtype=np.float64)
+    assert x.shape == ref.shape, what
+    assert rel_fro(x, ref) <= fro, (what, rel_fro(x, ref))
+    norms = np.linalg.norm(ref, axis=1)
+    err = np.linalg.norm(x - ref, axis=1)
+    rms = float(np.sqrt((norms ** 2).mean())) if norms.size else 0.0
+    bound = row_rel * norms + row_abs * rms
+    worst = int(np.argmax(err - bound)) if err.size else 0
+    assert (err <= bound).all(), (what, "row", worst, float(err[worst]), float(bound[worst]))
+    zero = norms == 0.0
+    assert (x[zero] == 0.0).all(), (what, "rows that carry no gradient must be exactly zero")
+
+
+def oracle_logprobs_cached(batch, pytest_cache):
+    """oracle_logprobs for a full-size workload, kept in pytest's cache directory between runs
+    (keyed by workload, seed and the oracle's source, written from oracle/ output only)."""
+    import hashlib
+    import os
+    spec = batch["spec"]
+    src = open(O.__file__, "rb").read()
+    key = "%s_%d_%s" % (spec.name, spec.seed, hashlib.sha1(src).hexdigest()[:12])
+    path = None
+    if pytest_cache is not None:
+        path = os.path.join(str(pytest_cache.mkdir("atgrpo_oracle")), key + ".npz")
+        if os.path.exists(path):
+            z = np.load(path)
+            if z["lse"].shape[0] == batch["T"]:
+                return z["lse"], z["logp"]
+    lse, logp = oracle_logprobs(batch)
+    if path is not None:
+        np.savez(path, lse=lse, logp=logp)
+    return lse, logp

@@ -52,6 +52,8 @@ def test_workspace_queries_are_monotone_and_aligned(lib):
         assert A.atgrpo_policy_loss_workspace_bytes(0, 64, 512, 1, bwd) > 0
         assert A.atgrpo_policy_loss_workspace_bytes(1, 64, 1, 8, bwd) > 0
     assert A.atgrpo_group_advantages_workspace_bytes(0, 1) >= 0
+    # the workspace-free entry point's built-in 4 MiB array holds the plan of its documented maxima
+    assert A.atgrpo_group_advantages_workspace_bytes(A.NOALLOC_MAX_CAND, A.NOALLOC_MAX_GROUPS) <= 4 << 20
 
 
 def test_host_side_argument_checks_need_no_gpu(lib):

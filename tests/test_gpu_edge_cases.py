@@ -165,3 +165,18 @@ def test_all_advantages_zero_gives_zero_gradients():
     assert g["status"] == 0 and (g["dH"] == 0).all()
     for w in g["dW"]:
         assert (w == 0).all()
+
+
+def test_a_bounded_wait_that_runs_out_reports_timeout_and_leaves_the_context_usable():
+    # A tiny library kernel waits on a barrier nothing arrives on, with a 2 ms limit: both kinds of
+    # wait (spinning and backing off) must give up, the status word must say so, and the next
+    # regular call on the same stream must work and match the oracle.
+    dev = U.DEV
+    st = A.new_status(dev)
+    waited = torch.zeros(2, dtype=torch.int32, device=dev)
+    assert A.atgrpo_selftest_bounded_wait(2_000_000, st, waited) == A.OK
+    torch.cuda.synchronize()
+    assert int(st.item()) == A.ERR_TIMEOUT
+    assert waited.cpu().tolist() == [1, 1]
+    assert A.atgrpo_selftest_bounded_wait(10**9, st, waited) == A.ERR_INVALID_ARG     # limits are capped
+    _check(WL.make_rollout(WL.SPECS["tiny"]))

@@ -5,8 +5,11 @@ that everything the library outputs is still checkable against it:
   * lse / logp on a random sample of tokens (each needs only its own logit row);
   * advantages are made SPARSE (non-zero for a few responses spread over the batch), so loss, the
     dH rows of those responses and the COMPLETE dW of every head depend only on tokens the oracle
-    can afford, while every GEMM tile of the full-size launch still runs; all other dH rows must be
-    exactly zero;
+    can afford; all other dH rows must be exactly zero.  The backward routes only tokens with a
+    non-zero gradient factor, so these cases run few row tiles but EVERY vocabulary tile and chunk:
+    they are the complete-dW check (every one of the V rows of every head is compared), also with
+    accumulation over two micro-batches.  The dense-advantage run of every row tile is compared
+    with the oracle on sampled rows in test_gpu_full_size_dense.py;
   * identities that hold at any size on a dense-advantage run (column sums of dW, <dH,H> = <dW,W>).
 The memory-bound stress input is compared in full."""
 import numpy as np
@@ -21,14 +24,14 @@ from tests import _util as U
 pytestmark = pytest.mark.gpu
 
 
-def _sparse_case(name, n_active_resp=6, n_sample=160):
-    b = WL.make_rollout(WL.SPECS[name])
+def _sparse_case(name, n_active_resp=6, n_sample=160, shift=0, batch=None):
+    b = batch if batch is not None else WL.make_rollout(WL.SPECS[name])
     spec, T, R, M = b["spec"], b["T"], b["R"], b["spec"].n_heads
     g = torch.Generator().manual_seed(spec.seed + 7)
     head, offsets, perm = U.oracle_heads(b)
     # a few responses spread over the batch (and over the roles) carry a non-zero advantage
     active_resp = torch.linspace(1, R - 2, n_active_resp).long() + torch.arange(n_active_resp) % spec.n_role
-    active_resp = torch.unique(active_resp.clamp(max=R - 1))
+    active_resp = torch.unique((active_resp + shift).clamp(max=R - 1))
     adv = torch.zeros(R, dtype=torch.float64)
     adv[active_resp] = torch.tensor([1.0, -0.7, 0.45, -1.3, 0.8, -0.25, 0.6, -0.9])[: active_resp.numel()].double()
     resp = b["resp_of_token"].long()
@@ -86,6 +89,43 @@ def test_full_size_sparse_advantages(name):
     assert (dH[rest] == 0).all()
     for m in range(M):
         assert U.rel_fro(g["dW"][m].numpy(), dW[m]) <= 5e-3, m
+
+
+@pytest.mark.parametrize("dw_dtype", [A.F32, A.BF16])
+def test_full_size_accumulation_over_two_micro_batches(dw_dtype):
+    # gradient accumulation (App. "Training Details": a global batch is several mini-batches): two
+    # micro-batches with different active responses are accumulated into ONE dW at the full
+    # vocabulary (10 chunks), and the sum is compared row by row with the oracle's summed gradient
+    name = "qwen3_1p7b"
+    b = WL.make_rollout(WL.SPECS[name])
+    cases = [_sparse_case(name, n_active_resp=4, n_sample=8, shift=0, batch=b),
+             _sparse_case(name, n_active_resp=4, n_sample=8, shift=5, batch=b)]
+    T, d, V = b["T"], b["spec"].d, b["spec"].V
+    dev = U.DEV
+    prm = A.Params(accumulate_dW=1, dW_dtype=dw_dtype)
+    acc = [torch.zeros(V, d, dtype=torch.float32 if dw_dtype == A.F32 else torch.bfloat16, device=dev)]
+    ws = A.workspace(A.atgrpo_policy_loss_workspace_bytes(T, d, V, 1, True), dev)
+    st = A.new_status(dev)
+    dH = torch.empty(T, d, dtype=torch.bfloat16, device=dev)
+    want = np.zeros((V, d))
+    for c in cases:
+        case = U.PolicyCase(c["b"], c["adv"], c["old"], prm=prm)
+        logp_in = torch.zeros(T)
+        lse_in = torch.full((T,), 12.0)
+        logp_in[torch.from_numpy(c["sample"])] = torch.from_numpy(c["logp_s"]).float()
+        lse_in[torch.from_numpy(c["sample"])] = torch.from_numpy(c["lse_s"]).float()
+        A.atgrpo_policy_loss_bwd(case.H, case.W, case.target, None, None, case.resp_of_token, case.adv,
+                                 case.old_logp, logp_in.to(dev), lse_in.to(dev), None, prm, dH, acc, st, ws)
+        ta = torch.from_numpy(c["act"])
+        n_act = float(c["act"].size)
+        _, dW = O.policy_loss_grads(b["H"][ta], b["W"], b["target"][ta], c["old"][ta], c["adv"],
+                                    b["resp_of_token"][ta], np.zeros(c["act"].size, dtype=np.int64),
+                                    grad_loss=np.array([n_act / T]))
+        want += dW[0]
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    assert not np.array_equal(cases[0]["act"], cases[1]["act"])
+    U.check_rows(acc[0].float().cpu().numpy(), want, "accumulated dW", row_rel=1.5e-2 if dw_dtype == A.BF16 else 1e-2)
 
 
 def test_full_size_dense_identities():

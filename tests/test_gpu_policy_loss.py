@@ -2,7 +2,8 @@
 element on shapes that span several tiles and ragged tails, through the C ABI.
 Tolerances (bf16 operands, fp32 accumulation; oracle on the same bf16-rounded inputs):
 token log-probs <= 1e-3 absolute, loss <= 1e-3 relative, dH and dW <= 5e-3 relative Frobenius;
-routing bit-exact."""
+routing bit-exact.  The gradients are also held to a per-row bound (U.check_rows), so one wrong
+token or vocabulary row cannot hide inside the norm of the whole tensor."""
 import numpy as np
 import pytest
 import torch
@@ -67,9 +68,10 @@ def test_backward(name, sigma):
     out = case.bwd(torch.from_numpy(logp).float(), torch.from_numpy(lse).float())
     assert out["status"] == 0
     dH, dW = _oracle_grads(b, adv, old, gl)
-    assert U.rel_fro(out["dH"].numpy(), dH) <= 5e-3
+    # whole-tensor relative Frobenius error AND a bound on every single row (token / vocabulary id)
+    U.check_rows(out["dH"].numpy(), dH, "dH")
     for m in range(M):
-        assert U.rel_fro(out["dW"][m].numpy(), dW[m]) <= 5e-3
+        U.check_rows(out["dW"][m].numpy(), dW[m], "dW[%d]" % m)
     # rows that carry no gradient (clipped ratio or zero advantage) are exactly zero
     zero_rows = np.abs(dH).sum(1) == 0
     assert zero_rows.any() and (out["dH"].numpy()[zero_rows] == 0).all()
