@@ -28,12 +28,35 @@ sys.path.insert(0, ROOT)
 
 from paper_2510_11062_b200 import workloads as WL  # noqa: E402
 
-# DRAM bytes (read + write) of ONE forward-sweep launch, from a 1-pass ncu capture of
-#   ncu --metrics dram__bytes_read.sum,dram__bytes_write.sum --clock-control none -k regex:k_lm_head
-#       --launch-skip 1 --launch-count 12 python bench.py --steps 1 --warmup 3 --no-cpu-baseline
-# (profiles/k_lm_head_qwen3_1p7b_dram_traffic.txt).  Valid for the kernel as captured; set the entry
-# to None when k_lm_head<kFwd> or its tiling changes.
-FWD_SWEEP_DRAM_BYTES = {"qwen3_1p7b": 2.08e9 + 79.5e6}   # capture of the current kernel (earlier builds: 1.34 - 2.64 GB read, timing dependent)
+# DRAM bytes of the k_lm_head launches of one step come from an earlier 1-pass ncu capture, kept in
+# profiles/k_lm_head_dram_traffic.json together with a digest of the kernel sources it was taken on
+# (profiles/k_lm_head_qwen3_1p7b_dram_traffic.txt says how to retake it).  They are reported only
+# while that digest still matches the sources: after any change to the kernel `traffic` is null.
+TRAFFIC_JSON = os.path.join(ROOT, "profiles", "k_lm_head_dram_traffic.json")
+KERNEL_SOURCES = ("lm_head.cu", "sm100.cuh")
+
+
+def kernel_digest():
+    import hashlib
+    h = hashlib.sha1()
+    for f in KERNEL_SOURCES:
+        with open(os.path.join(ROOT, "paper_2510_11062_b200", "csrc", f), "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()[:16]
+
+
+def captured_traffic(workload):
+    """(forward bytes, backward bytes) of one step's k_lm_head launches, or None."""
+    try:
+        with open(TRAFFIC_JSON) as f:
+            rec = json.load(f)
+    except (OSError, ValueError):
+        return None
+    e = rec.get("workloads", {}).get(workload)
+    if e is None or rec.get("kernel_digest") != kernel_digest():
+        return None
+    return float(e["forward_bytes"]), float(e["backward_bytes"])
+
 
 METRIC = "fused AT-GRPO loss fwd+bwd tokens/sec"
 UNIT = "tokens/s"
@@ -101,7 +124,7 @@ def run_reference(args):
     total = sum(times)
     value = n * len(times) / total
     sample = f"first {n} tokens of the batch, full vocabulary, fwd+bwd, plus advantages of all {batch['R']} candidates"
-    line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=args.gpus, steps=args.steps, warmup=args.warmup,
+    line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=1, steps=args.steps, warmup=args.warmup,
                 ms_per_step=1e3 * total / len(times), higher_is_better=True, scaling="weak", vs_baseline=None,
                 dtype="f64", data="synthetic", impl="reference",
                 config=dict(workload=spec.name, d=spec.d, V=spec.V, tokens=batch["T"], heads=spec.n_heads),
@@ -230,6 +253,18 @@ class Runner:
         self.host["old_logp"] = old.pin_memory()
         self.old_logp.copy_(self.host["old_logp"])
 
+    def count_routed_rows(self):
+        """Tokens whose gradient factor is non-zero: the rows the backward's three contractions run
+        on (the others -- clipped ratio or zero advantage -- are skipped).  Counted once, outside any
+        timed region, from the library's own factor (which tokens are non-zero does not depend on the head)."""
+        coef = torch.empty(self.T, dtype=torch.float32, device=self.dev)
+        loss = torch.zeros(1, dtype=torch.float32, device=self.dev)
+        ws = self.A.workspace(self.A.atgrpo_clipped_loss_workspace_bytes(self.T), self.dev)
+        self.A.atgrpo_clipped_loss(self.logp, self.old_logp, self.d["resp_of_token"], self.adv, self.prm, loss, coef,
+                                   None, self.status, ws)
+        torch.cuda.synchronize()
+        self.routed_rows = int((coef != 0).sum().item())
+
     def make_second_input_set(self):
         """A second set of device input buffers, so that the next step's inputs can be copied from
         the host while the current step runs."""
@@ -280,6 +315,7 @@ def run_ours(args):
 
     r = Runner(batch, dev, A)
     r.make_old_logp()
+    r.count_routed_rows()
     if world > 1:
         heads = batch["head_of_role"].long()[batch["role_of_token"].long()]
         counts = torch.bincount(heads, minlength=r.M).to(dev)
@@ -378,10 +414,26 @@ def run_ours(args):
     bwd_ms = statistics.mean(m[2].elapsed_time(m[3]) for m in marks)
     peaks = measured_peaks()
     pass_flops = 2.0 * r.T * spec.V * spec.d                  # one T x V x d contraction
-    fwd_tf = pass_flops / (fwd_ms * 1e-3) / 1e12
-    # dense-equivalent: logits recompute + dH + dW over ALL tokens (the backward skips rows with a
-    # zero gradient factor, about 3 % of this input, so slightly fewer flops are actually executed)
-    bwd_tf = 3.0 * pass_flops / (bwd_ms * 1e-3) / 1e12
+    lm_s = (fwd_ms + bwd_ms) * 1e-3                           # every k_lm_head launch of a step sits in these two calls
+    tf = lambda flops, sec: flops / sec / 1e12
+    # The roofline is that of the STEP's dominant kernel, k_lm_head, over all its launches (one
+    # forward sweep + one launch per vocabulary chunk + 1 in the backward): algorithmic work
+    # 6*T*V*d (logits, dH, dW) over the forward + backward time.  Beside it: what the tensor cores
+    # actually executed -- the forward on all T rows, and the backward's three contractions (logit
+    # recompute, dH, dW) on the rows that carry a gradient (counted on the device, outside the
+    # timed region) -- and the two calls on their own.
+    algo_tf = tf(3.0 * pass_flops, lm_s)
+    executed_flops = pass_flops * (1.0 + 3.0 * r.routed_rows / max(r.T, 1))
+    exec_tf = tf(executed_flops, lm_s)
+    traffic = captured_traffic(spec.name) if world == 1 else None
+    n_bwd_chunks = r.A.atgrpo_policy_loss_bwd_chunks(r.T, r.M, spec.V)[0]
+    dw_elem, dh_elem = 4.0, 2.0
+    fwd_bytes = 2.0 * spec.d * (spec.V * spec.n_heads + r.T)                        # W and H once
+    bwd_bytes = (2.0 * spec.d * (2 * spec.V * spec.n_heads + 3 * r.routed_rows)     # W for logits and dH; H for logits, dW + gather
+                 + 3.0 * 2.0 * r.routed_rows * spec.V                               # dZ written once, read by dH and by dW
+                 + dw_elem * spec.V * spec.d * spec.n_heads                         # dW written once
+                 + 2.0 * 4.0 * r.routed_rows * spec.d * n_bwd_chunks                # fp32 dH accumulator, once per chunk
+                 + dh_elem * r.T * spec.d)                                          # dH out
     value = tokens_all * args.steps / (ms_total * 1e-3)
     line = dict(
         metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=max(args.warmup, 3),
@@ -393,19 +445,29 @@ def run_ours(args):
                     old_logp="library logp + N(0,0.05) (perf-only input)"),
         gpu_launches=(r.launches) * args.steps,
         phases_ms=dict(advantages=adv_ms, forward=fwd_ms, backward=bwd_ms),
-        roofline=dict(bound="tensor", kernel="k_lm_head<kFwd> (forward call: routing + logits/logsumexp sweep "
-                      "+ combine + Eq. 2 reduction)", achieved=fwd_tf, peak=peaks["bf16_sustained"],
-                      unit="TFLOP/s", frac=fwd_tf / peaks["bf16_sustained"],
-                      traffic=FWD_SWEEP_DRAM_BYTES.get(spec.name) if world == 1 else None,
-                      algorithmic_bytes=2.0 * spec.d * (spec.V * spec.n_heads + r.T),
-                      peak_source=peaks["source"] + " sustained cuBLAS bf16",
-                      flops_per_launch=pass_flops,
-                      backward_dense_equiv_tflops=bwd_tf, backward_frac=bwd_tf / peaks["bf16_sustained"],
-                      backward_algorithmic_tflops=2.0 * pass_flops / (bwd_ms * 1e-3) / 1e12,   # dH + dW only
-                      backward_launches_per_call=r.A.atgrpo_policy_loss_bwd_chunks(r.T, r.M, spec.V)[0] + 1,
-                      fwd_bwd_algorithmic_tflops=3.0 * pass_flops / ((fwd_ms + bwd_ms) * 1e-3) / 1e12,
-                      fwd_bwd_dense_equiv_8TVd_tflops=4.0 * pass_flops / ((fwd_ms + bwd_ms) * 1e-3) / 1e12,
-                      frac_of_nominal_2250=4.0 * pass_flops / ((fwd_ms + bwd_ms) * 1e-3) / 1e12 / 2250.0),
+        roofline=dict(bound="tensor",
+                      kernel="k_lm_head, all launches of a step (forward sweep + %d backward launches)" % (n_bwd_chunks + 1),
+                      achieved=algo_tf, peak=peaks["bf16_sustained"], unit="TFLOP/s",
+                      frac=algo_tf / peaks["bf16_sustained"],
+                      peak_source=peaks["source"] + " sustained cuBLAS bf16 (the kernel is timed inside a long step)",
+                      flops="algorithmic 6*T*V*d = %.4g per step" % (3.0 * pass_flops),
+                      traffic=None if traffic is None else traffic[0] + traffic[1],
+                      traffic_source="profiles/k_lm_head_dram_traffic.json (earlier ncu capture of these sources)"
+                      if traffic is not None else "no capture of the current kernel sources",
+                      traffic_forward=None if traffic is None else traffic[0],
+                      traffic_backward=None if traffic is None else traffic[1],
+                      algorithmic_bytes=fwd_bytes + bwd_bytes, algorithmic_bytes_forward=fwd_bytes,
+                      algorithmic_bytes_backward=bwd_bytes,
+                      executed_tflops=exec_tf, executed_frac=exec_tf / peaks["bf16_sustained"],
+                      executed="forward on %d rows + recompute, dH, dW on the %d rows with a gradient" % (r.T, r.routed_rows),
+                      routed_rows=r.routed_rows,
+                      frac_of_nominal_2250=algo_tf / 2250.0, executed_frac_of_nominal_2250=exec_tf / 2250.0,
+                      forward_tflops=tf(pass_flops, fwd_ms * 1e-3),
+                      forward_frac=tf(pass_flops, fwd_ms * 1e-3) / peaks["bf16_sustained"],
+                      backward_algorithmic_tflops=tf(2.0 * pass_flops, bwd_ms * 1e-3),      # dH + dW
+                      backward_algorithmic_frac=tf(2.0 * pass_flops, bwd_ms * 1e-3) / peaks["bf16_sustained"],
+                      backward_executed_tflops=tf(3.0 * pass_flops * r.routed_rows / max(r.T, 1), bwd_ms * 1e-3),
+                      backward_launches_per_call=n_bwd_chunks + 1),
         e2e=dict(value=tokens_all * args.steps / (ms_e2e * 1e-3), unit=UNIT,
                  h2d_bytes_per_step=r.h2d_bytes, d2h_bytes_per_step=r.M * 4),
         clocks=clocks, cpu_baseline=cpu_baseline)
@@ -527,6 +589,43 @@ def run_adamw(args):
     print(json.dumps(line), flush=True)
 
 
+def relaunch_with_ranks(args):
+    """`python bench.py --gpus N` with N > 1 and no launcher around it: start N ranks of this same
+    script, one per GPU, through torch.distributed.run on 127.0.0.1 (what the documented torchrun
+    command does) and pass their exit code on.  Rank 0 prints the one JSON line."""
+    import socket
+    with socket.socket(socket.AF_INET, socket.SOCK_STREAM) as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    raise SystemExit(subprocess.call(cmd))
+
+
+def run_launcher_check(args):
+    """--launcher-check: what a multi-rank run does around the step, with no GPU and no kernel: every
+    rank joins a gloo group, draws its own batch's shape, the token counts are summed over the
+    ranks and rank 0 prints one line with "value": null.  It measures nothing; it exists so that
+    the rank start-up of `--gpus N` can be tested on a machine without GPUs."""
+    import torch.distributed as dist
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    if world > 1:
+        dist.init_process_group("gloo")
+    spec = WL.SPECS[args.workload]
+    spec = WL.RolloutSpec(**{**spec.__dict__, "seed": spec.seed + 1000 * rank})
+    tokens = torch.tensor([float(WL.make_rollout(spec, with_weights=False)["T"])], dtype=torch.float64)
+    if world > 1:
+        dist.all_reduce(tokens)
+        dist.barrier()
+        dist.destroy_process_group()
+    if rank == 0:
+        print(json.dumps(dict(metric=METRIC, value=None, unit=UNIT, n_gpus=world, steps=args.steps,
+                              warmup=args.warmup, launcher_check=True, scaling="weak",
+                              config=dict(workload=spec.name, parallelism=f"dp{world}",
+                                          tokens_all_ranks=tokens.item()))), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -535,8 +634,17 @@ def main():
     ap.add_argument("--workload", default="qwen3_1p7b", choices=sorted(WL.SPECS) + ["stress", "stress16", "stress_grouped", "stress16_grouped", "adamw"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--launcher-check", action="store_true",
+                    help="start the ranks, join a gloo group, print a line with value null; no GPU work")
     args = ap.parse_args()
-    if args.workload == "adamw":
+    world_env = os.environ.get("WORLD_SIZE")
+    if args.gpus > 1 and world_env is None and args.impl == "ours":
+        relaunch_with_ranks(args)                 # does not return
+    if world_env is not None and int(world_env) != args.gpus and int(os.environ.get("RANK", "0")) == 0:
+        print(f"bench.py: --gpus {args.gpus} but WORLD_SIZE={world_env}; running {world_env} ranks", file=sys.stderr)
+    if args.launcher_check:
+        run_launcher_check(args)
+    elif args.workload == "adamw":
         run_adamw(args)
     elif args.workload.startswith("stress"):
         run_stress(args)

@@ -30,6 +30,15 @@ def test_default_arm_line():
     rf = r["roofline"]
     assert rf["bound"] == "tensor" and rf["unit"] == "TFLOP/s" and rf["peak"] > 0
     assert abs(rf["frac"] - rf["achieved"] / rf["peak"]) < 1e-9
+    # the roofline is the whole step's: algorithmic 6*T*V*d over forward + backward time
+    ph = r["phases_ms"]
+    T, d, V = r["config"]["tokens_per_gpu"], r["config"]["d"], r["config"]["V"]
+    want = 6.0 * T * V * d / ((ph["forward"] + ph["backward"]) * 1e-3) / 1e12
+    assert abs(rf["achieved"] - want) <= 1e-6 * want and "all launches" in rf["kernel"]
+    assert 0 < rf["routed_rows"] <= T and rf["executed_frac"] >= rf["frac"] * 0.99
+    assert rf["frac_of_nominal_2250"] < rf["frac"] and rf["forward_frac"] > 0 and rf["backward_algorithmic_frac"] > 0
+    assert rf["algorithmic_bytes"] == rf["algorithmic_bytes_forward"] + rf["algorithmic_bytes_backward"]
+    assert rf["traffic"] is None or rf["traffic"] == rf["traffic_forward"] + rf["traffic_backward"]
     e = r["e2e"]
     assert e["value"] > 0 and e["h2d_bytes_per_step"] > 0 and e["d2h_bytes_per_step"] == 4
     c = r["cpu_baseline"]
@@ -38,7 +47,7 @@ def test_default_arm_line():
 
 def test_reference_arm_line():
     r = _run("--workload", "tiny", "--impl", "reference", "--steps", "2", "--warmup", "1")
-    assert r["impl"] == "reference" and r["dtype"] == "f64" and r["value"] > 0
+    assert r["impl"] == "reference" and r["dtype"] == "f64" and r["value"] > 0 and r["n_gpus"] == 1
     assert r["cpu_baseline"]["kind"] == "oracle" and r["cpu_baseline"]["value"] == r["value"]
     assert r["e2e"] == dict(value=r["value"], unit=r["unit"], h2d_bytes_per_step=0, d2h_bytes_per_step=0)
 
