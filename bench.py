@@ -185,7 +185,9 @@ class ClockSampler:
 class Runner:
     """Device-resident state of one rank: inputs, outputs, workspaces; step() enqueues the path."""
 
-    def __init__(self, batch, device, A):
+    def __init__(self, batch, device, A, W=None, dW=None, accumulate=False):
+        """W / dW: device tensors shared with other Runners (micro-batches of one update step);
+        accumulate: this Runner's backward adds into dW instead of overwriting it."""
         self.A = A
         self.dev = device
         spec = self.spec = batch["spec"]
@@ -194,10 +196,10 @@ class Runner:
         self.host = {k: batch[k].pin_memory() for k in
                      ("rewards", "env_id", "role_id", "turn_id", "H", "target", "resp_of_token", "role_of_token")}
         self.d = {k: v.to(device) for k, v in self.host.items()}
-        self.W = [w.to(device) for w in batch["W"]]
+        self.W = W if W is not None else [w.to(device) for w in batch["W"]]
         self.head_of_role = batch["head_of_role"].to(device) if self.M > 1 else None
         self.role_of_token = self.d["role_of_token"] if self.M > 1 else None
-        self.prm = A.Params()
+        self.prm = A.Params(accumulate_dW=1 if accumulate else 0)
         G = spec.n_env * spec.n_role * spec.n_turn
         T, V, dm, M = self.T, spec.V, spec.d, self.M
         self.adv = torch.zeros(self.R, dtype=f32, device=device)
@@ -206,7 +208,7 @@ class Runner:
         self.lse = torch.zeros(T, dtype=f32, device=device)
         self.old_logp = torch.zeros(T, dtype=f32, device=device)
         self.dH = torch.zeros(T, dm, dtype=torch.bfloat16, device=device)
-        self.dW = [torch.zeros(V, dm, dtype=f32, device=device) for _ in range(M)]
+        self.dW = dW if dW is not None else [torch.zeros(V, dm, dtype=f32, device=device) for _ in range(M)]
         self.grad_loss = None
         self.status = A.new_status(device)
         self.ws_adv = A.workspace(A.atgrpo_group_advantages_workspace_bytes(self.R, G), device)
@@ -474,6 +476,113 @@ def run_ours(args):
     print(json.dumps(line), flush=True)
 
 
+def run_update_step(args):
+    """Workload batch128: one policy update at the paper's batch scale (App. "Training Details":
+    global batch 128, responses of up to 4096 tokens, gradient clipping at 1.0, Adam with lr 1e-6 and
+    weight decay 0.01).  128 responses of 512-2048 tokens (T >> 100 K in total) are processed as two
+    micro-batches of 64 responses each -- advantages, forward, backward -- whose dW are ACCUMULATED
+    into one fp32 gradient (the second backward runs with accumulate_dW; each micro-batch weighs
+    T_i / T_total so the sum is the token mean over the whole batch), followed by the gradient norm
+    and one clipped AdamW step that rewrites the bf16 head.  value = tokens of the whole batch per
+    second of the whole update."""
+    from paper_2510_11062_b200 import atgrpo as A
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    A.lib()
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    base = WL.SPECS["long_resp"]
+    n_micro = 2
+    batches = [WL.make_rollout(WL.RolloutSpec(**{**base.__dict__, "seed": base.seed + 10 * i}),
+                               with_weights=(i == 0)) for i in range(n_micro)]
+    g = torch.Generator().manual_seed(base.seed + 99)
+    for b in batches[1:]:
+        b["H"] = torch.randn(b["T"], base.d, generator=g, dtype=torch.float32).to(torch.bfloat16)
+        b["W"] = batches[0]["W"]
+    V, dm = base.V, base.d
+    W = [batches[0]["W"][0].to(dev)]
+    dW = [torch.zeros(V, dm, dtype=torch.float32, device=dev)]
+    runners = [Runner(b, dev, A, W=W, dW=dW, accumulate=(i > 0)) for i, b in enumerate(batches)]
+    T_all = sum(r.T for r in runners)
+    for r in runners:
+        r.make_old_logp()
+        r.count_routed_rows()
+        r.grad_loss = torch.tensor([r.T / T_all], dtype=torch.float32, device=dev)
+    master = W[0].float().clone()
+    m1, m2 = torch.zeros_like(master), torch.zeros_like(master)
+    sumsq = torch.zeros(1, dtype=torch.float64, device=dev)
+    ws_n = A.workspace(A.atgrpo_grad_sumsq_workspace_bytes(), dev)
+    step_no = [0]
+
+    def step():
+        for r in runners:
+            r.advantages()
+            r.forward()
+            r.backward()
+        step_no[0] += 1
+        A.atgrpo_grad_sumsq(dW[0].view(-1), sumsq, ws_n)
+        A.atgrpo_adamw_step(dW[0].view(-1), master.view(-1), m1.view(-1), m2.view(-1), W[0].view(-1), sumsq,
+                            A.AdamWParams(step=step_no[0]))
+
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(local)
+    marks = [[ev() for _ in range(3)] for _ in range(args.steps)]
+    t0, t1 = ev(), ev()
+    t0.record()
+    for k in range(args.steps):
+        marks[k][0].record()
+        for r in runners:
+            r.advantages()
+            r.forward()
+            r.backward()
+        marks[k][1].record()
+        step_no[0] += 1
+        A.atgrpo_grad_sumsq(dW[0].view(-1), sumsq, ws_n)
+        A.atgrpo_adamw_step(dW[0].view(-1), master.view(-1), m1.view(-1), m2.view(-1), W[0].view(-1), sumsq,
+                            A.AdamWParams(step=step_no[0]))
+        marks[k][2].record()
+    t1.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    for r in runners:
+        st = int(r.status.item())
+        if st != 0:
+            raise SystemExit(f"device status {st}: {A.status_string(st)}")
+    ms_total = t0.elapsed_time(t1)
+    grad_ms = statistics.mean(m[0].elapsed_time(m[1]) for m in marks)
+    opt_ms = statistics.mean(m[1].elapsed_time(m[2]) for m in marks)
+    peaks = measured_peaks()
+    algo_tf = 6.0 * T_all * V * dm / (grad_ms * 1e-3) / 1e12
+    routed = sum(r.routed_rows for r in runners)
+    exec_tf = 2.0 * V * dm * (T_all + 3.0 * routed) / (grad_ms * 1e-3) / 1e12
+    n_par = V * dm
+    launches = sum(r.launches for r in runners) + 2
+    line = dict(
+        metric="AT-GRPO update step (accumulated micro-batches + clipped AdamW) tokens/sec",
+        value=T_all * args.steps / (ms_total * 1e-3), unit=UNIT, n_gpus=1, steps=args.steps,
+        warmup=max(args.warmup, 3), ms_per_step=ms_total / args.steps, higher_is_better=True, scaling="weak",
+        vs_baseline=None, dtype="bf16", data="synthetic",
+        config=dict(workload="batch128", d=dm, V=V, heads=1, responses=sum(r.R for r in runners), tokens=T_all,
+                    micro_batches=[r.T for r in runners], accumulate_dW="fp32, second micro-batch adds",
+                    optimizer="grad norm + AdamW(lr 1e-6, wd 0.01, clip 1.0) on the head, bf16 head rewritten",
+                    l2="inputs larger than L2", old_logp="library logp + N(0,0.05) (perf-only input)"),
+        gpu_launches=launches * args.steps,
+        phases_ms=dict(gradient=grad_ms, optimizer=opt_ms),
+        roofline=dict(bound="tensor", kernel="k_lm_head, all launches of the update step", achieved=algo_tf,
+                      peak=peaks["bf16_sustained"], unit="TFLOP/s", frac=algo_tf / peaks["bf16_sustained"],
+                      peak_source=peaks["source"] + " sustained cuBLAS bf16", traffic=None,
+                      executed_tflops=exec_tf, executed_frac=exec_tf / peaks["bf16_sustained"], routed_rows=routed,
+                      optimizer_gbs=34.0 * n_par / (opt_ms * 1e-3) / 1e9,
+                      optimizer_frac_of_hbm=34.0 * n_par / (opt_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                      optimizer_bytes="4 B (norm) + 30 B (update) per parameter"),
+        clocks=clocks)
+    print(json.dumps(line), flush=True)
+
+
 def run_stress(args):
     """Memory-bound workload: grouped advantages over 262144 (env, role, turn) slots and the Eq. 2
     reduction over 4 Mi tokens (x scale).  L2 is flushed before every timed call (outside the
@@ -485,10 +594,12 @@ def run_stress(args):
     dev = torch.device("cuda", int(os.environ.get("LOCAL_RANK", "0")))
     torch.cuda.set_device(dev)
     scale = 16 if args.workload.startswith("stress16") else 1
-    grouped = args.workload.endswith("_grouped")     # rollout order: the members of a group adjacent
+    grouped = "_grouped" in args.workload            # rollout order: the members of a group adjacent
+    packed = args.workload.endswith("_packed")       # one dense group id per candidate instead of three id arrays
     s = WL.make_stress(n_env=16384 * scale, n_tokens=4_194_304 * scale, shuffle=not grouped)
     R, G, T = s["R"], s["G"], s["T"]
-    d = {k: s[k].to(dev) for k in ("rewards", "env_id", "role_id", "turn_id", "resp_of_token", "logp", "old_logp")}
+    d = {k: s[k].to(dev) for k in ("rewards", "env_id", "role_id", "turn_id", "group_id", "resp_of_token", "logp",
+                                   "old_logp")}
     adv = torch.empty(R, device=dev)
     loss = torch.zeros(1, device=dev)
     status = A.new_status(dev)
@@ -498,8 +609,12 @@ def run_stress(args):
     prm = A.Params(candidates_grouped=1 if grouped else 0)
 
     def f_adv():
-        A.atgrpo_group_advantages(d["rewards"], d["env_id"], d["role_id"], d["turn_id"], s["n_env"], s["n_role"],
-                                  s["n_turn"], prm, adv, device_status=status, workspace=ws_a)
+        if packed:
+            A.atgrpo_group_advantages_packed(d["rewards"], d["group_id"], G, prm, adv, device_status=status,
+                                             workspace=ws_a)
+        else:
+            A.atgrpo_group_advantages(d["rewards"], d["env_id"], d["role_id"], d["turn_id"], s["n_env"], s["n_role"],
+                                      s["n_turn"], prm, adv, device_status=status, workspace=ws_a)
 
     def f_loss():
         A.atgrpo_clipped_loss(d["logp"], d["old_logp"], d["resp_of_token"], adv, prm, loss, None, None, status, ws_l)
@@ -523,14 +638,16 @@ def run_stress(args):
     if int(status.item()) != 0:
         raise SystemExit("device status %d" % int(status.item()))
     peaks = measured_peaks()
-    adv_gbs = 20.0 * R / (adv_ms * 1e-3) / 1e9
+    cand_bytes = 12.0 if packed else 20.0           # reward + ids (one packed id, or env/role/turn) + advantage
+    adv_gbs = cand_bytes * R / (adv_ms * 1e-3) / 1e9
     loss_bytes = 12.0 * T + 4.0 * R                 # logp, old_logp, response index per token; each advantage once
     loss_gbs = loss_bytes / (loss_ms * 1e-3) / 1e9
-    line = dict(metric="grouped advantage HBM GB/s (20 B per candidate)", value=adv_gbs, unit="GB/s", n_gpus=1,
+    line = dict(metric="grouped advantage HBM GB/s (%d B per candidate)" % cand_bytes, value=adv_gbs, unit="GB/s", n_gpus=1,
                 steps=args.steps, warmup=max(args.warmup, 3), ms_per_step=adv_ms, higher_is_better=True,
                 scaling="weak", vs_baseline=None, dtype="f32", data="synthetic",
                 config=dict(workload=args.workload, candidates=R, group_slots=G, tokens=T,
                             candidate_order="rollout order (groups adjacent)" if grouped else "shuffled",
+                            group_ids="one packed id per candidate" if packed else "env, role, turn arrays",
                             l2="flushed before every timed call"),
                 gpu_launches=(1 if grouped else 4) * args.steps,
                 roofline=dict(bound="hbm", kernel="k_run_advantages (one pass)" if grouped else
@@ -631,7 +748,8 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--workload", default="qwen3_1p7b", choices=sorted(WL.SPECS) + ["stress", "stress16", "stress_grouped", "stress16_grouped", "adamw"])
+    ap.add_argument("--workload", default="qwen3_1p7b", choices=sorted(WL.SPECS) + ["stress", "stress16", "stress_grouped", "stress16_grouped", "stress_grouped_packed",
+                                                                     "stress16_grouped_packed", "stress_packed", "adamw", "batch128"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--launcher-check", action="store_true",
@@ -646,6 +764,8 @@ def main():
         run_launcher_check(args)
     elif args.workload == "adamw":
         run_adamw(args)
+    elif args.workload == "batch128":
+        run_update_step(args)
     elif args.workload.startswith("stress"):
         run_stress(args)
     elif args.impl == "reference":

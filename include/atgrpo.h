@@ -138,6 +138,23 @@ int atgrpo_group_advantages(
     int32_t* device_status, void* workspace, size_t workspace_bytes, void* stream);
 
 /* ------------------------------------------------------------------------------------------
+ * Grouped advantage from ready-made group ids -- Eq. 1 again, for callers that already hold the
+ * group key of Algorithm 1 as one dense id per candidate (for instance the group_of_cand output
+ * of an earlier call, or an id assigned when the rollout was stored under its key): group_id[c]
+ * in [0, n_groups) replaces the three id arrays, which saves 8 of the 20 bytes the call moves per
+ * candidate.  Everything else -- params (ddof, std_eps, candidates_grouped), outputs, error
+ * reporting (an id out of range raises ATGRPO_ERR_BAD_INDEX and gets adv = 0), workspace size
+ * (atgrpo_group_advantages_workspace_bytes) -- is as in atgrpo_group_advantages.
+ * ------------------------------------------------------------------------------------------ */
+int atgrpo_group_advantages_packed(
+    const float* rewards, const int32_t* group_id, int64_t n_cand, int64_t n_groups,
+    const atgrpo_params* params /* host */,
+    float* adv,
+    int32_t* group_offsets, int32_t* group_perm,
+    float* group_mean, float* group_std,
+    int32_t* device_status, void* workspace, size_t workspace_bytes, void* stream);
+
+/* ------------------------------------------------------------------------------------------
  * Credit assignment, advantage and greedy selection in one call -- Eq. 3, Eq. 1 and the greedy
  * selection step of Algorithm 1's tree-structured sampling (the best candidate of a group).
  *

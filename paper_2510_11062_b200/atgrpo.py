@@ -24,7 +24,7 @@ MAX_HEADS = 8
 EXPORTS = (
     "atgrpo_status_string",
     "atgrpo_group_advantages_workspace_bytes", "atgrpo_group_advantages",
-    "atgrpo_group_advantages_noalloc",
+    "atgrpo_group_advantages_noalloc", "atgrpo_group_advantages_packed",
     "atgrpo_group_select_workspace_bytes", "atgrpo_group_select",
     "atgrpo_clipped_loss_workspace_bytes", "atgrpo_clipped_loss",
     "atgrpo_policy_loss_workspace_bytes", "atgrpo_policy_loss_launch_count",
@@ -114,6 +114,8 @@ def lib() -> ctypes.CDLL:
         L.atgrpo_group_advantages_noalloc.restype = ctypes.c_int
         L.atgrpo_group_advantages_noalloc.argtypes = [vp, vp, vp, vp, i64, i32, i32, i32, pp, vp, vp, vp, vp,
                                                       vp, vp, vp, vp]
+        L.atgrpo_group_advantages_packed.restype = ctypes.c_int
+        L.atgrpo_group_advantages_packed.argtypes = [vp, vp, i64, i64, pp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
         L.atgrpo_group_select_workspace_bytes.restype = sz
         L.atgrpo_group_select_workspace_bytes.argtypes = [i64, i64]
         L.atgrpo_group_select.restype = ctypes.c_int
@@ -209,6 +211,18 @@ def atgrpo_group_advantages(rewards, env_id, role_id, turn_id, n_env, n_role, n_
         _ptr(group_mean, f32), _ptr(group_std, f32), _ptr(device_status, i32),
         _ptr(workspace), workspace.numel(), _stream())
     _check(rc, "atgrpo_group_advantages")
+
+
+def atgrpo_group_advantages_packed(rewards, group_id, n_groups, params: Params, adv, group_offsets=None,
+                                   group_perm=None, group_mean=None, group_std=None, device_status=None,
+                                   workspace=None):
+    """Eq. 1 from one dense group id per candidate instead of the three id arrays; see include/atgrpo.h."""
+    i32, f32 = torch.int32, torch.float32
+    rc = lib().atgrpo_group_advantages_packed(
+        _ptr(rewards, f32), _ptr(group_id, i32), rewards.numel(), n_groups, ctypes.byref(params.c()),
+        _ptr(adv, f32), _ptr(group_offsets, i32), _ptr(group_perm, i32), _ptr(group_mean, f32),
+        _ptr(group_std, f32), _ptr(device_status, i32), _ptr(workspace), workspace.numel(), _stream())
+    _check(rc, "atgrpo_group_advantages_packed")
 
 
 NOALLOC_MAX_CAND, NOALLOC_MAX_GROUPS = 262144, 65536

@@ -123,6 +123,23 @@ int atgrpo_group_advantages(const float* rewards, const int32_t* env_id, const i
                           device_status, workspace, static_cast<cudaStream_t>(stream));
 }
 
+int atgrpo_group_advantages_packed(const float* rewards, const int32_t* group_id, int64_t n_cand,
+                                   int64_t n_groups, const atgrpo_params* params, float* adv,
+                                   int32_t* group_offsets, int32_t* group_perm, float* group_mean,
+                                   float* group_std, int32_t* device_status, void* workspace,
+                                   size_t workspace_bytes, void* stream) {
+  if (!params_ok(params)) return ATGRPO_ERR_INVALID_ARG;
+  if (n_cand < 0 || n_groups < 1) return ATGRPO_ERR_INVALID_ARG;
+  if (n_groups >= 2147483647ll || n_cand >= 2147483647ll) return ATGRPO_ERR_UNSUPPORTED;
+  if (n_cand > 0 && (rewards == nullptr || group_id == nullptr || adv == nullptr)) return ATGRPO_ERR_INVALID_ARG;
+  if (workspace == nullptr || !aligned(workspace, 256) ||
+      workspace_bytes < group_adv_workspace_bytes(n_cand, n_groups))
+    return ATGRPO_ERR_WORKSPACE;
+  return group_adv_launch(rewards, group_id, nullptr, nullptr, n_cand, (int32_t)n_groups, 1, 1, *params, adv,
+                          nullptr, group_offsets, group_perm, group_mean, group_std, device_status, workspace,
+                          static_cast<cudaStream_t>(stream), nullptr, true);
+}
+
 size_t atgrpo_group_select_workspace_bytes(int64_t n_cand, int64_t n_groups) {
   return group_select_workspace_bytes(n_cand, n_groups);
 }

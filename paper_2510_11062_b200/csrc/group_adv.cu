@@ -53,7 +53,9 @@ __device__ __forceinline__ int group_of(int e, int i, int t, int n_env, int n_ro
   return ok ? (e * n_role + i) * n_turn + t : -1;
 }
 
-template <bool kVec>
+// kPacked (here and in k_hash_minmax): `env` holds ready-made group ids in [0, n_env) and the
+// role / turn arrays are not read (n_role = n_turn = 1).
+template <bool kVec, bool kPacked>
 __global__ void __launch_bounds__(kThreads)
 k_key_count(const int32_t* __restrict__ env, const int32_t* __restrict__ role,
             const int32_t* __restrict__ turn, int n, int n_env, int n_role, int n_turn,
@@ -65,8 +67,9 @@ k_key_count(const int32_t* __restrict__ env, const int32_t* __restrict__ role,
     const int n4 = n >> 2;
     for (int q = tid; q < n4; q += stride) {
       const int4 e = reinterpret_cast<const int4*>(env)[q];
-      const int4 r = reinterpret_cast<const int4*>(role)[q];
-      const int4 t = reinterpret_cast<const int4*>(turn)[q];
+      const int4 zero = make_int4(0, 0, 0, 0);
+      const int4 r = kPacked ? zero : reinterpret_cast<const int4*>(role)[q];
+      const int4 t = kPacked ? zero : reinterpret_cast<const int4*>(turn)[q];
       int4 g, s;
       g.x = group_of(e.x, r.x, t.x, n_env, n_role, n_turn);
       g.y = group_of(e.y, r.y, t.y, n_env, n_role, n_turn);
@@ -89,7 +92,7 @@ k_key_count(const int32_t* __restrict__ env, const int32_t* __restrict__ role,
   }
   const int first = kVec ? (n & ~3) : 0;
   for (int c = first + tid; c < n; c += stride) {
-    const int g = group_of(env[c], role[c], turn[c], n_env, n_role, n_turn);
+    const int g = group_of(env[c], kPacked ? 0 : role[c], kPacked ? 0 : turn[c], n_env, n_role, n_turn);
     gid[c] = g;
     if (g >= 0) {
       slot[c] = atomicAdd(&count[g], 1);
@@ -216,7 +219,7 @@ __device__ __forceinline__ void minmax_one(int g, float r, int c, const GroupTab
   if (t.best) atomicMax(&t.best[g], ((unsigned long long)e << 32) | (0xFFFFFFFFu - (uint32_t)c));
 }
 
-template <bool kVec>
+template <bool kVec, bool kPacked>
 __global__ void __launch_bounds__(kThreads)
 k_hash_minmax(const int32_t* __restrict__ env, const int32_t* __restrict__ role,
               const int32_t* __restrict__ turn, const float* __restrict__ rewards, int n, int n_env,
@@ -228,8 +231,9 @@ k_hash_minmax(const int32_t* __restrict__ env, const int32_t* __restrict__ role,
     const int n4 = n >> 2;
     for (int q = tid; q < n4; q += stride) {
       const int4 e = reinterpret_cast<const int4*>(env)[q];
-      const int4 r = reinterpret_cast<const int4*>(role)[q];
-      const int4 u = reinterpret_cast<const int4*>(turn)[q];
+      const int4 zero = make_int4(0, 0, 0, 0);
+      const int4 r = kPacked ? zero : reinterpret_cast<const int4*>(role)[q];
+      const int4 u = kPacked ? zero : reinterpret_cast<const int4*>(turn)[q];
       const float4 w = reinterpret_cast<const float4*>(rewards)[q];
       int4 g;
       g.x = group_of(e.x, r.x, u.x, n_env, n_role, n_turn);
@@ -252,7 +256,7 @@ k_hash_minmax(const int32_t* __restrict__ env, const int32_t* __restrict__ role,
   }
   const int first = kVec ? (n & ~3) : 0;
   for (int c = first + tid; c < n; c += stride) {
-    const int g = group_of(env[c], role[c], turn[c], n_env, n_role, n_turn);
+    const int g = group_of(env[c], kPacked ? 0 : role[c], kPacked ? 0 : turn[c], n_env, n_role, n_turn);
     gid[c] = g;
     if (g >= 0) {
       minmax_one(g, rewards[c], c, t);
@@ -616,7 +620,9 @@ __device__ __forceinline__ int next_boundary(const unsigned* bnd, int pos) {
 
 constexpr int kRunBndWords = (kRunWin + 32) / 32 + 1;
 
-template <bool kVec>   // kVec: all five arrays are 16-byte aligned
+// kVec: all five arrays are 16-byte aligned.  kPacked: a.env holds ready-made group ids in
+// [0, n_env) and the role / turn arrays are not read (n_role = n_turn = 1).
+template <bool kVec, bool kPacked>
 __global__ void __launch_bounds__(kThreads, 4) k_run_advantages(RunArgs a) {
   __shared__ __align__(16) int g_s[kRunPad + kRunWin];     // g_s[kRunPad - 1] = key of the candidate before the tile
   __shared__ __align__(16) float r_s[kRunWin];             // rewards in; candidate i's advantage replaces its reward
@@ -641,8 +647,9 @@ __global__ void __launch_bounds__(kThreads, 4) k_run_advantages(RunArgs a) {
         if (q < n_quads) {
           const int c4 = (t0 >> 2) + q;
           const int4 ev = reinterpret_cast<const int4*>(a.env)[c4];
-          const int4 rv = reinterpret_cast<const int4*>(a.role)[c4];
-          const int4 tv = reinterpret_cast<const int4*>(a.turn)[c4];
+          const int4 zero = make_int4(0, 0, 0, 0);
+          const int4 rv = kPacked ? zero : reinterpret_cast<const int4*>(a.role)[c4];
+          const int4 tv = kPacked ? zero : reinterpret_cast<const int4*>(a.turn)[c4];
           const float4 w = reinterpret_cast<const float4*>(a.rewards)[c4];
           int4 g;
           g.x = group_of(ev.x, rv.x, tv.x, a.n_env, a.n_role, a.n_turn);
@@ -657,20 +664,21 @@ __global__ void __launch_bounds__(kThreads, 4) k_run_advantages(RunArgs a) {
     }
     for (int i = 4 * n_quads + threadIdx.x; i < cnt; i += kThreads) {
       const int c = t0 + i;
-      const int g = group_of(a.env[c], a.role[c], a.turn[c], a.n_env, a.n_role, a.n_turn);
+      const int g = group_of(a.env[c], kPacked ? 0 : a.role[c], kPacked ? 0 : a.turn[c], a.n_env, a.n_role, a.n_turn);
       g_s[kRunPad + i] = g;
       r_s[i] = a.rewards[c];
       if (a.gid_out && i < own) a.gid_out[c] = g;
     }
     if (threadIdx.x < kRunBndWords) bnd_s[threadIdx.x] = 0u;
     if (threadIdx.x == 0) {
-      g_s[kRunPad - 1] =
-          t0 > 0 ? group_of(a.env[t0 - 1], a.role[t0 - 1], a.turn[t0 - 1], a.n_env, a.n_role, a.n_turn) : -1;
+      g_s[kRunPad - 1] = t0 > 0 ? group_of(a.env[t0 - 1], kPacked ? 0 : a.role[t0 - 1], kPacked ? 0 : a.turn[t0 - 1],
+                                           a.n_env, a.n_role, a.n_turn)
+                                : -1;
       s_long = -1, s_heads = 0, s_big = 0;
     }
     __syncthreads();
     const int* gk = g_s + kRunPad;                    // gk[i] = key of staged candidate i, gk[-1] = the one before
-    if (kVec && threadIdx.x < 4) {
+    if (kVec && threadIdx.x < 4 && !(kPacked && (threadIdx.x == 1 || threadIdx.x == 2))) {
       // Blocks that start together stay in step (every tile costs the same), so without help all of
       // them load, then all of them compute.  Ask L2 for this block's next tile now: HBM then works
       // during the compute phases and the next staging loop finds its data in L2.
@@ -884,8 +892,8 @@ __global__ void __launch_bounds__(kThreads, 4) k_run_advantages(RunArgs a) {
       int end = t0 + cnt;                             // equal up to here
       for (;;) {
         const int c = end + threadIdx.x;
-        const bool same = c < a.n &&
-                          group_of(a.env[c], a.role[c], a.turn[c], a.n_env, a.n_role, a.n_turn) == g;
+        const bool same = c < a.n && group_of(a.env[c], kPacked ? 0 : a.role[c], kPacked ? 0 : a.turn[c], a.n_env,
+                                              a.n_role, a.n_turn) == g;
         const int n_same = __syncthreads_count(same);
         if (n_same == kThreads) {
           end += kThreads;
@@ -961,7 +969,9 @@ int group_adv_launch(const float* rewards, const int32_t* env_id, const int32_t*
                      int32_t n_turn, const atgrpo_params& prm, float* adv, int32_t* group_of_cand,
                      int32_t* group_offsets, int32_t* group_perm, float* group_mean,
                      float* group_std, int32_t* device_status, void* workspace, cudaStream_t st,
-                     const GroupExtras* ex) {
+                     const GroupExtras* ex, bool packed) {
+  // packed: env_id holds ready-made group ids in [0, n_env); role_id / turn_id are not read
+  if (packed) n_role = 1, n_turn = 1;
   const int64_t G = (int64_t)n_env * n_role * n_turn;
   const int n = (int)n_cand;
   const Plan pl = make_plan(n_cand, G);
@@ -1000,19 +1010,23 @@ int group_adv_launch(const float* rewards, const int32_t* env_id, const int32_t*
     RunArgs a{rewards, env_id, role_id, turn_id, n, n_env, n_role, n_turn, adv, group_of_cand, count,
               group_mean, group_std, prm.std_eps, prm.ddof, device_status};
     const int n_tiles = (n + kRunTile - 1) / kRunTile;
-    const bool vec = aligned16(env_id) && aligned16(role_id) && aligned16(turn_id) && aligned16(rewards) &&
-                     aligned16(adv) && (group_of_cand == nullptr || aligned16(group_of_cand));
+    const bool vec = aligned16(env_id) && (packed || (aligned16(role_id) && aligned16(turn_id))) &&
+                     aligned16(rewards) && aligned16(adv) && (group_of_cand == nullptr || aligned16(group_of_cand));
     // one resident wave of blocks; each walks its tiles with a grid stride
     int dev = 0, n_sm = 148, per_sm = 0;
     ATGRPO_CUDA_OK(cudaGetDevice(&dev));
     if (cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n_sm <= 0) n_sm = 148;
-    const cudaError_t oe = vec
-        ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_run_advantages<true>, kThreads, 0)
-        : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_run_advantages<false>, kThreads, 0);
-    if (oe != cudaSuccess || per_sm <= 0) per_sm = 4;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_run_advantages<true, false>, kThreads, 0) !=
+            cudaSuccess || per_sm <= 0)
+      per_sm = 4;
     const int grid = n_tiles < per_sm * n_sm ? n_tiles : per_sm * n_sm;
-    if (vec) k_run_advantages<true><<<grid, kThreads, 0, st>>>(a);
-    else k_run_advantages<false><<<grid, kThreads, 0, st>>>(a);
+    if (packed) {
+      if (vec) k_run_advantages<true, true><<<grid, kThreads, 0, st>>>(a);
+      else k_run_advantages<false, true><<<grid, kThreads, 0, st>>>(a);
+    } else {
+      if (vec) k_run_advantages<true, false><<<grid, kThreads, 0, st>>>(a);
+      else k_run_advantages<false, false><<<grid, kThreads, 0, st>>>(a);
+    }
     return launch_ok();
   }
   if (n > 0 && group_offsets == nullptr && group_perm == nullptr) {
@@ -1025,7 +1039,7 @@ int group_adv_launch(const float* rewards, const int32_t* env_id, const int32_t*
     t.sqhi = reinterpret_cast<unsigned long long*>(tb + (size_t)G * 32);
     t.best = best;
     ATGRPO_CUDA_OK(cudaMemsetAsync(tb, 0, (size_t)G * 40, st));
-    const bool v1 = aligned16(env_id) && aligned16(role_id) && aligned16(turn_id) &&
+    const bool v1 = aligned16(env_id) && (packed || (aligned16(role_id) && aligned16(turn_id))) &&
                     aligned16(rewards) && aligned16(hgid);
     const bool v2 = aligned16(rewards) && aligned16(hgid);
     const bool v3 = v2 && aligned16(adv);
@@ -1033,12 +1047,17 @@ int group_adv_launch(const float* rewards, const int32_t* env_id, const int32_t*
       int64_t b = ((v ? (n + 3) / 4 : n) + kThreads - 1) / kThreads;
       return (int)(b > 148 * 16 ? 148 * 16 : b);
     };
-    if (v1)
-      k_hash_minmax<true><<<grid_of(true), kThreads, 0, st>>>(env_id, role_id, turn_id, rewards, n, n_env,
-                                                              n_role, n_turn, t, hgid, adv, device_status);
-    else
-      k_hash_minmax<false><<<grid_of(false), kThreads, 0, st>>>(env_id, role_id, turn_id, rewards, n, n_env,
-                                                                n_role, n_turn, t, hgid, adv, device_status);
+#define ATGRPO_MINMAX(V, P)                                                                                 \
+  k_hash_minmax<V, P><<<grid_of(V), kThreads, 0, st>>>(env_id, role_id, turn_id, rewards, n, n_env, n_role, \
+                                                       n_turn, t, hgid, adv, device_status)
+    if (packed) {
+      if (v1) ATGRPO_MINMAX(true, true);
+      else ATGRPO_MINMAX(false, true);
+    } else {
+      if (v1) ATGRPO_MINMAX(true, false);
+      else ATGRPO_MINMAX(false, false);
+    }
+#undef ATGRPO_MINMAX
     if (v2) k_hash_moments<true><<<grid_of(true), kThreads, 0, st>>>(hgid, rewards, n, t);
     else k_hash_moments<false><<<grid_of(false), kThreads, 0, st>>>(hgid, rewards, n, t);
     k_hash_finalize<<<(int)((G + kThreads - 1) / kThreads), kThreads, 0, st>>>(t, (int)G, prm.std_eps, prm.ddof,
@@ -1055,16 +1074,21 @@ int group_adv_launch(const float* rewards, const int32_t* env_id, const int32_t*
     if (group_std) ATGRPO_CUDA_OK(cudaMemsetAsync(group_std, 0, (size_t)G * sizeof(float), st));
     return ATGRPO_OK;
   }
-  const bool vec = aligned16(env_id) && aligned16(role_id) && aligned16(turn_id) &&
+  const bool vec = aligned16(env_id) && (packed || (aligned16(role_id) && aligned16(turn_id))) &&
                    aligned16(gid) && aligned16(slot);
   const int work = vec ? (n + 3) / 4 : n;
   const int grid_c = (int)((work + kThreads - 1) / kThreads);
-  if (vec)
-    k_key_count<true><<<grid_c, kThreads, 0, st>>>(env_id, role_id, turn_id, n, n_env, n_role,
-                                                   n_turn, count, slot, gid, adv, device_status);
-  else
-    k_key_count<false><<<grid_c, kThreads, 0, st>>>(env_id, role_id, turn_id, n, n_env, n_role,
-                                                    n_turn, count, slot, gid, adv, device_status);
+#define ATGRPO_KEYCOUNT(V, P)                                                                          \
+  k_key_count<V, P><<<grid_c, kThreads, 0, st>>>(env_id, role_id, turn_id, n, n_env, n_role, n_turn, count, \
+                                                 slot, gid, adv, device_status)
+  if (packed) {
+    if (vec) ATGRPO_KEYCOUNT(true, true);
+    else ATGRPO_KEYCOUNT(false, true);
+  } else {
+    if (vec) ATGRPO_KEYCOUNT(true, false);
+    else ATGRPO_KEYCOUNT(false, false);
+  }
+#undef ATGRPO_KEYCOUNT
   const int nb = (int)((G + kScanBlock - 1) / kScanBlock);
   k_block_sums<<<nb, kThreads, 0, st>>>(count, (int)G, block_sum);
   k_scan_offsets<<<nb, kThreads, 0, st>>>(count, (int)G, block_sum, offsets);

@@ -39,7 +39,7 @@ int group_adv_launch(const float* rewards, const int32_t* env_id, const int32_t*
                      int32_t n_turn, const atgrpo_params& prm, float* adv, int32_t* group_of_cand,
                      int32_t* group_offsets, int32_t* group_perm, float* group_mean,
                      float* group_std, int32_t* device_status, void* workspace, cudaStream_t st,
-                     const GroupExtras* extras = nullptr);
+                     const GroupExtras* extras = nullptr, bool packed = false);
 
 // Padded 128-row tile schedule the GEMM kernels read.
 struct Schedule {                       // lives in device memory

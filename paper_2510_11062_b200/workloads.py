@@ -168,6 +168,7 @@ def make_stress(n_env: int = 16384, n_role: int = 4, n_turn: int = 4, k_max: int
     logp = (torch.rand(n_tokens, generator=g, dtype=torch.float32) * 11.9 - 12.0)
     old_logp = logp + torch.randn(n_tokens, generator=g, dtype=torch.float32) * 0.05
     return dict(rewards=rewards, env_id=env_id, role_id=role_id, turn_id=turn_id,
+                group_id=slot.to(torch.int32),       # the slot each candidate was drawn for, as one dense id
                 n_env=n_env, n_role=n_role, n_turn=n_turn, R=R, G=G,
                 resp_of_token=resp_of_token.to(torch.int32), logp=logp, old_logp=old_logp,
                 T=n_tokens)

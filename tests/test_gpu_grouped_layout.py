@@ -122,28 +122,50 @@ def test_broken_promise_is_flagged():
 
 
 def test_full_size_stress_in_rollout_order():
-    # 262144 slots, 2.23 M candidates: the one-pass result against the general pipeline's (itself checked
-    # against the oracle elsewhere) on every candidate, and against the oracle on sampled groups
+    # 262144 slots, 2.23 M candidates in the launch configuration the benchmark times: every
+    # candidate, group id, group mean and std against the fp64 oracle
     s = WL.make_stress(shuffle=False)
-    R, G = s["R"], s["G"]
     args = (s["rewards"], s["env_id"], s["role_id"], s["turn_id"], s["n_env"], s["n_role"], s["n_turn"])
+    ref = U.oracle_group_advantages(*args)
     fast = U.gpu_group_advantages(*args, A.Params(candidates_grouped=1), bucketing=False)
-    slow = U.gpu_group_advantages(*args, A.Params(), bucketing=False)
-    assert fast["status"] == 0 and slow["status"] == 0
-    assert torch.equal(fast["group_of_cand"], slow["group_of_cand"])
-    a, b = fast["adv"].double(), slow["adv"].double()
-    assert ((a - b).abs() <= 1e-5 * b.abs().clamp(min=1.0)).all()
-    assert ((b == 0) == (a == 0)).all()
-    key = fast["group_of_cand"].numpy().astype(np.int64)
-    rng = np.random.default_rng(0)
-    rew = s["rewards"].numpy().astype(np.float64)
-    starts = np.flatnonzero(np.r_[True, key[1:] != key[:-1]])
-    for i in rng.choice(len(starts), 200, replace=False):
-        lo = starts[i]
-        hi = starts[i + 1] if i + 1 < len(starts) else R
-        r = rew[lo:hi]
-        mu, sd = r.mean(), r.std()
-        want = (r - mu) / (sd + 1e-6) if hi - lo > 1 else np.zeros(1)
-        got = fast["adv"].numpy()[lo:hi].astype(np.float64)
-        assert (np.abs(got - want) <= 1e-5 * np.maximum(1.0, np.abs(want))).all()
-        assert abs(fast["group_mean"][key[lo]].item() - mu) <= 1e-6
+    U.check_group_advantages(fast, ref)
+    assert (ref["adv"] == 0).sum() > 0.01 * s["G"]
+    again = U.gpu_group_advantages(*args, A.Params(candidates_grouped=1), bucketing=False)
+    assert torch.equal(fast["adv"], again["adv"])                  # bit-reproducible
+
+
+def _packed(s, prm, bucketing=False, device_slice=None):
+    dev = U.DEV
+    R, G = s["R"], s["G"]
+    out = dict(adv=torch.full((R,), 7.0, device=dev), group_mean=torch.full((G,), 7.0, device=dev),
+               group_std=torch.full((G,), 7.0, device=dev))
+    if bucketing:
+        out.update(group_offsets=torch.full((G + 1,), -5, dtype=torch.int32, device=dev),
+                   group_perm=torch.full((R,), -5, dtype=torch.int32, device=dev))
+    st = A.new_status(dev)
+    ws = A.workspace(A.atgrpo_group_advantages_workspace_bytes(R, G), dev)
+    A.atgrpo_group_advantages_packed(s["rewards"].to(dev), s["group_id"].to(dev), G, prm, device_status=st,
+                                     workspace=ws, **out)
+    torch.cuda.synchronize()
+    res = {k: v.cpu() for k, v in out.items()}
+    res["status"] = int(st.item())
+    return res
+
+
+@pytest.mark.parametrize("shuffle,grouped,bucketing", [(False, 1, False), (True, 0, False), (True, 0, True)])
+def test_packed_group_ids_take_every_pipeline(shuffle, grouped, bucketing):
+    # one dense group id per candidate instead of the three id arrays: the streaming pass on
+    # adjacent groups, the sort-free pipeline and the counting sort, each against the oracle
+    s = WL.make_stress(n_env=519, n_role=4, n_turn=4, n_tokens=10, seed=6, shuffle=shuffle)
+    ref = U.oracle_group_advantages(s["rewards"], s["env_id"], s["role_id"], s["turn_id"], 519, 4, 4)
+    assert np.array_equal(ref["group_of_cand"], s["group_id"].numpy())          # the generator's slot IS the key
+    got = _packed(s, A.Params(candidates_grouped=grouped), bucketing=bucketing)
+    U.check_group_advantages(got, ref)
+
+
+def test_packed_group_id_out_of_range_is_flagged():
+    s = WL.make_stress(n_env=40, n_role=2, n_turn=2, n_tokens=10, seed=7, shuffle=False)
+    s["group_id"] = s["group_id"].clone()
+    s["group_id"][5] = s["G"] + 3
+    got = _packed(s, A.Params(candidates_grouped=1))
+    assert got["status"] in (A.ERR_BAD_INDEX, A.ERR_LAYOUT) and got["adv"][5] == 0
