@@ -428,7 +428,7 @@ def run_ours(args):
     executed_flops = pass_flops * (1.0 + 3.0 * r.routed_rows / max(r.T, 1))
     exec_tf = tf(executed_flops, lm_s)
     traffic = captured_traffic(spec.name) if world == 1 else None
-    n_bwd_chunks = r.A.atgrpo_policy_loss_bwd_chunks(r.T, r.M, spec.V)[0]
+    n_bwd_chunks = r.A.atgrpo_policy_loss_bwd_chunks(r.T, spec.d, spec.V, r.M)[0]
     dw_elem, dh_elem = 4.0, 2.0
     fwd_bytes = 2.0 * spec.d * (spec.V * spec.n_heads + r.T)                        # W and H once
     bwd_bytes = (2.0 * spec.d * (2 * spec.V * spec.n_heads + 3 * r.routed_rows)     # W for logits and dH; H for logits, dW + gather

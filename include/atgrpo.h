@@ -298,14 +298,15 @@ int atgrpo_policy_loss_bwd(
  * is still being computed.
  *
  * atgrpo_policy_loss_bwd_chunks: the backward call walks the vocabulary in *n_chunks pieces of
- * *rows_per_chunk rows (the last one shorter); a function of (T, M, V) only.
+ * *rows_per_chunk rows (the last one shorter); a function of (T, d, V, M) only.
  * atgrpo_policy_loss_bwd_notify: as atgrpo_policy_loss_bwd; in addition chunk_events is a HOST
  * array of n_events CUDA events (cudaEvent_t, created by the caller; n_events must equal
  * n_chunks), and event c is recorded on `stream` as soon as the rows
  * [c*rows_per_chunk, min(V, (c+1)*rows_per_chunk)) of every dW_m are final.  dH is final when the
  * call's last kernel has run, as usual.  With T = 0 all events are recorded after the zero fill.
  * ------------------------------------------------------------------------------------------ */
-int atgrpo_policy_loss_bwd_chunks(int64_t T, int32_t M, int32_t V, int32_t* n_chunks, int32_t* rows_per_chunk);
+int atgrpo_policy_loss_bwd_chunks(int64_t T, int32_t d, int32_t V, int32_t M, int32_t* n_chunks,
+                                  int32_t* rows_per_chunk);
 
 int atgrpo_policy_loss_bwd_notify(
     const void* H, int64_t ldH, const void* const* W /* host array */, int32_t M,

@@ -138,7 +138,7 @@ def lib() -> ctypes.CDLL:
                                              i64, vp, vp, vp, vp, i64, i32, i32, pp, vp,
                                              ctypes.POINTER(vp), vp, vp, sz, vp]
         L.atgrpo_policy_loss_bwd_chunks.restype = ctypes.c_int
-        L.atgrpo_policy_loss_bwd_chunks.argtypes = [i64, i32, i32, ctypes.POINTER(i32), ctypes.POINTER(i32)]
+        L.atgrpo_policy_loss_bwd_chunks.argtypes = [i64, i32, i32, i32, ctypes.POINTER(i32), ctypes.POINTER(i32)]
         L.atgrpo_policy_loss_bwd_notify.restype = ctypes.c_int
         L.atgrpo_policy_loss_bwd_notify.argtypes = [vp, i64, ctypes.POINTER(vp), i32, vp, vp, vp, i32, vp, vp,
                                                     i64, vp, vp, vp, vp, i64, i32, i32, pp, vp,
@@ -308,10 +308,10 @@ def atgrpo_policy_loss_fwd(H, W, target, role_of_token, head_of_role, resp_of_to
     _check(rc, "atgrpo_policy_loss_fwd")
 
 
-def atgrpo_policy_loss_bwd_chunks(T: int, M: int, V: int):
+def atgrpo_policy_loss_bwd_chunks(T: int, d: int, V: int, M: int):
     """(n_chunks, rows_per_chunk) of the vocabulary walk of one backward call; see include/atgrpo.h."""
     n, rows = ctypes.c_int32(0), ctypes.c_int32(0)
-    _check(lib().atgrpo_policy_loss_bwd_chunks(T, M, V, ctypes.byref(n), ctypes.byref(rows)),
+    _check(lib().atgrpo_policy_loss_bwd_chunks(T, d, V, M, ctypes.byref(n), ctypes.byref(rows)),
            "atgrpo_policy_loss_bwd_chunks")
     return n.value, rows.value
 

@@ -195,7 +195,7 @@ int32_t atgrpo_policy_loss_launch_count(int64_t T, int32_t d, int32_t V, int32_t
   if (!is_bwd) return route + (M > 1 ? 1 : 0) + 3;   // (+ row gather) + GEMM sweep, logsumexp combine, Eq. 2 reduction
   // routing for the counts, coef, routing of the gradient-carrying tokens, row gather,
   // one GEMM launch per vocabulary chunk plus one, dH cast
-  return route + 1 + 3 + 1 + lm_head_bwd_chunks(padded_rows(T, M), V) + 1 + 1;
+  return route + 1 + 3 + 1 + lm_head_bwd_chunks(padded_rows(T, M), d, V) + 1 + 1;
 }
 
 int atgrpo_policy_loss_fwd(const void* H, int64_t ldH, const void* const* W, int32_t M,
@@ -262,11 +262,12 @@ int atgrpo_policy_loss_bwd(const void* H, int64_t ldH, const void* const* W, int
                               false, device_status, workspace, workspace_bytes, stream);
 }
 
-int atgrpo_policy_loss_bwd_chunks(int64_t T, int32_t M, int32_t V, int32_t* n_chunks, int32_t* rows_per_chunk) {
-  if (T < 0 || M < 1 || V < 1 || n_chunks == nullptr || rows_per_chunk == nullptr) return ATGRPO_ERR_INVALID_ARG;
+int atgrpo_policy_loss_bwd_chunks(int64_t T, int32_t d, int32_t V, int32_t M, int32_t* n_chunks,
+                                  int32_t* rows_per_chunk) {
+  if (T < 0 || d < 1 || M < 1 || V < 1 || n_chunks == nullptr || rows_per_chunk == nullptr) return ATGRPO_ERR_INVALID_ARG;
   const int64_t T_pad = padded_rows(T, M);
-  *n_chunks = lm_head_bwd_chunks(T_pad, V);
-  *rows_per_chunk = lm_head_bwd_chunk_rows(T_pad, V);
+  *n_chunks = lm_head_bwd_chunks(T_pad, d, V);
+  *rows_per_chunk = lm_head_bwd_chunk_rows(T_pad, d, V);
   return ATGRPO_OK;
 }
 
@@ -302,7 +303,7 @@ int policy_loss_bwd_impl(const void* H, int64_t ldH, const void* const* W, int32
   if (rc != ATGRPO_OK) return rc;
   if (dW == nullptr) return ATGRPO_ERR_INVALID_ARG;
   if (notify) {
-    if (chunk_events == nullptr || n_events != lm_head_bwd_chunks(padded_rows(T, M), V)) return ATGRPO_ERR_INVALID_ARG;
+    if (chunk_events == nullptr || n_events != lm_head_bwd_chunks(padded_rows(T, M), d, V)) return ATGRPO_ERR_INVALID_ARG;
     for (int c = 0; c < n_events; ++c)
       if (chunk_events[c] == nullptr) return ATGRPO_ERR_INVALID_ARG;
   }

@@ -116,8 +116,8 @@ int lm_head_bwd_launch(const LmHeadProblem& p, const float* lse, const float* co
                        const int32_t* row_of_token, const atgrpo_params& prm, void* dH,
                        void* const* dW, void* workspace, cudaStream_t st,
                        void* const* chunk_events = nullptr);
-int lm_head_bwd_chunk_rows(int64_t T_pad, int32_t V);   // vocabulary rows per chunk
+int lm_head_bwd_chunk_rows(int64_t T_pad, int32_t d, int32_t V);   // vocabulary rows per chunk
 int device_sm_count(int* n_sm, int* cc_major);
-int lm_head_bwd_chunks(int64_t T_pad, int32_t V);   // vocabulary chunks of one backward call (it makes one GEMM launch more)
+int lm_head_bwd_chunks(int64_t T_pad, int32_t d, int32_t V);   // vocabulary chunks of one backward call (it makes one GEMM launch more)
 
 }  // namespace atgrpo

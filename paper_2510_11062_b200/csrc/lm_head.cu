@@ -718,17 +718,26 @@ int row_block_tiles(int64_t n_pt, int d) {
   return (int)gm;
 }
 
-// Width of one dZ chunk buffer (a multiple of 256 columns, each of the two buffers <= 512 MiB).
-// A backward launch mixes the long tiles of one chunk with the short ones of the next, so wave
-// quantisation does not depend on the width; wide chunks mean fewer launches and fewer
-// read-modify-write passes over the dH accumulator, as long as the chunk's rows of W (vc * d * 2
-// bytes, re-read by every wave of dH tiles) still fit in L2: at the Qwen3-1.7B shape 256 MiB and
-// 1 GiB buffers both measured 4-5 % slower than 512 MiB.  The vocabulary is cut into equal chunks.
-int bwd_chunk_width(int64_t T_pad, int V) {
-  const int64_t budget = 512ll << 20;
+// Width of one dZ chunk buffer (a multiple of 256 columns).  A backward launch mixes the long
+// tiles of one chunk with the short ones of the next, so wave quantisation does not depend on the
+// width; wide chunks mean fewer launches and fewer read-modify-write passes over the dH
+// accumulator, as long as the chunk's rows of W (vc * d * 2 bytes, re-read by every wave of dH
+// tiles) still fit in L2: at the Qwen3-1.7B shape 256 MiB and 1 GiB buffers both measured 4-5 %
+// slower than 512 MiB (vc = 16384 there, 64 MiB of W).  So: each buffer gets 512 MiB, or for
+// batches whose 512 MiB would be narrower than that, as many columns as keep the chunk's rows of
+// W within 64 MiB (at most 16384), up to 3 GiB per buffer (a long-response micro-batch of 78 K
+// tokens then walks the vocabulary in 10 chunks instead of 46).  The vocabulary is cut into
+// equal chunks.
+int bwd_chunk_width(int64_t T_pad, int d, int V) {
+  const int64_t budget = 512ll << 20, budget_max = 3072ll << 20, w_bytes = 64ll << 20;
   if (T_pad < kPairRows) T_pad = kPairRows;            // T = 0: keep the arithmetic below defined
   const int64_t vmax = (int64_t)(V + BN - 1) / BN * BN;
   int64_t cap = budget / (T_pad * 2) / BN * BN;
+  int64_t wide = w_bytes / ((int64_t)(d > 0 ? d : 1) * 2) / BN * BN;
+  const int64_t wide_fit = budget_max / (T_pad * 2) / BN * BN;
+  if (wide > 16384) wide = 16384;
+  if (wide > wide_fit) wide = wide_fit;
+  if (cap < wide) cap = wide;
   if (cap < BN) cap = BN;
   if (cap > vmax) cap = vmax;
   const int64_t n_chunks = (V + cap - 1) / cap;
@@ -754,7 +763,7 @@ FwdPlan fwd_plan(int64_t T_pad, int V, int n_sm) {
 struct BwdPlan { size_t dz[2], dh_acc, total; int vc; };
 BwdPlan bwd_plan(int64_t T_pad, int d, int V, bool dH_direct) {
   BwdPlan p;
-  p.vc = bwd_chunk_width(T_pad, V);
+  p.vc = bwd_chunk_width(T_pad, d, V);
   Carver c(nullptr);
   for (int i = 0; i < 2; ++i) {
     p.dz[i] = c.off;
@@ -813,12 +822,12 @@ int device_sm_count(int* n_sm, int* cc_major) {
   return ATGRPO_OK;
 }
 
-int lm_head_bwd_chunks(int64_t T_pad, int32_t V) {
-  const int vc = bwd_chunk_width(T_pad, V);
+int lm_head_bwd_chunks(int64_t T_pad, int32_t d, int32_t V) {
+  const int vc = bwd_chunk_width(T_pad, d, V);
   return (V + vc - 1) / vc;
 }
 
-int lm_head_bwd_chunk_rows(int64_t T_pad, int32_t V) { return bwd_chunk_width(T_pad, V); }
+int lm_head_bwd_chunk_rows(int64_t T_pad, int32_t d, int32_t V) { return bwd_chunk_width(T_pad, d, V); }
 
 size_t lm_head_fwd_workspace_bytes(int64_t T_pad, int32_t d, int32_t V, int32_t n_sm) {
   (void)d;

@@ -79,7 +79,7 @@ def backward_overlapped(A, bwd_kwargs: dict, comm_stream, group=None):
     arguments of A.atgrpo_policy_loss_bwd (H, W, ..., dH, dW, device_status, workspace)."""
     H, W, dW = bwd_kwargs["H"], bwd_kwargs["W"], bwd_kwargs["dW"]
     V = W[0].shape[0]
-    n_chunks, rows = A.atgrpo_policy_loss_bwd_chunks(H.shape[0], len(W), V)
+    n_chunks, rows = A.atgrpo_policy_loss_bwd_chunks(H.shape[0], H.shape[1], V, len(W))
     events = [torch.cuda.Event() for _ in range(n_chunks)]
     A.atgrpo_policy_loss_bwd(**bwd_kwargs, chunk_events=events)
     main = torch.cuda.current_stream()

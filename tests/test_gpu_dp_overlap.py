@@ -38,7 +38,7 @@ def _bwd_kwargs(case, f, dH, dW, status, ws):
 def test_notify_matches_plain_backward_and_overlapped_allreduce():
     b, case, f = _case()
     T, d, V, M = b["T"], SPEC.d, SPEC.V, SPEC.n_heads
-    n_chunks, rows = A.atgrpo_policy_loss_bwd_chunks(T, M, V)
+    n_chunks, rows = A.atgrpo_policy_loss_bwd_chunks(T, d, V, M)
     assert n_chunks >= 2 and rows % 256 == 0 and (n_chunks - 1) * rows < V <= n_chunks * rows
     ranges = DP.chunk_row_ranges(V, n_chunks, rows)
     assert ranges[0][0] == 0 and ranges[-1][1] == V and all(a[1] == b_[0] for a, b_ in zip(ranges, ranges[1:]))
@@ -91,7 +91,7 @@ def test_notify_matches_plain_backward_and_overlapped_allreduce():
 
 def test_notify_with_no_tokens_records_every_event():
     d, V, M = 64, 1000, 1
-    n_chunks, _ = A.atgrpo_policy_loss_bwd_chunks(0, M, V)
+    n_chunks, _ = A.atgrpo_policy_loss_bwd_chunks(0, d, V, M)
     z = lambda dt: torch.zeros(0, dtype=dt, device=U.DEV)
     W = [torch.zeros(V, d, dtype=torch.bfloat16, device=U.DEV)]
     dW = [torch.full((V, d), 3.0, dtype=torch.float32, device=U.DEV)]

@@ -74,7 +74,7 @@ def test_full_size_dense_backward_rows(name, request):
     g = case.bwd(torch.from_numpy(logp).float(), torch.from_numpy(lse).float())
     assert g["status"] == 0
     c = O.dloss_dlogp(logp, old, adv, b["resp_of_token"], head, M, None if gl is None else gl.numpy())
-    n_chunks, rows_per_chunk = A.atgrpo_policy_loss_bwd_chunks(T, M, V)
+    n_chunks, rows_per_chunk = A.atgrpo_policy_loss_bwd_chunks(T, spec.d, V, M)
     assert n_chunks >= 2                                           # both dZ buffers alternate
     dH = g["dH"].numpy()
     for m in range(M):
