@@ -49,6 +49,8 @@ SPECS = {
     "multi3": RolloutSpec("multi3", 24, 3, 2, 4, (96, 32, 32), (128, 80, 80), 2048, 151936, 3, 1237),
     # single policy, Qwen3-8B-shaped head
     "qwen3_8b": RolloutSpec("qwen3_8b", 32, 2, 4, 4, (16, 16), (48, 48), 4096, 151936, 1, 1238),
+    # the same head on a quarter of the batch (~8K tokens): dense parity at d = 4096 within the oracle's reach
+    "qwen3_8b_quarter": RolloutSpec("qwen3_8b_quarter", 8, 2, 4, 4, (16, 16), (48, 48), 4096, 151936, 1, 1244),
     # long responses (the paper allows up to 4096 generated tokens): few responses, ~80K tokens
     "long_resp": RolloutSpec("long_resp", 4, 2, 2, 4, (512, 512), (2048, 2048), 2048, 151936, 1, 1243),
     # mid-size shapes for dense element-by-element comparison (several tiles + ragged tails)
