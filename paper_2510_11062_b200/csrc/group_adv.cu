@@ -769,7 +769,44 @@ __global__ void __launch_bounds__(kThreads, 4) k_run_advantages(RunArgs a) {
       // fetched ONCE into registers; everything after that is register arithmetic.
       float* p = r_s + i;
       double mu, sd = 0.0;
+      bool done = false;
       if (K <= kRunRegK) {
+        // Runs of up to 16 members, the common case: everything in fp32 on SHIFTED values
+        // x = r - c, c = the run's first reward (exact for close values, 2^-24 relative otherwise;
+        // identical rewards give x = 0 throughout, hence exact zeros).  Two passes: the mean of at
+        // most 16 values of the run's own scale, then squared deviations, which cannot cancel.
+        const float c = p[0];
+        float x[kRunRegK];
+#pragma unroll
+        for (int k = 0; k < kRunRegK; ++k) x[k] = k < K ? p[k] - c : 0.f;
+        float sum = 0.f;
+#pragma unroll
+        for (int k = 0; k < kRunRegK; ++k) sum += x[k];      // ascending order; the padding adds exact zeros
+        const float kf = (float)K;
+        const float mean_x = __fdividef(sum, kf);
+        float ss = 0.f;
+#pragma unroll
+        for (int k = 0; k < kRunRegK; ++k) {
+          const float dlt = k < K ? x[k] - mean_x : 0.f;
+          x[k] = dlt;
+          ss = fmaf(dlt, dlt, ss);
+        }
+        if (ss < 1e30f) {                             // otherwise (squares beyond fp32) the fp64 route below
+          const int dof = K - a.ddof;
+          const float var = dof > 0 ? __fdividef(ss, (float)dof) : 0.f;
+          const float sdf = sqrtf(var);               // an underflow to 0 is harmless: eps dominates there
+          const float invf = K > 1 ? 1.0f / (sdf + a.std_eps) : 0.f;
+#pragma unroll
+          for (int k = 0; k < kRunRegK; ++k)
+            if (k < K) p[k] = x[k] * invf;
+          mu = (double)c + (double)mean_x;
+          sd = (double)sdf;
+          done = true;
+        }
+      }
+      if (done) {
+        // finished above
+      } else if (K <= kRunRegK) {
         double v[kRunRegK];
 #pragma unroll
         for (int k = 0; k < kRunRegK; ++k) v[k] = k < K ? (double)p[k] : 0.0;

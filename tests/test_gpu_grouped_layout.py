@@ -93,6 +93,21 @@ def test_single_candidate_and_constant_long_run():
     assert (gpu["adv"] == 0).all()
 
 
+def test_nearly_equal_and_wide_range_rewards_in_adjacent_groups():
+    # groups whose rewards differ in the last bit, negative rewards, magnitudes from 1e-20 to 1e20 next
+    # to one another: every run is shifted by its own first reward, and squares beyond fp32 take fp64
+    one = torch.tensor(1.0)
+    up = torch.nextafter(one, torch.tensor(2.0))
+    rewards = torch.tensor([1.0, up, 1.0, up, -3.0, -3.0, -3.0, -2.9999998, 1e-20, 3e-20, 2e-20, 5e20, -5e20, 0.0,
+                            7.5, 2e19, -2e19, 1e19, 4.0, 4.0, 4.0], dtype=torch.float32)
+    slot = torch.tensor([0, 0, 0, 0, 1, 1, 1, 1, 2, 2, 2, 3, 3, 3, 4, 5, 5, 5, 6, 6, 6])
+    env = slot.to(torch.int32)
+    zero = torch.zeros_like(env)
+    for ddof in (0, 1):
+        gpu, ref = _check(rewards, env, zero, zero, 7, 1, 1, ddof=ddof)
+    assert (gpu["adv"][-3:] == 0).all() and gpu["adv"][14] == 0
+
+
 def test_bad_ids_inside_and_between_runs():
     rewards = torch.tensor([0.1, 0.9, 0.5, 0.3, 0.2, 0.8, 0.4], dtype=torch.float32)
     env = torch.tensor([0, 0, 5, 0, 1, -1, 1], dtype=torch.int32)      # a bad id splits group 0 and group 1
