@@ -57,3 +57,14 @@ def test_memory_bound_line():
     assert r["roofline"]["bound"] == "hbm" and r["unit"] == "GB/s" and r["value"] > 0
     assert r["config"]["candidate_order"].startswith("rollout order")
     assert r["loss_reduction"]["gbs"] > 0
+
+
+def test_update_step_line():
+    # one whole policy update at the paper's batch scale: two long-response micro-batches accumulated
+    # into one dW, gradient norm, clipped AdamW
+    r = _run("--workload", "batch128", "--steps", "1", "--warmup", "3")
+    assert r["config"]["workload"] == "batch128" and r["config"]["responses"] == 128
+    assert r["config"]["tokens"] > 100_000 and len(r["config"]["micro_batches"]) == 2
+    assert r["value"] > 0 and r["phases_ms"]["gradient"] > r["phases_ms"]["optimizer"] > 0
+    rf = r["roofline"]
+    assert rf["bound"] == "tensor" and 0 < rf["frac"] <= rf["executed_frac"] and rf["optimizer_gbs"] > 0
