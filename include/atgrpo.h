@@ -114,9 +114,10 @@ const char* atgrpo_status_string(int status);
  * paper's hash(e,i,t); G = n_env*n_role*n_turn slots, empty slots allowed, G < 2^31.
  * For each non-empty group of K members: mu = mean, sigma = std (params->ddof), and
  *   adv[c] = (rewards[c] - mu) / (sigma + params->std_eps);   K = 1 gives adv = 0.
- * The result is bit-reproducible and a group of identical rewards yields exact zeros (fp64 sums
- * in ascending candidate order when bucketing outputs are requested or candidates_grouped is set;
- * exact integer accumulation of rewards quantised to 2^-25 of the group's range otherwise).
+ * The result is bit-reproducible and a group of identical rewards yields exact zeros (sums in
+ * ascending candidate order when bucketing outputs are requested or candidates_grouped is set --
+ * fp64, or, for adjacent groups of up to 16 members, fp32 on rewards shifted by the group's first
+ * one; exact integer accumulation of rewards quantised to 2^-25 of the group's range otherwise).
  *
  * Outputs: adv[n_cand] (required).  Optional (NULL to skip): group_of_cand[n_cand] = g;
  * group_offsets[G+1] and group_perm[n_cand], the stable bucketing (slot s owns

@@ -26,7 +26,8 @@
 //     group are adjacent, which is the order Algorithm 1 appends them in (the K samples of one
 //     (environment, agent, turn) together).  One streaming pass: a block stages a tile of
 //     candidates in shared memory and marks where runs of equal keys begin; one thread per run
-//     fetches the run's members once into registers, sums them in fp64 in ascending order and
+//     fetches the run's members once into registers, sums them in ascending order (fp32 on values
+//     shifted by the run's first reward for runs of up to 16 members, fp64 otherwise) and
 //     writes the advantages back over the staged rewards, and the tile leaves with coalesced
 //     stores; longer runs loop over shared memory, are summed by a warp, or (beyond the staged
 //     window) by the whole block.  One integer atomic per RUN checks the promise (a key that
@@ -750,7 +751,7 @@ __global__ void __launch_bounds__(kThreads, 4) k_run_advantages(RunArgs a) {
       s_lead = (bnd_s[0] & 1u) ? 0 : next_boundary(bnd_s, 1);
       s_cross = own < cnt ? next_boundary(bnd_s, own) : own;
     }
-    // ---- one thread per run (the list is dense, so every lane works): fp64 sums in ascending order
+    // ---- one thread per run (the list is dense, so every lane works): sums in ascending order
     const int n_heads = s_heads;
     for (int h = threadIdx.x; h < n_heads; h += kThreads) {
       const int i = head_s[h];
