@@ -199,7 +199,9 @@ class Runner:
         self.W = W if W is not None else [w.to(device) for w in batch["W"]]
         self.head_of_role = batch["head_of_role"].to(device) if self.M > 1 else None
         self.role_of_token = self.d["role_of_token"] if self.M > 1 else None
-        self.prm = A.Params(accumulate_dW=1 if accumulate else 0)
+        # the rollout generator appends the K candidates of a group together (Algorithm 1's order), so
+        # the advantages take the one-pass path; the flag means nothing to the loss calls
+        self.prm = A.Params(accumulate_dW=1 if accumulate else 0, candidates_grouped=1)
         G = spec.n_env * spec.n_role * spec.n_turn
         T, V, dm, M = self.T, spec.V, spec.d, self.M
         self.adv = torch.zeros(self.R, dtype=f32, device=device)
@@ -214,7 +216,7 @@ class Runner:
         self.ws_adv = A.workspace(A.atgrpo_group_advantages_workspace_bytes(self.R, G), device)
         self.ws_fwd = A.workspace(A.atgrpo_policy_loss_workspace_bytes(T, dm, V, M, False), device)
         self.ws_bwd = A.workspace(A.atgrpo_policy_loss_workspace_bytes(T, dm, V, M, True), device)
-        self.launches = 4 + A.atgrpo_policy_loss_launch_count(T, dm, V, M, False) + \
+        self.launches = 1 + A.atgrpo_policy_loss_launch_count(T, dm, V, M, False) + \
             A.atgrpo_policy_loss_launch_count(T, dm, V, M, True)
         self.host_loss = torch.zeros(M, dtype=f32).pin_memory()
         self.h2d_bytes = sum(self.host[k].numel() * self.host[k].element_size() for k in self.host
