@@ -127,7 +127,9 @@ def run_reference(args):
     line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=1, steps=args.steps, warmup=args.warmup,
                 ms_per_step=1e3 * total / len(times), higher_is_better=True, scaling="weak", vs_baseline=None,
                 dtype="f64", data="synthetic", impl="reference",
-                config=dict(workload=spec.name, d=spec.d, V=spec.V, tokens=batch["T"], heads=spec.n_heads),
+                config=dict(workload=spec.name, d=spec.d, V=spec.V, heads=spec.n_heads, tokens_per_gpu=batch["T"],
+                            responses_per_gpu=batch["R"], parallelism="dp1",
+                            sample="each step: the first %d tokens of the workload's batch" % n),
                 cpu_baseline=dict(value=value, unit=UNIT, cores=blas_threads(), kind="oracle", sample=sample),
                 e2e=dict(value=value, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0))
     print(json.dumps(line), flush=True)
