@@ -36,9 +36,9 @@ def test_rollout_batches_are_grouped(name):
 
 @pytest.mark.parametrize("ddof", [0, 1])
 def test_stress_shape_in_rollout_order(ddof):
-    # K ~ U{1..16} with K = 1 and all-equal groups; several tiles of 2048 candidates and a ragged tail
+    # K ~ U{1..16} with K = 1 and all-equal groups; several tiles of 4096 candidates and a ragged tail
     s = WL.make_stress(n_env=519, n_role=4, n_turn=4, n_tokens=10, seed=5, shuffle=False)
-    assert s["R"] > 4 * 2048 and s["R"] % 2048 != 0
+    assert s["R"] > 4 * 4096 and s["R"] % 4096 != 0
     _check(s["rewards"], s["env_id"], s["role_id"], s["turn_id"], 519, 4, 4, ddof=ddof)
 
 
@@ -53,12 +53,12 @@ def test_groups_in_random_order_with_empty_slots():
     _check(rewards, e, r, t, 70, 5, 2)
 
 
-@pytest.mark.parametrize("shift", [0, 1, 1791, 2047])
+@pytest.mark.parametrize("shift", [0, 1, 1791, 2047, 3839, 4095])
 def test_runs_that_cross_tiles_and_outgrow_the_window(shift):
-    # runs of 6000 (spans whole tiles), 2304 and 257 (just beyond the look-ahead), 256, 255 members,
-    # placed so that they start at different offsets inside a 2048-candidate tile
+    # runs of 9000 (spans whole tiles), 4352 and 257 (just beyond the look-ahead), 256, 255 members,
+    # placed so that they start at different offsets inside a 4096-candidate tile (4096 + 256 staged)
     g = torch.Generator().manual_seed(3)
-    sizes = [shift, 6000, 3, 2304, 1, 257, 256, 255, 2040, 700, 65, 33] + [3] * 50 + [1] * 7 + [0] * 5
+    sizes = [shift, 9000, 3, 4352, 1, 257, 256, 255, 4090, 2304, 700, 65, 33] + [3] * 50 + [1] * 7 + [0] * 5
     slot = torch.repeat_interleave(torch.arange(len(sizes)), torch.tensor(sizes))
     rewards = WL.draw_rewards(g, slot.numel())
     e, r, t = _ids(slot, 3, 2)
@@ -69,7 +69,7 @@ def test_runs_that_cross_tiles_and_outgrow_the_window(shift):
 def test_unaligned_pointers_take_the_scalar_staging_path():
     s = WL.make_stress(n_env=300, n_role=2, n_turn=2, n_tokens=10, seed=8, shuffle=False)
     R = s["R"]
-    assert R > 2 * 2048
+    assert R > 2 * 4096
     pad = lambda t: torch.cat([torch.zeros(1, dtype=t.dtype), t]).to(U.DEV)[1:]   # 4-byte aligned only
     rewards, e, r, t = pad(s["rewards"]), pad(s["env_id"]), pad(s["role_id"]), pad(s["turn_id"])
     adv = torch.empty(R + 1, dtype=torch.float32, device=U.DEV)[1:]
@@ -87,7 +87,7 @@ def test_single_candidate_and_constant_long_run():
     one = torch.zeros(1, dtype=torch.int32)
     gpu, _ = _check(torch.tensor([0.7]), one, one, one, 1, 1, 1)
     assert gpu["adv"].tolist() == [0.0]
-    n = 5000                                     # one constant run longer than the staged window
+    n = 9000                                     # one constant run longer than the staged window
     z = torch.zeros(n, dtype=torch.int32)
     gpu, _ = _check(torch.full((n,), 0.3), z, z, z, 1, 1, 1)
     assert (gpu["adv"] == 0).all()
