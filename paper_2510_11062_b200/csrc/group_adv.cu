@@ -908,7 +908,7 @@ __global__ void __launch_bounds__(kThreads, 4) k_run_advantages(RunArgs a) {
       for (int k = lane; k < K; k += 32) r_s[i + k] = (float)(((double)r_s[i + k] - mu) * inv);
       if (lane == 0) run_publish(a, g, atomicAdd(&a.seen[g], 1), mu, sd);
     }
-    __syncthreads();
+    if (n_big > 0) __syncthreads();                   // n_big is the same in every thread: no barrier for the usual tile
 
     // ---- the tile leaves with coalesced stores
     const int lh = s_long;
