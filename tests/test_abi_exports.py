@@ -80,3 +80,24 @@ def test_binding_refuses_cpu_tensors(lib):
     t = torch.zeros(4)
     with pytest.raises(A.AtgrpoError):
         A.atgrpo_clipped_loss(t, t, t.int(), t, A.Params(), t[:1], workspace=torch.zeros(256, dtype=torch.uint8))
+
+
+def test_parameter_structs_have_the_same_layout_in_c_and_in_the_binding(tmp_path):
+    # compile a tiny C program against include/atgrpo.h and compare sizes and offsets with ctypes
+    import subprocess
+    fields_p = [f[0] for f in A._Params._fields_]
+    fields_a = [f[0] for f in A._AdamWParams._fields_]
+    src = tmp_path / "layout.c"
+    lines = ['#include <stdio.h>', '#include <stddef.h>', '#include "atgrpo.h"', 'int main(void) {',
+             '  printf("%zu\\n", sizeof(atgrpo_params));']
+    lines += ['  printf("%%zu\\n", offsetof(atgrpo_params, %s));' % f for f in fields_p]
+    lines += ['  printf("%zu\\n", sizeof(atgrpo_adamw_params));']
+    lines += ['  printf("%%zu\\n", offsetof(atgrpo_adamw_params, %s));' % f for f in fields_a]
+    lines += ['  return 0;', '}']
+    src.write_text("\n".join(lines))
+    exe = tmp_path / "layout"
+    subprocess.run(["gcc", "-I", os.path.join(ROOT, "include"), str(src), "-o", str(exe)], check=True)
+    got = [int(x) for x in subprocess.run([str(exe)], capture_output=True, text=True, check=True).stdout.split()]
+    want = [ctypes.sizeof(A._Params)] + [getattr(A._Params, f).offset for f in fields_p] + \
+           [ctypes.sizeof(A._AdamWParams)] + [getattr(A._AdamWParams, f).offset for f in fields_a]
+    assert got == want
