@@ -784,9 +784,12 @@ __global__ void __launch_bounds__(kThreads, 4) k_run_advantages(RunArgs a) {
         float x[kRunRegK];
 #pragma unroll
         for (int k = 0; k < kRunRegK; ++k) x[k] = k < K ? p[k] - c : 0.f;
-        float sum = 0.f;
+        float sum = 0.f, amax = 0.f;
 #pragma unroll
-        for (int k = 0; k < kRunRegK; ++k) sum += x[k];      // ascending order; the padding adds exact zeros
+        for (int k = 0; k < kRunRegK; ++k) {
+          sum += x[k];                                // ascending order; the padding adds exact zeros
+          amax = fmaxf(amax, fabsf(x[k]));
+        }
         const float kf = (float)K;
         const float mean_x = __fdividef(sum, kf);
         float ss = 0.f;
@@ -796,11 +799,13 @@ __global__ void __launch_bounds__(kThreads, 4) k_run_advantages(RunArgs a) {
           x[k] = dlt;
           ss = fmaf(dlt, dlt, ss);
         }
-        if (ss < 1e30f) {                             // otherwise (squares beyond fp32) the fp64 route below
+        // fp32 is trusted while the squares sit well inside its normal range (and for identical
+        // rewards, whose deviations are exactly zero); otherwise the fp64 route below
+        if (amax == 0.f || (ss > 1e-25f && ss < 1e30f)) {
           const int dof = K - a.ddof;
           const float var = dof > 0 ? __fdividef(ss, (float)dof) : 0.f;
-          const float sdf = sqrtf(var);               // an underflow to 0 is harmless: eps dominates there
-          const float invf = K > 1 ? 1.0f / (sdf + a.std_eps) : 0.f;
+          const float sdf = sqrtf(var);
+          const float invf = amax != 0.f ? 1.0f / (sdf + a.std_eps) : 0.f;   // identical rewards (K = 1 too): exact zeros
 #pragma unroll
           for (int k = 0; k < kRunRegK; ++k)
             if (k < K) p[k] = x[k] * invf;
@@ -836,25 +841,12 @@ __global__ void __launch_bounds__(kThreads, 4) k_run_advantages(RunArgs a) {
             const double dlt = k < K ? v[k] - mu : 0.0;
             ss = fma(dlt, dlt, ss);
           }
-          // The advantage is wanted to 1e-5: the deviation r - mean is taken in fp64, std and
-          // 1/(std + eps) in fp32 (one MUFU square root and reciprocal instead of two software
-          // fp64 routines per run).  A variance outside the comfortable fp32 range takes the fp64 route.
-          const int dof = K - a.ddof;
-          const double var = dof > 0 ? ss * c_inv_k[dof] : 0.0;
-          if (var < 1e30) {
-            const float sdf = sqrtf((float)var);      // an underflow to 0 is harmless: eps dominates there
-            const float invf = 1.0f / (sdf + a.std_eps);
-            sd = (double)sdf;
+          // only runs whose squares leave the comfortable fp32 range get here: fp64 throughout
+          double inv;
+          run_stats(ss, K, a.ddof, a.std_eps, sd, inv);
 #pragma unroll
-            for (int k = 0; k < kRunRegK; ++k)
-              if (k < K) p[k] = (float)(v[k] - mu) * invf;
-          } else {
-            double inv;
-            run_stats(ss, K, a.ddof, a.std_eps, sd, inv);
-#pragma unroll
-            for (int k = 0; k < kRunRegK; ++k)
-              if (k < K) p[k] = (float)((v[k] - mu) * inv);
-          }
+          for (int k = 0; k < kRunRegK; ++k)
+            if (k < K) p[k] = (float)((v[k] - mu) * inv);
         }
       } else {
         const double first = (double)p[0];

@@ -108,6 +108,23 @@ def test_nearly_equal_and_wide_range_rewards_in_adjacent_groups():
     assert (gpu["adv"][-3:] == 0).all() and gpu["adv"][14] == 0
 
 
+@pytest.mark.parametrize("scale", [1e-18, 1e18])
+def test_rewards_of_extreme_scale_with_an_epsilon_to_match(scale):
+    # rewards around 1e-18 (squared deviations fall into the fp32 denormal range) and around 1e18 (they
+    # overflow fp32), with std_eps scaled alike so that it does not mask the standard deviation
+    s = WL.make_stress(n_env=200, n_role=2, n_turn=2, n_tokens=10, seed=12, shuffle=False)
+    rewards = (s["rewards"] * scale).contiguous()
+    eps = 1e-6 * scale
+    args = (rewards, s["env_id"], s["role_id"], s["turn_id"], 200, 2, 2)
+    ref = U.oracle_group_advantages(*args, eps=eps)
+    gpu = U.gpu_group_advantages(*args, A.Params(std_eps=eps, candidates_grouped=1), bucketing=False)
+    assert gpu["status"] == 0
+    a, r = gpu["adv"].numpy().astype(np.float64), ref["adv"]
+    assert (np.abs(a - r) <= 1e-5 * np.maximum(1.0, np.abs(r))).all()
+    assert (a[r == 0.0] == 0.0).all()
+    np.testing.assert_allclose(gpu["group_std"].numpy(), ref["group_std"], rtol=2e-6)
+
+
 def test_bad_ids_inside_and_between_runs():
     rewards = torch.tensor([0.1, 0.9, 0.5, 0.3, 0.2, 0.8, 0.4], dtype=torch.float32)
     env = torch.tensor([0, 0, 5, 0, 1, -1, 1], dtype=torch.int32)      # a bad id splits group 0 and group 1
