@@ -103,3 +103,31 @@ def test_notify_with_no_tokens_records_every_event():
                              dW, device_status=A.new_status(U.DEV), workspace=ws, chunk_events=events)
     torch.cuda.synchronize()
     assert all(ev.query() for ev in events) and (dW[0] == 0).all()
+
+
+def test_multi_chunk_multi_head_configuration_matches_the_oracle():
+    # the configuration of this file (three heads, a vocabulary walked in several chunks, d = 64) with
+    # old_logp built from the ORACLE's log-probs: forward, loss and the complete dH / dW of every head
+    import numpy as np
+    from oracle import atgrpo_oracle as O
+    b = WL.make_rollout(SPEC)
+    T, d, V, M = b["T"], SPEC.d, SPEC.V, SPEC.n_heads
+    n_chunks, _ = A.atgrpo_policy_loss_bwd_chunks(T, d, V, M)
+    assert n_chunks >= 2
+    lse, logp = U.oracle_logprobs(b, chunk=1024)
+    adv = U.batch_advantages(b)
+    old = U.keep_off_the_kinks(logp, WL.make_old_logp(torch.from_numpy(logp), 17, 0.3))
+    head, offsets, perm = U.oracle_heads(b)
+    gl = torch.tensor([1.0, 0.5, 2.0])
+    case = U.PolicyCase(b, adv, old, grad_loss=gl)
+    out = case.fwd()
+    assert out["status"] == 0
+    assert np.abs(out["lse"].numpy() - lse).max() <= 1e-3 and np.abs(out["logp"].numpy() - logp).max() <= 1e-3
+    rl, _, _ = O.policy_loss(logp, old, adv, b["resp_of_token"], head, M)
+    np.testing.assert_allclose(out["loss"].numpy(), rl, rtol=1e-3)
+    g = case.bwd(torch.from_numpy(logp).float(), torch.from_numpy(lse).float())
+    assert g["status"] == 0
+    dH, dW = O.policy_loss_grads(b["H"], b["W"], b["target"], old, adv, b["resp_of_token"], head, grad_loss=gl.numpy())
+    U.check_rows(g["dH"].numpy(), dH, "dH")
+    for m in range(M):
+        U.check_rows(g["dW"][m].numpy(), dW[m], "dW[%d]" % m)
