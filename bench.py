@@ -184,12 +184,21 @@ class ClockSampler:
 
 
 # ------------------------------------------------------------------------------- GPU leg
+def logits_note(keep, T, V):
+    if not keep:
+        return "recomputed in the backward (no [T, V] buffer)"
+    return "kept: the forward stores [T, V] fp32 in a lent buffer (%.1f GB), the backward reads it" % (
+        T * ((V + 255) // 256 * 256) * 4 / 1e9)
+
+
 class Runner:
     """Device-resident state of one rank: inputs, outputs, workspaces; step() enqueues the path."""
 
-    def __init__(self, batch, device, A, W=None, dW=None, accumulate=False):
+    def __init__(self, batch, device, A, W=None, dW=None, accumulate=False, keep_logits=True, logits=None):
         """W / dW: device tensors shared with other Runners (micro-batches of one update step);
-        accumulate: this Runner's backward adds into dW instead of overwriting it."""
+        accumulate: this Runner's backward adds into dW instead of overwriting it; keep_logits: lend
+        the library a [T, V] fp32 buffer so that the backward reads the logits instead of repeating
+        the contraction (`logits`: such a buffer shared with other Runners, large enough for each)."""
         self.A = A
         self.dev = device
         spec = self.spec = batch["spec"]
@@ -203,9 +212,13 @@ class Runner:
         self.role_of_token = self.d["role_of_token"] if self.M > 1 else None
         # the rollout generator appends the K candidates of a group together (Algorithm 1's order), so
         # the advantages take the one-pass path; the flag means nothing to the loss calls
-        self.prm = A.Params(accumulate_dW=1 if accumulate else 0, candidates_grouped=1)
         G = spec.n_env * spec.n_role * spec.n_turn
         T, V, dm, M = self.T, spec.V, spec.d, self.M
+        self.logits = None
+        if keep_logits:
+            n = A.atgrpo_policy_loss_logits_bytes(T, V) // 4
+            self.logits = logits[:n] if logits is not None else torch.empty(n, dtype=f32, device=device)
+        self.prm = A.Params(accumulate_dW=1 if accumulate else 0, candidates_grouped=1, logits=self.logits)
         self.adv = torch.zeros(self.R, dtype=f32, device=device)
         self.loss = torch.zeros(M, dtype=f32, device=device)
         self.logp = torch.zeros(T, dtype=f32, device=device)
@@ -319,7 +332,7 @@ def run_ours(args):
                             sample=f"first {n} tokens, full vocabulary, fwd+bwd, plus advantages of all "
                                    f"{batch['R']} candidates; {dt:.1f} s")
 
-    r = Runner(batch, dev, A)
+    r = Runner(batch, dev, A, keep_logits=args.logits == "keep")
     r.make_old_logp()
     r.count_routed_rows()
     if world > 1:
@@ -429,13 +442,17 @@ def run_ours(args):
     # recompute, dH, dW) on the rows that carry a gradient (counted on the device, outside the
     # timed region) -- and the two calls on their own.
     algo_tf = tf(3.0 * pass_flops, lm_s)
-    executed_flops = pass_flops * (1.0 + 3.0 * r.routed_rows / max(r.T, 1))
+    bwd_passes = 2.0 if r.logits is not None else 3.0         # dH, dW (+ the logits again unless they were kept)
+    executed_flops = pass_flops * (1.0 + bwd_passes * r.routed_rows / max(r.T, 1))
     exec_tf = tf(executed_flops, lm_s)
     traffic = captured_traffic(spec.name) if world == 1 else None
     n_bwd_chunks = r.A.atgrpo_policy_loss_bwd_chunks(r.T, spec.d, spec.V, r.M)[0]
     dw_elem, dh_elem = 4.0, 2.0
+    kept = r.logits is not None
     fwd_bytes = 2.0 * spec.d * (spec.V * spec.n_heads + r.T)                        # W and H once
-    bwd_bytes = (2.0 * spec.d * (2 * spec.V * spec.n_heads + 3 * r.routed_rows)     # W for logits and dH; H for logits, dW + gather
+    fwd_bytes += 4.0 * r.T * spec.V if kept else 0.0                                # kept logits written once
+    bwd_bytes = ((4.0 * r.routed_rows * spec.V if kept else 2.0 * spec.d * (spec.V * spec.n_heads + r.routed_rows))   # logits read back, or W and H once more
+                 + 2.0 * spec.d * (spec.V * spec.n_heads + 2 * r.routed_rows)       # W for dH; H for dW + gather
                  + 3.0 * 2.0 * r.routed_rows * spec.V                               # dZ written once, read by dH and by dW
                  + dw_elem * spec.V * spec.d * spec.n_heads                         # dW written once
                  + 2.0 * 4.0 * r.routed_rows * spec.d * n_bwd_chunks                # fp32 dH accumulator, once per chunk
@@ -448,6 +465,7 @@ def run_ours(args):
         config=dict(workload=spec.name, d=spec.d, V=spec.V, heads=spec.n_heads, tokens_per_gpu=r.T,
                     responses_per_gpu=r.R, parallelism=f"dp{world}",
                     l2="inputs larger than L2 (W alone is %.0f MB)" % (spec.V * spec.d * 2 / 1e6),
+                    logits=logits_note(r.logits is not None, r.T, spec.V),
                     old_logp="library logp + N(0,0.05) (perf-only input)"),
         gpu_launches=(r.launches) * args.steps,
         phases_ms=dict(advantages=adv_ms, forward=fwd_ms, backward=bwd_ms),
@@ -465,7 +483,8 @@ def run_ours(args):
                       algorithmic_bytes=fwd_bytes + bwd_bytes, algorithmic_bytes_forward=fwd_bytes,
                       algorithmic_bytes_backward=bwd_bytes,
                       executed_tflops=exec_tf, executed_frac=exec_tf / peaks["bf16_sustained"],
-                      executed="forward on %d rows + recompute, dH, dW on the %d rows with a gradient" % (r.T, r.routed_rows),
+                      executed="forward on %d rows + %sdH, dW on the %d rows with a gradient"
+                               % (r.T, "" if r.logits is not None else "recompute, ", r.routed_rows),
                       routed_rows=r.routed_rows,
                       frac_of_nominal_2250=algo_tf / 2250.0, executed_frac_of_nominal_2250=exec_tf / 2250.0,
                       forward_tflops=tf(pass_flops, fwd_ms * 1e-3),
@@ -507,7 +526,13 @@ def run_update_step(args):
     V, dm = base.V, base.d
     W = [batches[0]["W"][0].to(dev)]
     dW = [torch.zeros(V, dm, dtype=torch.float32, device=dev)]
-    runners = [Runner(b, dev, A, W=W, dW=dW, accumulate=(i > 0)) for i, b in enumerate(batches)]
+    keep = args.logits == "keep"
+    shared = None
+    if keep:                                   # one logits buffer, sized for the larger micro-batch, used by each in turn
+        shared = torch.empty(max(A.atgrpo_policy_loss_logits_bytes(b["T"], V) for b in batches) // 4,
+                             dtype=torch.float32, device=dev)
+    runners = [Runner(b, dev, A, W=W, dW=dW, accumulate=(i > 0), keep_logits=keep, logits=shared)
+               for i, b in enumerate(batches)]
     T_all = sum(r.T for r in runners)
     for r in runners:
         r.make_old_logp()
@@ -562,7 +587,7 @@ def run_update_step(args):
     peaks = measured_peaks()
     algo_tf = 6.0 * T_all * V * dm / (grad_ms * 1e-3) / 1e12
     routed = sum(r.routed_rows for r in runners)
-    exec_tf = 2.0 * V * dm * (T_all + 3.0 * routed) / (grad_ms * 1e-3) / 1e12
+    exec_tf = 2.0 * V * dm * (T_all + (2.0 if keep else 3.0) * routed) / (grad_ms * 1e-3) / 1e12
     n_par = V * dm
     launches = sum(r.launches for r in runners) + 2
     line = dict(
@@ -572,6 +597,7 @@ def run_update_step(args):
         vs_baseline=None, dtype="bf16", data="synthetic",
         config=dict(workload="batch128", d=dm, V=V, heads=1, responses=sum(r.R for r in runners), tokens=T_all,
                     micro_batches=[r.T for r in runners], accumulate_dW="fp32, second micro-batch adds",
+                    logits=logits_note(keep, max(r.T for r in runners), V),
                     optimizer="grad norm + AdamW(lr 1e-6, wd 0.01, clip 1.0) on the head, bf16 head rewritten",
                     l2="inputs larger than L2", old_logp="library logp + N(0,0.05) (perf-only input)"),
         gpu_launches=launches * args.steps,
@@ -755,6 +781,9 @@ def main():
     ap.add_argument("--workload", default="qwen3_1p7b", choices=sorted(WL.SPECS) + ["stress", "stress16", "stress_grouped", "stress16_grouped", "stress_grouped_packed",
                                                                      "stress16_grouped_packed", "stress_packed", "adamw", "batch128"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--logits", default="keep", choices=["keep", "recompute"],
+                    help="keep: the forward stores the [T, V] fp32 logits in a buffer lent by the caller and the "
+                         "backward reads them; recompute: the backward repeats the contraction (no extra memory)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--launcher-check", action="store_true",
                     help="start the ranks, join a gloo group, print a line with value null; no GPU work")

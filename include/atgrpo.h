@@ -82,6 +82,10 @@ typedef struct atgrpo_params {
   int32_t* group_scratch;       /* device, [n_groups] int32 owned by the caller, private to the call
                                  * while it runs; the library zeroes it and counts K_g in it      */
   int32_t n_groups;
+  /* atgrpo_policy_loss_fwd / _bwd / _bwd_notify only (NULL / 0 by default): logits kept from the
+   * forward call for the backward call, see atgrpo_policy_loss_logits_bytes().                  */
+  float* logits;                /* device, 256-byte aligned, owned by the caller                    */
+  size_t logits_bytes;          /* size of that buffer in bytes                                     */
 } atgrpo_params;
 
 /* Readings of the expectation in Eq. 2.
@@ -234,7 +238,8 @@ int atgrpo_clipped_loss(
  * M device pointers, W[m] = bf16 [V, d] contiguous (16-byte aligned): the head of policy m.
  * target[j] in [0,V) is the sampled token.  Policy of token j: m = head_of_role[role_of_token[j]]
  * (sigma of the paper) when M > 1; with M == 1 both arrays may be NULL and every token uses W[0].
- *   z_jv = <H_j, W_m[v]>  (bf16 x bf16, fp32 accumulation on tensor cores; never stored)
+ *   z_jv = <H_j, W_m[v]>  (bf16 x bf16, fp32 accumulation on tensor cores; stored only if
+ *                          params->logits is given)
  *   lse[j]  = log sum_v exp(z_jv)          logp[j] = z_{j,target[j]} - lse[j]
  *   rho_j = exp(logp[j] - old_logp[j]),  A = adv[resp_of_token[j]]
  *   loss[m] = (1/T_m) sum_{j of policy m} -min(rho_j*A, clip(rho_j)*A)   (0 if T_m = 0)
@@ -248,6 +253,20 @@ int atgrpo_clipped_loss(
  * token with A = 0.
  * ------------------------------------------------------------------------------------------ */
 size_t atgrpo_policy_loss_workspace_bytes(int64_t T, int32_t d, int32_t V, int32_t M, int32_t is_bwd);
+
+/* Kept logits (optional).  The backward call needs the softmax of every routed token again.  By
+ * default it repeats the contraction z = H W_m^T chunk by chunk (2*T*V*d flop more, no memory).
+ * A caller with HBM to spare can instead lend params->logits, a buffer of
+ * atgrpo_policy_loss_logits_bytes(T, V) bytes = T rows of V rounded up to a multiple of 256 fp32
+ * values (2.45 G logits = 9.8 GB at T = 16157, V = 151936): the forward call then also stores
+ * z_jv (row j = token j, columns >= V unspecified; rows of tokens that belong to no policy are
+ * left untouched), and a backward call that is given the same buffer -- after a forward call
+ * with the same H, W, target and routing arguments, nothing having written to it in between --
+ * reads the logits back instead of recomputing them: a quarter less tensor work for one write and
+ * one read of the buffer.  Both ways produce bit-identical dH and dW.  A buffer that is
+ * misaligned or too small is rejected with ATGRPO_ERR_INVALID_ARG; the library cannot tell
+ * whether the contents belong to these inputs. */
+size_t atgrpo_policy_loss_logits_bytes(int64_t T, int32_t V);
 
 /* Number of kernels one forward (is_bwd = 0) or backward (is_bwd = 1) call enqueues for these
  * sizes on the current device (memsets not counted).  A bookkeeping query with no counterpart in
@@ -279,8 +298,9 @@ int atgrpo_policy_loss_fwd(
  *                overwritten or accumulated into (params->accumulate_dW).
  * dW is a HOST array of M device pointers; dH and every dW[m] must be 32-byte aligned.
  * A policy without tokens gets dW = 0 (or is left unchanged when accumulating).  The [T, V]
- * logits and their gradient are never materialised: dZ lives in a bounded vocabulary-chunk
- * buffer inside the workspace.
+ * gradient of the logits is never materialised: dZ lives in a bounded vocabulary-chunk buffer
+ * inside the workspace; the logits themselves exist in memory only if the caller lends
+ * params->logits (then they are read from there instead of being recomputed).
  * ------------------------------------------------------------------------------------------ */
 int atgrpo_policy_loss_bwd(
     const void* H, int64_t ldH, const void* const* W /* host array */, int32_t M,

@@ -27,7 +27,7 @@ EXPORTS = (
     "atgrpo_group_advantages_noalloc", "atgrpo_group_advantages_packed",
     "atgrpo_group_select_workspace_bytes", "atgrpo_group_select",
     "atgrpo_clipped_loss_workspace_bytes", "atgrpo_clipped_loss",
-    "atgrpo_policy_loss_workspace_bytes", "atgrpo_policy_loss_launch_count",
+    "atgrpo_policy_loss_workspace_bytes", "atgrpo_policy_loss_launch_count", "atgrpo_policy_loss_logits_bytes",
     "atgrpo_policy_loss_fwd", "atgrpo_policy_loss_bwd",
     "atgrpo_policy_loss_bwd_chunks", "atgrpo_policy_loss_bwd_notify",
     "atgrpo_grad_sumsq_workspace_bytes", "atgrpo_grad_sumsq", "atgrpo_adamw_step",
@@ -46,7 +46,8 @@ class _Params(ctypes.Structure):
                 ("accumulate_dW", ctypes.c_int32), ("reduction", ctypes.c_int32),
                 ("candidates_grouped", ctypes.c_int32),
                 ("group_of_resp", ctypes.c_void_p), ("group_scratch", ctypes.c_void_p),
-                ("n_groups", ctypes.c_int32)]
+                ("n_groups", ctypes.c_int32),
+                ("logits", ctypes.c_void_p), ("logits_bytes", ctypes.c_size_t)]
 
 
 class _AdamWParams(ctypes.Structure):
@@ -83,13 +84,16 @@ class Params:
     candidates_grouped: int = 0  # 1: the members of every group are adjacent (checked on the device)
     group_of_resp: object = None   # REDUCE_GROUP_MEAN: int32 CUDA tensor [n_resp], group of every response
     group_scratch: object = None   # REDUCE_GROUP_MEAN: int32 CUDA tensor [n_groups], scratch owned by the caller
+    logits: object = None          # policy loss: fp32 CUDA tensor of atgrpo_policy_loss_logits_bytes(T, V) bytes, kept logits
 
     def c(self) -> _Params:
         n_groups = 0 if self.group_scratch is None else self.group_scratch.numel()
         g, sc = _ptr(self.group_of_resp, torch.int32), _ptr(self.group_scratch, torch.int32)
+        z = _ptr(self.logits, torch.float32)
         return _Params(self.clip_eps_low, self.clip_eps_high, self.std_eps, self.ddof,
                        self.dH_dtype, self.dW_dtype, self.accumulate_dW, self.reduction,
-                       self.candidates_grouped, g.value if g else None, sc.value if sc else None, n_groups)
+                       self.candidates_grouped, g.value if g else None, sc.value if sc else None, n_groups,
+                       z.value if z else None, 0 if self.logits is None else self.logits.numel() * 4)
 
 
 _lib = None
@@ -127,6 +131,8 @@ def lib() -> ctypes.CDLL:
         L.atgrpo_clipped_loss.argtypes = [vp, vp, vp, vp, i64, i64, pp, vp, vp, vp, vp, vp, sz, vp]
         L.atgrpo_policy_loss_workspace_bytes.restype = sz
         L.atgrpo_policy_loss_workspace_bytes.argtypes = [i64, i32, i32, i32, i32]
+        L.atgrpo_policy_loss_logits_bytes.restype = sz
+        L.atgrpo_policy_loss_logits_bytes.argtypes = [i64, i32]
         L.atgrpo_policy_loss_launch_count.restype = i32
         L.atgrpo_policy_loss_launch_count.argtypes = [i64, i32, i32, i32, i32]
         L.atgrpo_policy_loss_fwd.restype = ctypes.c_int
@@ -282,6 +288,10 @@ def atgrpo_clipped_loss(logp, old_logp, resp_of_token, adv, params: Params, loss
 
 def atgrpo_policy_loss_workspace_bytes(T: int, d: int, V: int, M: int, is_bwd: bool) -> int:
     return int(lib().atgrpo_policy_loss_workspace_bytes(T, d, V, M, 1 if is_bwd else 0))
+
+
+def atgrpo_policy_loss_logits_bytes(T: int, V: int) -> int:
+    return int(lib().atgrpo_policy_loss_logits_bytes(T, V))
 
 
 def atgrpo_policy_loss_launch_count(T: int, d: int, V: int, M: int, is_bwd: bool) -> int:

@@ -105,17 +105,20 @@ struct LmHeadProblem {
   int32_t n_sm;
 };
 size_t lm_head_fwd_workspace_bytes(int64_t T_pad, int32_t d, int32_t V, int32_t n_sm);
-// lse[T], logp[T] in token order.
+// lse[T], logp[T] in token order.  keep_logits (optional): [T, lm_head_logits_ld(V)] fp32 in token
+// order, receives every logit of every routed token.
+int64_t lm_head_logits_ld(int32_t V);
 int lm_head_fwd_launch(const LmHeadProblem& p, float* lse, float* logp, void* workspace,
-                       cudaStream_t st);
+                       cudaStream_t st, float* keep_logits = nullptr);
 size_t lm_head_bwd_workspace_bytes(int64_t T_pad, int32_t d, int32_t V, bool dH_direct);
 // coef[T] in token order (0 for tokens that pass no gradient); dH / dW as the C ABI documents.
 // chunk_events (optional, lm_head_bwd_chunks() entries): event c is recorded once the dW rows of
-// vocabulary chunk c are final.
+// vocabulary chunk c are final.  kept_logits (optional): what the forward call stored through
+// keep_logits for the same H, W and routing inputs; dZ is then formed from it instead of a second contraction.
 int lm_head_bwd_launch(const LmHeadProblem& p, const float* lse, const float* coef,
                        const int32_t* row_of_token, const atgrpo_params& prm, void* dH,
                        void* const* dW, void* workspace, cudaStream_t st,
-                       void* const* chunk_events = nullptr);
+                       void* const* chunk_events = nullptr, const float* kept_logits = nullptr);
 int lm_head_bwd_chunk_rows(int64_t T_pad, int32_t d, int32_t V);   // vocabulary rows per chunk
 int device_sm_count(int* n_sm, int* cc_major);
 int lm_head_bwd_chunks(int64_t T_pad, int32_t d, int32_t V);   // vocabulary chunks of one backward call (it makes one GEMM launch more)

@@ -23,6 +23,15 @@
 // owner, warps 2-9 = epilogue (two warps per TMEM lane quarter, each taking half of the columns).
 // Rows are addressed in the "padded row space": the tokens of policy m occupy whole 256-row pair
 // tiles starting at tile_begin[m], so no tile mixes two heads (grouped GEMM).
+//
+// Kept logits (optional): when the caller lends a [T, ldz] fp32 buffer, the kFwd epilogue also
+// stores every logit it reads from tensor memory, and the backward call forms dZ from those
+// instead of repeating the contraction: no kDz items, a quarter of the backward's tensor work
+// gone for 4 bytes per logit written once and read once.  The conversion of chunk c is done by
+// kConvWarps extra warps of the launch that holds the dH and dW tiles of chunk c-1 (plain loads
+// and stores, no barriers), so it runs under the tensor work; chunk 0 has a small launch of its
+// own.  Both ways give the same bits: the stored value is the accumulator the recomputation would
+// produce again.
 #include <cuda_bf16.h>
 #include <cstring>
 #include "internal.h"
@@ -41,6 +50,8 @@ constexpr int kStageBytes = kABytes + kBBytes;     // 32 KiB per CTA and k-step
 constexpr int kBoxBytes = 64 * 64 * 2;             // one 64 x 64 MN-major box, 8 KiB
 constexpr int kGemmThreads = 320;               // producer warp, MMA warp, 8 epilogue warps
 constexpr int kEpilogueThreads = 256;
+constexpr int kConvWarps = 8;                   // kBwd with kept logits: warps that turn logits into dZ
+constexpr int kConvCols = 2048;                 // columns one conversion step covers (eight 32-byte loads per lane in flight)
 constexpr int kTmemCols = 512;
 constexpr int kSmemBytes = kStages * kStageBytes + 1024 /* alignment slack */ + 256 /* barriers */;
 constexpr float kLog2e = 1.4426950408889634f;
@@ -78,6 +89,8 @@ struct GemmArgs {
   const float* coef;      // kDz in, token order
   __nv_bfloat16* dz;      // kDz out: [T_pad, vc]
   int vc;                 // chunk buffer width (multiple of 256)
+  float* logits;          // kept logits [T, ldz] in token order (NULL: none): written by kFwd, read instead of kDz items
+  int64_t ldz;            // row stride of `logits` in elements (V rounded up to a multiple of 256)
   // kDh / kDw: the chunk whose dZ an earlier launch wrote (the maps a_h / a_w point at its buffer)
   int has_g;              // kBwd: the launch holds kDh and kDw items
   int g_begin;            // first vocabulary row of that chunk
@@ -107,6 +120,27 @@ __device__ __forceinline__ void ld_global_v8(const void* p, uint32_t* v) {
   asm volatile("ld.global.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
                : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
                : "l"(p)
+               : "memory");
+}
+
+// Streaming variants for the kept logits: every byte is written once and read once, far apart, so
+// both directions ask L2 to drop the line first and leave the operands of the contractions alone.
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+
+__device__ __forceinline__ void st_stream_v8(void* p, const uint32_t* v, uint64_t policy) {
+  asm volatile("st.global.L2::cache_hint.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8}, %9;" ::"l"(p), "r"(v[0]),
+               "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]), "l"(policy)
+               : "memory");
+}
+
+__device__ __forceinline__ void ld_stream_v8(const void* p, uint32_t* v, uint64_t policy) {
+  asm volatile("ld.global.L1::no_allocate.L2::cache_hint.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8], %9;"
+               : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
+               : "l"(p), "l"(policy)
                : "memory");
 }
 
@@ -196,7 +230,7 @@ struct ItemSeq {
       return;
     }
     small_mode = kDz;
-    n_small = g.has_z ? n_pt * g.n_chunks : 0;
+    n_small = g.has_z && g.logits == nullptr ? n_pt * g.n_chunks : 0;   // kept logits: dZ comes from the conversion warps
     if (g.has_g) {
       const int n_vt = (g.vc_valid + kPairRows - 1) / kPairRows;
       n_h = n_pt * n_dt;
@@ -244,8 +278,74 @@ struct ItemSeq {
   }
 };
 
+// dZ of one vocabulary chunk from kept logits: the element-wise half of the kDz epilogue, for warps
+// that hold no accumulator.  A step is one row of the chunk buffer x kConvCols columns (8 KiB of
+// logits, lanes on consecutive 32-byte pieces); steps are dealt round-robin to `n_workers` warps.
+// Same expression, same operand values, hence the same bits as the kDz epilogue.
+__device__ __forceinline__ void dz_from_logits(const GemmArgs& g, int64_t rows, int worker, int n_workers,
+                                               int lane) {
+  const int n_cols = g.n_vtiles * BN;                       // columns of the chunk buffer this chunk fills
+  const int n_seg = (n_cols + kConvCols - 1) / kConvCols;
+  const int64_t n_steps = rows * n_seg;
+  const uint64_t drop = l2_policy_evict_first();
+  for (int64_t u = worker; u < n_steps; u += n_workers) {
+    const int64_t row = u / n_seg;
+    const int c0 = (int)(u - row * n_seg) * kConvCols + lane * 8;   // this lane's first column in the buffer
+    const int tok = g.tok_of_row[row];
+    int y = -1;
+    float lse2 = 0.f, cf = 0.f;
+    const float* src = g.logits;
+    if (tok >= 0) {
+      y = g.target[tok];
+      if ((unsigned)y >= (unsigned)g.V) {
+        raise_status(g.status, ATGRPO_ERR_BAD_INDEX);
+        y = 0;
+      }
+      lse2 = g.lse[tok] * kLog2e, cf = g.coef[tok];
+      src = g.logits + (size_t)tok * g.ldz + g.v_begin + c0;
+    }
+    uint32_t z[kConvCols / BN][8];
+#pragma unroll
+    for (int j = 0; j < kConvCols / BN; ++j) {
+      const int col = c0 + j * BN;
+      // a padding row, or a piece that lies wholly beyond the vocabulary, is not read at all
+      if (tok >= 0 && col < n_cols && g.v_begin + col < g.V) {
+        ld_stream_v8(src + j * BN, z[j], drop);
+      } else {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) z[j][i] = 0u;
+      }
+    }
+#pragma unroll
+    for (int j = 0; j < kConvCols / BN; ++j) {
+      const int col = c0 + j * BN;
+      if (col >= n_cols) continue;
+      const int v0 = g.v_begin + col;                        // vocabulary row of z[j][0]
+      float gz[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        gz[i] = cf * ex2(fmaf(__uint_as_float(z[j][i]), kLog2e, -lse2));
+        if (v0 + i == y) gz[i] -= cf;
+        if (tok < 0 || v0 + i >= g.V) gz[i] = 0.f;
+      }
+      uint4 w;
+      __nv_bfloat162* wh = reinterpret_cast<__nv_bfloat162*>(&w);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) wh[i] = __floats2bfloat162_rn(gz[2 * i], gz[2 * i + 1]);
+      *reinterpret_cast<uint4*>(g.dz + (size_t)row * g.vc + col) = w;
+    }
+  }
+}
+
+// The conversion on its own, for the first chunk of a backward call (no tensor work to hide under yet).
+__global__ void __launch_bounds__(256)
+k_dz_from_logits(const GemmArgs g) {
+  const int64_t rows = (int64_t)g.sched->tile_begin[g.M] * BM;
+  dz_from_logits(g, rows, blockIdx.x * 8 + (threadIdx.x >> 5), gridDim.x * 8, threadIdx.x & 31);
+}
+
 template <int kMode>    // kFwd or kBwd
-__global__ void __launch_bounds__(kGemmThreads, 1)
+__global__ void __launch_bounds__(kMode == kBwd ? kGemmThreads + 32 * kConvWarps : kGemmThreads, 1)
 k_lm_head(const __grid_constant__ Maps maps, const GemmArgs g) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -381,6 +481,11 @@ k_lm_head(const __grid_constant__ Maps maps, const GemmArgs g) {
         }
       }
     }
+  } else if (warp >= kGemmThreads / 32) {
+    // ------------------------------------------------------------------ conversion warps (kBwd, kept logits)
+    if (kMode == kBwd && g.has_z && g.logits != nullptr)
+      dz_from_logits(g, (int64_t)sched->tile_begin[g.M] * BM, blockIdx.x * kConvWarps + (warp - kGemmThreads / 32),
+                     gridDim.x * kConvWarps, lane);
   } else {
     // ------------------------------------------------------------------ epilogue warps
     // Two warps per TMEM lane quarter (a warp can only read the quarter warp_id % 4): the first
@@ -394,6 +499,7 @@ k_lm_head(const __grid_constant__ Maps maps, const GemmArgs g) {
     int acc = 0;
     uint32_t acc_phase = 0;
     bool ok = true;
+    const uint64_t drop = l2_policy_evict_first();
     const uint32_t tempty_leader0 = mapa_shared(tempty_bar(0), 0), tempty_leader1 = mapa_shared(tempty_bar(1), 0);
     while (ok && seq.next(item_mode, it)) {
       const int mode = kMode == kFwd ? (int)kFwd : item_mode;
@@ -416,6 +522,8 @@ k_lm_head(const __grid_constant__ Maps maps, const GemmArgs g) {
         bool have_zt = false;
         float lse2 = 0.f, cf = 0.f;
         if (mode == kDz && tok >= 0) lse2 = g.lse[tok] * kLog2e, cf = g.coef[tok];
+        float* keep_row = nullptr;
+        if (mode == kFwd && g.logits != nullptr && tok >= 0) keep_row = g.logits + (size_t)tok * g.ldz;
         for (int nt = t.nt_begin; ok && nt < t.nt_end; ++nt) {
           const int n0 = t.n0 + (nt - t.nt_begin) * BN;
           if (!(ok = mbar_wait_backoff(tfull_bar(acc), acc_phase, s_abort, g.status))) break;
@@ -427,6 +535,11 @@ k_lm_head(const __grid_constant__ Maps maps, const GemmArgs g) {
             tmem_ld32(lane_addr + acc * BN + c * 32, r);
             tmem_ld_wait();
             if (mode == kFwd) {
+              if (keep_row != nullptr) {
+                // the logits as the tensor cores delivered them, 128 bytes of this token's row
+#pragma unroll
+                for (int q8 = 0; q8 < 4; ++q8) st_stream_v8(keep_row + col0 + 8 * q8, r + 8 * q8, drop);
+              }
               if (y >= col0 && y < col0 + 32) {
 #pragma unroll
                 for (int i = 0; i < 32; ++i)
@@ -778,7 +891,8 @@ BwdPlan bwd_plan(int64_t T_pad, int d, int V, bool dH_direct) {
 // Launches `pairs` clusters of two CTAs (never more than can be resident at once); `items` is an
 // upper bound of the launch's work items.
 template <int kMode>
-int launch_gemm(const Maps& maps, const GemmArgs& g, int64_t items, int n_sm, cudaStream_t st) {
+int launch_gemm(const Maps& maps, const GemmArgs& g, int64_t items, int n_sm, cudaStream_t st,
+                int threads = kGemmThreads) {
   if (cudaFuncSetAttribute(k_lm_head<kMode>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            kSmemBytes) != cudaSuccess)
     return ATGRPO_ERR_CUDA;
@@ -787,7 +901,7 @@ int launch_gemm(const Maps& maps, const GemmArgs& g, int64_t items, int n_sm, cu
   attr[0].val.clusterDim.x = 2, attr[0].val.clusterDim.y = 1, attr[0].val.clusterDim.z = 1;
   cudaLaunchConfig_t cfg;
   memset(&cfg, 0, sizeof(cfg));
-  cfg.blockDim = dim3(kGemmThreads, 1, 1);
+  cfg.blockDim = dim3(threads, 1, 1);
   cfg.dynamicSmemBytes = kSmemBytes;
   cfg.stream = st;
   cfg.attrs = attr;
@@ -834,8 +948,10 @@ size_t lm_head_fwd_workspace_bytes(int64_t T_pad, int32_t d, int32_t V, int32_t 
   return fwd_plan(T_pad, V, n_sm).total;
 }
 
+int64_t lm_head_logits_ld(int32_t V) { return ((int64_t)V + BN - 1) / BN * BN; }
+
 int lm_head_fwd_launch(const LmHeadProblem& p, float* lse, float* logp, void* workspace,
-                       cudaStream_t st) {
+                       cudaStream_t st, float* keep_logits) {
   const FwdPlan pl = fwd_plan(p.T_pad, p.V, p.n_sm);
   char* ws = static_cast<char*>(workspace);
   Maps maps;
@@ -849,6 +965,7 @@ int lm_head_fwd_launch(const LmHeadProblem& p, float* lse, float* logp, void* wo
   g.part_m = reinterpret_cast<float*>(ws + pl.part_m);
   g.part_s = reinterpret_cast<float*>(ws + pl.part_s);
   g.zt = reinterpret_cast<float*>(ws + pl.zt);
+  g.logits = keep_logits, g.ldz = lm_head_logits_ld(p.V);
   int rc = launch_gemm<kFwd>(maps, g, (p.T_pad / kPairRows) * pl.n_chunks, p.n_sm, st);
   if (rc != ATGRPO_OK) return rc;
   const int cgrid = (int)((p.T_pad + 31) / 32 > 0 ? (p.T_pad + 31) / 32 : 1);
@@ -863,7 +980,8 @@ size_t lm_head_bwd_workspace_bytes(int64_t T_pad, int32_t d, int32_t V, bool dH_
 
 int lm_head_bwd_launch(const LmHeadProblem& p, const float* lse, const float* coef,
                        const int32_t* row_of_token, const atgrpo_params& prm, void* dH,
-                       void* const* dW, void* workspace, cudaStream_t st, void* const* chunk_events) {
+                       void* const* dW, void* workspace, cudaStream_t st, void* const* chunk_events,
+                       const float* kept_logits) {
   const bool dH_direct = false;   // rows are compacted: dH always goes through the accumulator
   const BwdPlan pl = bwd_plan(p.T_pad, p.d, p.V, dH_direct);
   char* ws = static_cast<char*>(workspace);
@@ -896,6 +1014,7 @@ int lm_head_bwd_launch(const LmHeadProblem& p, const float* lse, const float* co
     int64_t items = 0;
     g.vc = pl.vc;
     g.lse = lse, g.coef = coef;
+    g.logits = const_cast<float*>(kept_logits), g.ldz = lm_head_logits_ld(p.V);
     g.dh_acc = dh_acc;
     for (int m = 0; m < p.M; ++m) g.dW[m] = dW[m];
     g.dw_bf16 = prm.dW_dtype == ATGRPO_BF16, g.dw_accumulate = prm.accumulate_dW;
@@ -919,7 +1038,16 @@ int lm_head_bwd_launch(const LmHeadProblem& p, const float* lse, const float* co
       maps.a_w = a_w[(c - 1) % n_buf];
       items += n_pt * n_dt + (int64_t)p.M * ((g.vc_valid + kPairRows - 1) / kPairRows) * n_dt;
     }
-    const int rc = launch_gemm<kBwd>(maps, g, items, p.n_sm, st);
+    if (kept_logits != nullptr && c == 0) {
+      // nothing to hide the first chunk's conversion under: a launch of its own, every SM full of warps
+      k_dz_from_logits<<<4 * p.n_sm, 256, 0, st>>>(g);
+      const int rc0 = launch_ok();
+      if (rc0 != ATGRPO_OK) return rc0;
+      continue;
+    }
+    const int rc = launch_gemm<kBwd>(maps, g, items, p.n_sm, st,
+                                     kept_logits != nullptr && c < n_chunks ? kGemmThreads + 32 * kConvWarps
+                                                                            : kGemmThreads);
     if (rc != ATGRPO_OK) return rc;
     if (chunk_events != nullptr && c > 0)             // the dW rows of chunk c - 1 are final
       ATGRPO_CUDA_OK(cudaEventRecord(static_cast<cudaEvent_t>(chunk_events[c - 1]), st));

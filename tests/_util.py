@@ -90,6 +90,32 @@ class PolicyCase:
         self.old_logp = to_dev(old_logp.to(torch.float32))
         self.grad_loss = None if grad_loss is None else to_dev(grad_loss.to(torch.float32))
 
+    def lend_logits(self):
+        """Lends the library a logits buffer (params.logits) full of NaN: the next forward stores
+        the logits there and the backward calls after it read them instead of recomputing.
+        Whatever the library leaves unwritten must never reach a result."""
+        import dataclasses
+        n = A.atgrpo_policy_loss_logits_bytes(self.T, self.spec.V) // 4
+        buf = torch.full((n,), float("nan"), dtype=torch.float32, device=DEV)
+        self.prm = dataclasses.replace(self.prm, logits=buf)
+        return buf
+
+    def bwd_both_ways(self, logp, lse):
+        """Backward from the kept logits (lend_logits() and fwd() came first) and again with the
+        contraction recomputed: the two must agree bit for bit.  Returns the first."""
+        import dataclasses
+        assert self.prm.logits is not None
+        kept = self.bwd(logp, lse)
+        lent = self.prm
+        self.prm = dataclasses.replace(lent, logits=None)
+        again = self.bwd(logp, lse)
+        self.prm = lent
+        assert again["status"] == kept["status"]
+        assert torch.equal(kept["dH"], again["dH"]), "dH: kept logits vs recomputed"
+        for m in range(self.M):
+            assert torch.equal(kept["dW"][m], again["dW"][m]), ("dW: kept logits vs recomputed", m)
+        return kept
+
     def fwd(self, want_routing=True):
         f32, i32 = torch.float32, torch.int32
         T, M = self.T, self.M

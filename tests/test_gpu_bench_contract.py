@@ -35,7 +35,10 @@ def test_default_arm_line():
     T, d, V = r["config"]["tokens_per_gpu"], r["config"]["d"], r["config"]["V"]
     want = 6.0 * T * V * d / ((ph["forward"] + ph["backward"]) * 1e-3) / 1e12
     assert abs(rf["achieved"] - want) <= 1e-6 * want and "all launches" in rf["kernel"]
-    assert 0 < rf["routed_rows"] <= T and rf["executed_frac"] >= rf["frac"] * 0.99
+    # by default the forward keeps the logits: the tensor cores execute T + 2*routed row passes, at most the algorithmic 3*T
+    assert r["config"]["logits"].startswith("kept")
+    assert 0 < rf["routed_rows"] <= T
+    assert abs(rf["executed_frac"] / rf["frac"] - (T + 2.0 * rf["routed_rows"]) / (3.0 * T)) < 1e-6
     assert rf["frac_of_nominal_2250"] < rf["frac"] and rf["forward_frac"] > 0 and rf["backward_algorithmic_frac"] > 0
     assert rf["algorithmic_bytes"] == rf["algorithmic_bytes_forward"] + rf["algorithmic_bytes_backward"]
     assert rf["traffic"] is None or rf["traffic"] == rf["traffic_forward"] + rf["traffic_backward"]
@@ -43,6 +46,14 @@ def test_default_arm_line():
     assert e["value"] > 0 and e["h2d_bytes_per_step"] > 0 and e["d2h_bytes_per_step"] == 4
     c = r["cpu_baseline"]
     assert c["kind"] == "oracle" and c["value"] > 0 and c["cores"] >= 1 and "tokens" in c["sample"]
+
+
+def test_recompute_arm_line():
+    # --logits recompute: no [T, V] buffer, the backward repeats the contraction on the routed rows
+    r = _run("--workload", "tiny", "--steps", "3", "--warmup", "3", "--logits", "recompute", "--no-cpu-baseline")
+    rf, T = r["roofline"], r["config"]["tokens_per_gpu"]
+    assert r["config"]["logits"].startswith("recomputed") and r["value"] > 0
+    assert abs(rf["executed_frac"] / rf["frac"] - (T + 3.0 * rf["routed_rows"]) / (3.0 * T)) < 1e-6
 
 
 def test_reference_arm_line():
@@ -67,4 +78,5 @@ def test_update_step_line():
     assert r["config"]["tokens"] > 100_000 and len(r["config"]["micro_batches"]) == 2
     assert r["value"] > 0 and r["phases_ms"]["gradient"] > r["phases_ms"]["optimizer"] > 0
     rf = r["roofline"]
-    assert rf["bound"] == "tensor" and 0 < rf["frac"] <= rf["executed_frac"] and rf["optimizer_gbs"] > 0
+    assert r["config"]["logits"].startswith("kept")
+    assert rf["bound"] == "tensor" and 0 < rf["executed_frac"] <= rf["frac"] and rf["optimizer_gbs"] > 0

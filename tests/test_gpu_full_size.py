@@ -58,6 +58,7 @@ def test_full_size_sparse_advantages(name):
     c = _sparse_case(name, n_active_resp=2) if name == "long_resp" else _sparse_case(name)
     b, head, act, M = c["b"], c["head"], c["act"], c["b"]["spec"].n_heads
     case = U.PolicyCase(b, c["adv"], c["old"])
+    case.lend_logits()                                    # the timed configuration: logits kept by the forward
     out = case.fwd()
     assert out["status"] == 0
     assert np.array_equal(out["role_offsets"].numpy(), c["offsets"])
@@ -77,7 +78,7 @@ def test_full_size_sparse_advantages(name):
     lse_in = torch.from_numpy(np.full(b["T"], 12.0, dtype=np.float32))
     logp_in[torch.from_numpy(c["sample"])] = torch.from_numpy(c["logp_s"]).float()
     lse_in[torch.from_numpy(c["sample"])] = torch.from_numpy(c["lse_s"]).float()
-    g = case.bwd(logp_in, lse_in)
+    g = case.bwd_both_ways(logp_in, lse_in)               # from the kept logits, and recomputed: same bits
     assert g["status"] == 0
     ta = torch.from_numpy(act)
     dH_act, dW = O.policy_loss_grads(b["H"][ta], b["W"], b["target"][ta], c["old"][ta], c["adv"], resp_act,

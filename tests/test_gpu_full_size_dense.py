@@ -4,7 +4,9 @@ chunks) on a quarter of its batch.
 
 Inputs are the benchmark's batch with every response carrying its Eq. 1 advantage and old_logp
 built from the ORACLE's log-probs, so the backward runs every row tile, every vocabulary chunk and
-both alternating dZ buffers exactly as in the timed step.  The oracle computes the full forward
+both alternating dZ buffers exactly as in the timed step: the forward keeps the logits in a lent
+buffer and the backward reads them (the backward that recomputes them instead is run as well and
+must give the same bits in every element of dH and dW).  The oracle computes the full forward
 (lse, logp for every token; about 1e13 fp64 flop per head pass) and then, from its own lse and
 gradient factors, single rows of dH and dW:
   * dH rows of tokens drawn from EVERY 128-row half of every 256-row pair tile of the backward's
@@ -64,6 +66,7 @@ def test_full_size_dense_backward_rows(name, request):
     gl = torch.tensor([1.0, 0.5, 2.0][:M]) if M > 1 else None
 
     case = U.PolicyCase(b, adv, old, grad_loss=gl)
+    case.lend_logits()                                             # as in the timed step: the forward keeps the logits
     out = case.fwd()
     assert out["status"] == 0
     assert np.array_equal(out["role_offsets"].numpy(), offsets) and np.array_equal(out["role_perm"].numpy(), perm)
@@ -73,7 +76,8 @@ def test_full_size_dense_backward_rows(name, request):
     np.testing.assert_allclose(out["loss"].numpy(), rloss, rtol=1e-3)
     assert np.abs(out["clip_counts"].numpy() - rcc).max() <= 2 and rcc.sum() > 100
 
-    g = case.bwd(torch.from_numpy(logp).float(), torch.from_numpy(lse).float())
+    # the backward as timed (from the kept logits) and with the contraction recomputed: same bits
+    g = case.bwd_both_ways(torch.from_numpy(logp).float(), torch.from_numpy(lse).float())
     assert g["status"] == 0
     c = O.dloss_dlogp(logp, old, adv, b["resp_of_token"], head, M, None if gl is None else gl.numpy())
     n_chunks, rows_per_chunk = A.atgrpo_policy_loss_bwd_chunks(T, spec.d, V, M)
