@@ -6,6 +6,12 @@ backward to dH and dW, on one synthetic on-policy batch.  Default workload: the
 Qwen3-1.7B-shaped single-policy head (d=2048, V=151936, ~16K response tokens).
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+                  [--logits keep|recompute]
+
+By default the forward keeps the [T, V] fp32 logits in a buffer lent to the library and the backward
+reads them (a quarter less tensor work for 8 bytes of DRAM traffic per logit); --logits recompute
+times the path that never writes the logits to memory and repeats the contraction in the backward.
+On one GPU the default line carries that second configuration as well ("logits_recomputed").
 
 Prints ONE JSON line (rank 0).  With --impl reference the fp64 CPU oracle is timed instead, on a
 bounded token sample of the same workload.
@@ -13,6 +19,7 @@ bounded token sample of the same workload.
 from __future__ import annotations
 
 import argparse
+import dataclasses
 import json
 import os
 import statistics
@@ -45,14 +52,15 @@ def kernel_digest():
     return h.hexdigest()[:16]
 
 
-def captured_traffic(workload):
-    """(forward bytes, backward bytes) of one step's k_lm_head launches, or None."""
+def captured_traffic(workload, mode):
+    """(forward bytes, backward bytes) of one step's LM-head launches with the logits kept
+    (mode "keep") or recomputed ("recompute"), or None."""
     try:
         with open(TRAFFIC_JSON) as f:
             rec = json.load(f)
     except (OSError, ValueError):
         return None
-    e = rec.get("workloads", {}).get(workload)
+    e = rec.get("workloads", {}).get(workload, {}).get(mode)
     if e is None or rec.get("kernel_digest") != kernel_digest():
         return None
     return float(e["forward_bytes"]), float(e["backward_bytes"])
@@ -413,6 +421,31 @@ def run_ours(args):
     torch.cuda.synchronize()
     ms_e2e = e_start.elapsed_time(e_end)
 
+    # ---- the same step with the logits recomputed in the backward (nothing of size T x V in memory),
+    # timed the same way right after, so that one line carries both ways of running the path
+    alt = None
+    if world == 1 and r.logits is not None:
+        r.prm = dataclasses.replace(r.prm, logits=None)
+        for _ in range(3):
+            step()
+        torch.cuda.synchronize()
+        am = [[ev() for _ in range(3)] for _ in range(args.steps)]
+        a_start, a_end = ev(), ev()
+        a_start.record()
+        for k in range(args.steps):
+            r.advantages()
+            am[k][0].record()
+            r.forward()
+            am[k][1].record()
+            r.backward(comm)
+            am[k][2].record()
+        a_end.record()
+        torch.cuda.synchronize()
+        alt = dict(ms_total=a_start.elapsed_time(a_end),
+                   fwd_ms=statistics.mean(m[0].elapsed_time(m[1]) for m in am),
+                   bwd_ms=statistics.mean(m[1].elapsed_time(m[2]) for m in am))
+        r.prm = dataclasses.replace(r.prm, logits=r.logits)
+
     t = torch.tensor([ms_total, ms_e2e], dtype=torch.float64, device=dev)
     tokens = torch.tensor([float(r.T)], dtype=torch.float64, device=dev)
     if world > 1:
@@ -445,7 +478,7 @@ def run_ours(args):
     bwd_passes = 2.0 if r.logits is not None else 3.0         # dH, dW (+ the logits again unless they were kept)
     executed_flops = pass_flops * (1.0 + bwd_passes * r.routed_rows / max(r.T, 1))
     exec_tf = tf(executed_flops, lm_s)
-    traffic = captured_traffic(spec.name) if world == 1 else None
+    traffic = captured_traffic(spec.name, args.logits) if world == 1 else None
     n_bwd_chunks = r.A.atgrpo_policy_loss_bwd_chunks(r.T, spec.d, spec.V, r.M)[0]
     dw_elem, dh_elem = 4.0, 2.0
     kept = r.logits is not None
@@ -496,6 +529,16 @@ def run_ours(args):
         e2e=dict(value=tokens_all * args.steps / (ms_e2e * 1e-3), unit=UNIT,
                  h2d_bytes_per_step=r.h2d_bytes, d2h_bytes_per_step=r.M * 4),
         clocks=clocks, cpu_baseline=cpu_baseline)
+    if alt is not None:
+        a_s = (alt["fwd_ms"] + alt["bwd_ms"]) * 1e-3
+        a_exec = tf(pass_flops * (1.0 + 3.0 * r.routed_rows / max(r.T, 1)), a_s)
+        line["logits_recomputed"] = dict(
+            note="the same step with --logits recompute, timed right after the main region (same steps, "
+                 "3 warm-up steps): no [T, V] buffer, the backward repeats the contraction",
+            value=r.T * args.steps / (alt["ms_total"] * 1e-3), unit=UNIT, ms_per_step=alt["ms_total"] / args.steps,
+            phases_ms=dict(forward=alt["fwd_ms"], backward=alt["bwd_ms"]),
+            frac=tf(3.0 * pass_flops, a_s) / peaks["bf16_sustained"], executed_tflops=a_exec,
+            executed_frac=a_exec / peaks["bf16_sustained"], executed_frac_of_nominal_2250=a_exec / 2250.0)
     print(json.dumps(line), flush=True)
 
 
