@@ -36,6 +36,16 @@ def _check(b, sigma=0.3, prm=None, tol_fro=5e-3):
             assert U.rel_fro(g["dW"][m].numpy(), dW[m]) <= tol_fro
         else:
             assert (g["dW"][m] == 0).all()
+    # once more with the logits kept by the forward: same forward outputs, same gradient bits
+    case.lend_logits()
+    out2 = case.fwd()
+    assert out2["status"] == 0
+    for k in ("loss", "logp", "lse", "role_offsets", "role_perm", "clip_counts"):
+        assert torch.equal(out2[k], out[k]), k
+    g2 = case.bwd(torch.from_numpy(logp).float(), torch.from_numpy(lse).float())
+    assert g2["status"] == 0 and torch.equal(g2["dH"], g["dH"])
+    for m in range(M):
+        assert torch.equal(g2["dW"][m], g["dW"][m]), m
     return out, g
 
 
@@ -77,6 +87,14 @@ def test_zero_tokens():
     A.atgrpo_policy_loss_fwd(H, W, e_i, None, None, e_i, adv, e_f, A.Params(), loss, e_f, e_f, device_status=st, workspace=ws)
     dW = [torch.full((V, d), 7.0, device=dev)]
     A.atgrpo_policy_loss_bwd(H, W, e_i, None, None, e_i, adv, e_f, e_f, e_f, None, A.Params(), H, dW, st, ws)
+    torch.cuda.synchronize()
+    assert loss.item() == 0 and (dW[0] == 0).all() and int(st.item()) == 0
+    # the same with a (necessarily empty) logits buffer lent
+    assert A.atgrpo_policy_loss_logits_bytes(0, V) == 0
+    prm = A.Params(logits=torch.zeros(64, device=dev))
+    loss.fill_(7.0), dW[0].fill_(7.0)
+    A.atgrpo_policy_loss_fwd(H, W, e_i, None, None, e_i, adv, e_f, prm, loss, e_f, e_f, device_status=st, workspace=ws)
+    A.atgrpo_policy_loss_bwd(H, W, e_i, None, None, e_i, adv, e_f, e_f, e_f, None, prm, H, dW, st, ws)
     torch.cuda.synchronize()
     assert loss.item() == 0 and (dW[0] == 0).all() and int(st.item()) == 0
 

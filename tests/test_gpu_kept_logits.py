@@ -154,3 +154,51 @@ def test_a_logits_buffer_that_is_too_small_or_misaligned_is_rejected():
     assert A.atgrpo_policy_loss_logits_bytes(0, V) == 0
     case.prm = dataclasses.replace(case.prm, logits=big[:n])
     assert case.fwd(want_routing=False)["status"] == 0
+
+
+def test_bad_target_with_kept_logits_is_flagged_in_both_calls_and_stays_in_bounds():
+    # a target id outside the vocabulary is read as token 0 (documented); forward and backward each flag it
+    b, case, f = _case(WL.SPECS["tiny"])
+    T, V = b["T"], WL.SPECS["tiny"].V
+    j = int((b["resp_of_token"] == 1).nonzero()[0])        # a token whose response has a non-zero advantage
+    b2 = dict(b)
+    b2["target"] = b["target"].clone()
+    b2["target"][j] = V + 5
+    b0 = dict(b)
+    b0["target"] = b["target"].clone()
+    b0["target"][j] = 0
+    adv = case.adv.cpu()
+    res = []
+    for batch in (b2, b0):
+        c = U.PolicyCase(batch, adv, torch.zeros(T))
+        c.lend_logits()
+        out = c.fwd(want_routing=False)
+        c.old_logp = (out["logp"] + 0.1).to(U.DEV)
+        g = c.bwd(out["logp"], out["lse"])
+        res.append((out, g))
+    (o_bad, g_bad), (o_ok, g_ok) = res
+    assert o_bad["status"] == A.ERR_BAD_INDEX and g_bad["status"] == A.ERR_BAD_INDEX
+    assert o_ok["status"] == 0 and g_ok["status"] == 0
+    assert torch.equal(o_bad["logp"], o_ok["logp"]) and torch.equal(g_bad["dH"], g_ok["dH"])
+    assert torch.equal(g_bad["dW"][0], g_ok["dW"][0])
+
+
+def test_group_mean_reduction_from_kept_logits():
+    # the per-group reading of Eq. 2 changes only the gradient factor: kept and recomputed logits agree bit for bit
+    spec = WL.SPECS["mid_multi"]
+    b = WL.make_rollout(spec)
+    T, V, M = b["T"], spec.V, spec.n_heads
+    ref = U.oracle_group_advantages(b["rewards"], b["env_id"], b["role_id"], b["turn_id"], spec.n_env, spec.n_role,
+                                    spec.n_turn)
+    G = spec.n_env * spec.n_role * spec.n_turn
+    gof = torch.from_numpy(ref["group_of_cand"].astype(np.int32)).to(U.DEV)
+    prm = A.Params(reduction=A.REDUCE_GROUP_MEAN, group_of_resp=gof,
+                   group_scratch=torch.zeros(G, dtype=torch.int32, device=U.DEV))
+    case = U.PolicyCase(b, torch.from_numpy(ref["adv"]), torch.zeros(T), prm=prm)
+    f = case.fwd(want_routing=False)
+    assert f["status"] == 0
+    case.old_logp = (f["logp"] + 0.002 * torch.sin(torch.arange(T).float())).to(U.DEV)
+    case.lend_logits()
+    assert case.fwd(want_routing=False)["status"] == 0
+    g = case.bwd_both_ways(f["logp"], f["lse"])
+    assert g["status"] == 0 and float(g["dH"].abs().max()) > 0
