@@ -259,9 +259,10 @@ size_t atgrpo_policy_loss_workspace_bytes(int64_t T, int32_t d, int32_t V, int32
  * A caller with HBM to spare can instead lend params->logits, a buffer of
  * atgrpo_policy_loss_logits_bytes(T, V) bytes = T rows of V rounded up to a multiple of 256 fp32
  * values (2.45 G logits = 9.8 GB at T = 16157, V = 151936): the forward call then also stores
- * z_jv (row j = token j, columns >= V unspecified; rows of tokens that belong to no policy are
- * left untouched), and a backward call that is given the same buffer -- after a forward call
- * with the same H, W, target and routing arguments, nothing having written to it in between --
+ * z_jv (row j = token j, columns >= V unspecified; rows of tokens that belong to no policy, or
+ * whose response has advantage 0 and therefore passes no gradient, are left untouched), and a
+ * backward call that is given the same buffer -- after a forward call
+ * with the same H, W, target, adv and routing arguments, nothing having written to it in between --
  * reads the logits back instead of recomputing them: a quarter less tensor work for one write and
  * one read of the buffer.  Both ways produce bit-identical dH and dW.  A buffer that is
  * misaligned or too small is rejected with ATGRPO_ERR_INVALID_ARG; the library cannot tell

@@ -248,6 +248,7 @@ int atgrpo_policy_loss_fwd(const void* H, int64_t ldH, const void* const* W, int
   for (int m = 0; m < M; ++m) p.W[m] = W[m];
   p.M = M, p.d = d, p.V = V, p.T = T, p.T_pad = pl.T_pad;
   p.sched = sched, p.tok_of_row = tok_of_row, p.target = target, p.device_status = device_status;
+  p.resp_of_token = resp_of_token, p.adv = adv, p.n_resp = n_resp;
   p.n_sm = n_sm;
   rc = lm_head_fwd_launch(p, lse, logp, ws + pl.gemm, st, params->logits);
   if (rc != ATGRPO_OK) return rc;
@@ -363,6 +364,7 @@ int policy_loss_bwd_impl(const void* H, int64_t ldH, const void* const* W, int32
   for (int m = 0; m < M; ++m) p.W[m] = W[m];
   p.M = M, p.d = d, p.V = V, p.T = T, p.T_pad = pl.T_pad;
   p.sched = sched, p.tok_of_row = tok_of_row, p.target = target, p.device_status = device_status;
+  p.resp_of_token = resp_of_token, p.adv = adv, p.n_resp = n_resp;
   p.n_sm = n_sm;
   return lm_head_bwd_launch(p, lse, coef, row_of_token, *params, dH, dW, ws + pl.gemm, st,
                             notify ? chunk_events : nullptr, params->logits);

@@ -101,6 +101,9 @@ struct LmHeadProblem {
   const Schedule* sched;     // device
   const int32_t* tok_of_row; // device, [T_pad]
   const int32_t* target;     // device, [T] in token order
+  const int32_t* resp_of_token;   // device, [T]; with adv[n_resp]: read by the forward only when it keeps the logits
+  const float* adv;
+  int64_t n_resp;
   int32_t* device_status;
   int32_t n_sm;
 };

@@ -25,7 +25,8 @@
 // tiles starting at tile_begin[m], so no tile mixes two heads (grouped GEMM).
 //
 // Kept logits (optional): when the caller lends a [T, ldz] fp32 buffer, the kFwd epilogue also
-// stores every logit it reads from tensor memory, and the backward call forms dZ from those
+// stores every logit it reads from tensor memory (rows of tokens whose response has advantage 0 are
+// skipped: they pass no gradient whatever their ratio), and the backward call forms dZ from those
 // instead of repeating the contraction: no kDz items, a quarter of the backward's tensor work
 // gone for 4 bytes per logit written once and read once.  The conversion of chunk c is done by
 // kConvWarps extra warps of the launch that holds the dH and dW tiles of chunk c-1 (plain loads
@@ -91,6 +92,9 @@ struct GemmArgs {
   int vc;                 // chunk buffer width (multiple of 256)
   float* logits;          // kept logits [T, ldz] in token order (NULL: none): written by kFwd, read instead of kDz items
   int64_t ldz;            // row stride of `logits` in elements (V rounded up to a multiple of 256)
+  const int32_t* resp_of_token;   // kFwd with kept logits: a token whose response has advantage 0 passes no
+  const float* adv;               // gradient whatever its ratio, so its logits are not stored
+  int64_t n_resp;
   // kDh / kDw: the chunk whose dZ an earlier launch wrote (the maps a_h / a_w point at its buffer)
   int has_g;              // kBwd: the launch holds kDh and kDw items
   int g_begin;            // first vocabulary row of that chunk
@@ -523,7 +527,10 @@ k_lm_head(const __grid_constant__ Maps maps, const GemmArgs g) {
         float lse2 = 0.f, cf = 0.f;
         if (mode == kDz && tok >= 0) lse2 = g.lse[tok] * kLog2e, cf = g.coef[tok];
         float* keep_row = nullptr;
-        if (mode == kFwd && g.logits != nullptr && tok >= 0) keep_row = g.logits + (size_t)tok * g.ldz;
+        if (mode == kFwd && g.logits != nullptr && tok >= 0) {
+          const int rsp = g.resp_of_token[tok];
+          if ((unsigned)rsp < (unsigned)g.n_resp && g.adv[rsp] != 0.f) keep_row = g.logits + (size_t)tok * g.ldz;
+        }
         for (int nt = t.nt_begin; ok && nt < t.nt_end; ++nt) {
           const int n0 = t.n0 + (nt - t.nt_begin) * BN;
           if (!(ok = mbar_wait_backoff(tfull_bar(acc), acc_phase, s_abort, g.status))) break;
@@ -966,6 +973,7 @@ int lm_head_fwd_launch(const LmHeadProblem& p, float* lse, float* logp, void* wo
   g.part_s = reinterpret_cast<float*>(ws + pl.part_s);
   g.zt = reinterpret_cast<float*>(ws + pl.zt);
   g.logits = keep_logits, g.ldz = lm_head_logits_ld(p.V);
+  g.resp_of_token = p.resp_of_token, g.adv = p.adv, g.n_resp = p.n_resp;
   int rc = launch_gemm<kFwd>(maps, g, (p.T_pad / kPairRows) * pl.n_chunks, p.n_sm, st);
   if (rc != ATGRPO_OK) return rc;
   const int cgrid = (int)((p.T_pad + 31) / 32 > 0 ? (p.T_pad + 31) / 32 : 1);

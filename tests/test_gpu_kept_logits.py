@@ -43,7 +43,9 @@ def test_forward_stores_the_logits_of_every_routed_token(name):
     if spec.n_heads > 1:
         b["role_of_token"][7] = spec.n_role + 3            # one token that belongs to no policy
     T, V, M = b["T"], spec.V, spec.n_heads
-    case = U.PolicyCase(b, torch.ones(b["R"]), torch.zeros(T))
+    adv = torch.ones(b["R"])
+    adv[::3] = 0.0                                         # every third response carries no gradient
+    case = U.PolicyCase(b, adv, torch.zeros(T))
     plain = case.fwd(want_routing=False)
     buf, ld = _lend(case, T, V)
     kept = case.fwd(want_routing=False)
@@ -57,15 +59,17 @@ def test_forward_stores_the_logits_of_every_routed_token(name):
         role = b["role_of_token"].numpy()
         ok = (role >= 0) & (role < spec.n_role)
         head = np.where(ok, b["head_of_role"].numpy()[np.clip(role, 0, spec.n_role - 1)], -1)
+    live = adv.numpy()[b["resp_of_token"].numpy()] != 0
+    assert 0 < live.sum() < T
     Hf = b["H"].double().numpy()
     for m in range(M):
-        rows = np.nonzero(head == m)[0]
+        rows = np.nonzero((head == m) & live)[0]
         ref = Hf[rows] @ b["W"][m].double().numpy().T
         # bf16 x bf16 products are exact in fp32; only the order of the d additions differs
         np.testing.assert_allclose(z[rows], ref, rtol=0, atol=2e-5 * np.sqrt(spec.d) * np.abs(ref).max())
-    lost = np.nonzero(head < 0)[0]
-    assert np.isnan(z[lost]).all()                         # rows of unroutable tokens are not written
-    assert lost.size == (1 if spec.n_heads > 1 else 0)
+    lost = np.nonzero((head < 0) | ~live)[0]
+    assert np.isnan(z[lost]).all()         # rows of unroutable tokens and of zero-advantage responses are not written
+    assert (head < 0).sum() == (1 if spec.n_heads > 1 else 0)
 
 
 @pytest.mark.parametrize("spec,prm", [
