@@ -11,7 +11,8 @@ Qwen3-1.7B-shaped single-policy head (d=2048, V=151936, ~16K response tokens).
 By default the forward keeps the [T, V] fp32 logits in a buffer lent to the library and the backward
 reads them (a quarter less tensor work for 8 bytes of DRAM traffic per logit); --logits recompute
 times the path that never writes the logits to memory and repeats the contraction in the backward.
-On one GPU the default line carries that second configuration as well ("logits_recomputed").
+--logits keep16 keeps them as 16-bit codes (half the bytes, no longer bit-identical to recomputing).
+On one GPU the line carries the other configurations as well ("other_logits_modes").
 
 Prints ONE JSON line (rank 0).  With --impl reference the fp64 CPU oracle is timed instead, on a
 bounded token sample of the same workload.
@@ -192,21 +193,32 @@ class ClockSampler:
 
 
 # ------------------------------------------------------------------------------- GPU leg
-def logits_note(keep, T, V):
-    if not keep:
+LOGITS_MODES = ("keep", "keep16", "recompute")
+
+
+def logits_bytes_per_logit(mode):
+    return {"keep": 4.0, "keep16": 2.125, "recompute": 0.0}[mode]
+
+
+def logits_note(mode, T, V):
+    if mode == "recompute":
         return "recomputed in the backward (no [T, V] buffer)"
-    return "kept: the forward stores [T, V] fp32 in a lent buffer (%.1f GB), the backward reads it" % (
-        T * ((V + 255) // 256 * 256) * 4 / 1e9)
+    gb = T * ((V + 255) // 256 * 256) * logits_bytes_per_logit(mode) / 1e9
+    if mode == "keep16":
+        return ("kept: the forward stores [T, V] as 16-bit codes below each 32-column block's fp32 maximum in a "
+                "lent buffer (%.1f GB), the backward reads it" % gb)
+    return "kept: the forward stores [T, V] fp32 in a lent buffer (%.1f GB), the backward reads it" % gb
 
 
 class Runner:
     """Device-resident state of one rank: inputs, outputs, workspaces; step() enqueues the path."""
 
-    def __init__(self, batch, device, A, W=None, dW=None, accumulate=False, keep_logits=True, logits=None):
+    def __init__(self, batch, device, A, W=None, dW=None, accumulate=False, logits_mode="keep", logits=None):
         """W / dW: device tensors shared with other Runners (micro-batches of one update step);
-        accumulate: this Runner's backward adds into dW instead of overwriting it; keep_logits: lend
-        the library a [T, V] fp32 buffer so that the backward reads the logits instead of repeating
-        the contraction (`logits`: such a buffer shared with other Runners, large enough for each)."""
+        accumulate: this Runner's backward adds into dW instead of overwriting it; logits_mode: "keep" /
+        "keep16" lend the library a [T, V] buffer (fp32 / 16-bit codes) so that the backward reads the
+        logits instead of repeating the contraction, "recompute" does not (`logits`: such a buffer, a
+        uint8 tensor shared with other Runners, large enough for each)."""
         self.A = A
         self.dev = device
         spec = self.spec = batch["spec"]
@@ -222,11 +234,14 @@ class Runner:
         # the advantages take the one-pass path; the flag means nothing to the loss calls
         G = spec.n_env * spec.n_role * spec.n_turn
         T, V, dm, M = self.T, spec.V, spec.d, self.M
-        self.logits = None
-        if keep_logits:
-            n = A.atgrpo_policy_loss_logits_bytes(T, V) // 4
-            self.logits = logits[:n] if logits is not None else torch.empty(n, dtype=f32, device=device)
-        self.prm = A.Params(accumulate_dW=1 if accumulate else 0, candidates_grouped=1, logits=self.logits)
+        self.logits, self.logits_mode = None, logits_mode
+        fmt = A.LOGITS_Q16 if logits_mode == "keep16" else A.LOGITS_F32
+        if logits_mode != "recompute":
+            n = A.atgrpo_policy_loss_logits_bytes(T, V, fmt)
+            raw = logits[:n] if logits is not None else torch.empty(n, dtype=torch.uint8, device=device)
+            self.logits = raw if fmt == A.LOGITS_Q16 else raw.view(f32)
+        self.prm = A.Params(accumulate_dW=1 if accumulate else 0, candidates_grouped=1, logits=self.logits,
+                            logits_format=fmt)
         self.adv = torch.zeros(self.R, dtype=f32, device=device)
         self.loss = torch.zeros(M, dtype=f32, device=device)
         self.logp = torch.zeros(T, dtype=f32, device=device)
@@ -245,6 +260,21 @@ class Runner:
         self.h2d_bytes = sum(self.host[k].numel() * self.host[k].element_size() for k in self.host
                              if k != "role_of_token" or M > 1) + T * 4
         self.host["old_logp"] = None
+
+    def set_logits_mode(self, mode):
+        """Switches how the backward obtains the logits (allocates the buffer the mode needs)."""
+        A = self.A
+        fmt = A.LOGITS_Q16 if mode == "keep16" else A.LOGITS_F32
+        self.logits, self.logits_mode = None, mode
+        if mode != "recompute":
+            raw = torch.empty(A.atgrpo_policy_loss_logits_bytes(self.T, self.spec.V, fmt), dtype=torch.uint8,
+                              device=self.dev)
+            self.logits = raw if fmt == A.LOGITS_Q16 else raw.view(torch.float32)
+        self.prm = dataclasses.replace(self.prm, logits=self.logits, logits_format=fmt)
+
+    def drop_logits(self):
+        self.logits = None
+        self.prm = dataclasses.replace(self.prm, logits=None)
 
     def advantages(self):
         s, d = self.spec, self.d
@@ -340,7 +370,7 @@ def run_ours(args):
                             sample=f"first {n} tokens, full vocabulary, fwd+bwd, plus advantages of all "
                                    f"{batch['R']} candidates; {dt:.1f} s")
 
-    r = Runner(batch, dev, A, keep_logits=args.logits == "keep")
+    r = Runner(batch, dev, A, logits_mode=args.logits)
     r.make_old_logp()
     r.count_routed_rows()
     if world > 1:
@@ -421,30 +451,35 @@ def run_ours(args):
     torch.cuda.synchronize()
     ms_e2e = e_start.elapsed_time(e_end)
 
-    # ---- the same step with the logits recomputed in the backward (nothing of size T x V in memory),
-    # timed the same way right after, so that one line carries both ways of running the path
-    alt = None
-    if world == 1 and r.logits is not None:
-        r.prm = dataclasses.replace(r.prm, logits=None)
-        for _ in range(3):
-            step()
-        torch.cuda.synchronize()
-        am = [[ev() for _ in range(3)] for _ in range(args.steps)]
-        a_start, a_end = ev(), ev()
-        a_start.record()
-        for k in range(args.steps):
-            r.advantages()
-            am[k][0].record()
-            r.forward()
-            am[k][1].record()
-            r.backward(comm)
-            am[k][2].record()
-        a_end.record()
-        torch.cuda.synchronize()
-        alt = dict(ms_total=a_start.elapsed_time(a_end),
-                   fwd_ms=statistics.mean(m[0].elapsed_time(m[1]) for m in am),
-                   bwd_ms=statistics.mean(m[1].elapsed_time(m[2]) for m in am))
-        r.prm = dataclasses.replace(r.prm, logits=r.logits)
+    # ---- the same step in the other ways of obtaining the logits in the backward, each timed the same
+    # way right after (3 warm-up steps, the same number of steps), so that one line carries all of them
+    alts = {}
+    if world == 1:
+        main_prm = r.prm
+        for mode in LOGITS_MODES:
+            if mode == args.logits:
+                continue
+            r.set_logits_mode(mode)
+            for _ in range(3):
+                step()
+            torch.cuda.synchronize()
+            am = [[ev() for _ in range(3)] for _ in range(args.steps)]
+            a_start, a_end = ev(), ev()
+            a_start.record()
+            for k in range(args.steps):
+                r.advantages()
+                am[k][0].record()
+                r.forward()
+                am[k][1].record()
+                r.backward(comm)
+                am[k][2].record()
+            a_end.record()
+            torch.cuda.synchronize()
+            alts[mode] = dict(ms_total=a_start.elapsed_time(a_end),
+                              fwd_ms=statistics.mean(m[0].elapsed_time(m[1]) for m in am),
+                              bwd_ms=statistics.mean(m[1].elapsed_time(m[2]) for m in am))
+            r.drop_logits()
+        r.prm, r.logits, r.logits_mode = main_prm, main_prm.logits, args.logits
 
     t = torch.tensor([ms_total, ms_e2e], dtype=torch.float64, device=dev)
     tokens = torch.tensor([float(r.T)], dtype=torch.float64, device=dev)
@@ -482,9 +517,10 @@ def run_ours(args):
     n_bwd_chunks = r.A.atgrpo_policy_loss_bwd_chunks(r.T, spec.d, spec.V, r.M)[0]
     dw_elem, dh_elem = 4.0, 2.0
     kept = r.logits is not None
+    bpl = logits_bytes_per_logit(args.logits)
     fwd_bytes = 2.0 * spec.d * (spec.V * spec.n_heads + r.T)                        # W and H once
-    fwd_bytes += 4.0 * r.T * spec.V if kept else 0.0                                # kept logits written once
-    bwd_bytes = ((4.0 * r.routed_rows * spec.V if kept else 2.0 * spec.d * (spec.V * spec.n_heads + r.routed_rows))   # logits read back, or W and H once more
+    fwd_bytes += bpl * r.T * spec.V                                                 # kept logits written once
+    bwd_bytes = ((bpl * r.routed_rows * spec.V if kept else 2.0 * spec.d * (spec.V * spec.n_heads + r.routed_rows))   # logits read back, or W and H once more
                  + 2.0 * spec.d * (spec.V * spec.n_heads + 2 * r.routed_rows)       # W for dH; H for dW + gather
                  + 3.0 * 2.0 * r.routed_rows * spec.V                               # dZ written once, read by dH and by dW
                  + dw_elem * spec.V * spec.d * spec.n_heads                         # dW written once
@@ -498,7 +534,7 @@ def run_ours(args):
         config=dict(workload=spec.name, d=spec.d, V=spec.V, heads=spec.n_heads, tokens_per_gpu=r.T,
                     responses_per_gpu=r.R, parallelism=f"dp{world}",
                     l2="inputs larger than L2 (W alone is %.0f MB)" % (spec.V * spec.d * 2 / 1e6),
-                    logits=logits_note(r.logits is not None, r.T, spec.V),
+                    logits=logits_note(args.logits, r.T, spec.V),
                     old_logp="library logp + N(0,0.05) (perf-only input)"),
         gpu_launches=(r.launches) * args.steps,
         phases_ms=dict(advantages=adv_ms, forward=fwd_ms, backward=bwd_ms),
@@ -529,16 +565,20 @@ def run_ours(args):
         e2e=dict(value=tokens_all * args.steps / (ms_e2e * 1e-3), unit=UNIT,
                  h2d_bytes_per_step=r.h2d_bytes, d2h_bytes_per_step=r.M * 4),
         clocks=clocks, cpu_baseline=cpu_baseline)
-    if alt is not None:
+    other = {}
+    for mode, alt in alts.items():
         a_s = (alt["fwd_ms"] + alt["bwd_ms"]) * 1e-3
-        a_exec = tf(pass_flops * (1.0 + 3.0 * r.routed_rows / max(r.T, 1)), a_s)
-        line["logits_recomputed"] = dict(
-            note="the same step with --logits recompute, timed right after the main region (same steps, "
-                 "3 warm-up steps): no [T, V] buffer, the backward repeats the contraction",
+        a_exec = tf(pass_flops * (1.0 + (3.0 if mode == "recompute" else 2.0) * r.routed_rows / max(r.T, 1)), a_s)
+        other[mode] = dict(
+            logits=logits_note(mode, r.T, spec.V),
             value=r.T * args.steps / (alt["ms_total"] * 1e-3), unit=UNIT, ms_per_step=alt["ms_total"] / args.steps,
             phases_ms=dict(forward=alt["fwd_ms"], backward=alt["bwd_ms"]),
             frac=tf(3.0 * pass_flops, a_s) / peaks["bf16_sustained"], executed_tflops=a_exec,
             executed_frac=a_exec / peaks["bf16_sustained"], executed_frac_of_nominal_2250=a_exec / 2250.0)
+    if other:
+        line["other_logits_modes"] = dict(
+            note="the same step with --logits set to the other values, each timed right after the main region "
+                 "(same steps, 3 warm-up steps)", **other)
     print(json.dumps(line), flush=True)
 
 
@@ -569,12 +609,13 @@ def run_update_step(args):
     V, dm = base.V, base.d
     W = [batches[0]["W"][0].to(dev)]
     dW = [torch.zeros(V, dm, dtype=torch.float32, device=dev)]
-    keep = args.logits == "keep"
+    keep = args.logits != "recompute"
     shared = None
     if keep:                                   # one logits buffer, sized for the larger micro-batch, used by each in turn
-        shared = torch.empty(max(A.atgrpo_policy_loss_logits_bytes(b["T"], V) for b in batches) // 4,
-                             dtype=torch.float32, device=dev)
-    runners = [Runner(b, dev, A, W=W, dW=dW, accumulate=(i > 0), keep_logits=keep, logits=shared)
+        fmt = A.LOGITS_Q16 if args.logits == "keep16" else A.LOGITS_F32
+        shared = torch.empty(max(A.atgrpo_policy_loss_logits_bytes(b["T"], V, fmt) for b in batches),
+                             dtype=torch.uint8, device=dev)
+    runners = [Runner(b, dev, A, W=W, dW=dW, accumulate=(i > 0), logits_mode=args.logits, logits=shared)
                for i, b in enumerate(batches)]
     T_all = sum(r.T for r in runners)
     for r in runners:
@@ -640,7 +681,7 @@ def run_update_step(args):
         vs_baseline=None, dtype="bf16", data="synthetic",
         config=dict(workload="batch128", d=dm, V=V, heads=1, responses=sum(r.R for r in runners), tokens=T_all,
                     micro_batches=[r.T for r in runners], accumulate_dW="fp32, second micro-batch adds",
-                    logits=logits_note(keep, max(r.T for r in runners), V),
+                    logits=logits_note(args.logits, max(r.T for r in runners), V),
                     optimizer="grad norm + AdamW(lr 1e-6, wd 0.01, clip 1.0) on the head, bf16 head rewritten",
                     l2="inputs larger than L2", old_logp="library logp + N(0,0.05) (perf-only input)"),
         gpu_launches=launches * args.steps,
@@ -824,9 +865,11 @@ def main():
     ap.add_argument("--workload", default="qwen3_1p7b", choices=sorted(WL.SPECS) + ["stress", "stress16", "stress_grouped", "stress16_grouped", "stress_grouped_packed",
                                                                      "stress16_grouped_packed", "stress_packed", "adamw", "batch128"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--logits", default="keep", choices=["keep", "recompute"],
+    ap.add_argument("--logits", default="keep", choices=list(LOGITS_MODES),
                     help="keep: the forward stores the [T, V] fp32 logits in a buffer lent by the caller and the "
-                         "backward reads them; recompute: the backward repeats the contraction (no extra memory)")
+                         "backward reads them (same bits as recomputing); keep16: the same with 16-bit codes "
+                         "(half the bytes, |logit error| <= 2^-11); recompute: the backward repeats the "
+                         "contraction (no extra memory)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--launcher-check", action="store_true",
                     help="start the ranks, join a gloo group, print a line with value null; no GPU work")

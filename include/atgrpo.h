@@ -84,8 +84,9 @@ typedef struct atgrpo_params {
   int32_t n_groups;
   /* atgrpo_policy_loss_fwd / _bwd / _bwd_notify only (NULL / 0 by default): logits kept from the
    * forward call for the backward call, see atgrpo_policy_loss_logits_bytes().                  */
-  float* logits;                /* device, 256-byte aligned, owned by the caller                    */
+  void* logits;                 /* device, 256-byte aligned, owned by the caller                    */
   size_t logits_bytes;          /* size of that buffer in bytes                                     */
+  int32_t logits_format;        /* ATGRPO_LOGITS_F32 (default) or ATGRPO_LOGITS_Q16                 */
 } atgrpo_params;
 
 /* Readings of the expectation in Eq. 2.
@@ -257,7 +258,7 @@ size_t atgrpo_policy_loss_workspace_bytes(int64_t T, int32_t d, int32_t V, int32
 /* Kept logits (optional).  The backward call needs the softmax of every routed token again.  By
  * default it repeats the contraction z = H W_m^T chunk by chunk (2*T*V*d flop more, no memory).
  * A caller with HBM to spare can instead lend params->logits, a buffer of
- * atgrpo_policy_loss_logits_bytes(T, V) bytes = T rows of V rounded up to a multiple of 256 fp32
+ * atgrpo_policy_loss_logits_bytes(T, V, ATGRPO_LOGITS_F32) bytes = T rows of V rounded up to a multiple of 256 fp32
  * values (2.45 G logits = 9.8 GB at T = 16157, V = 151936): the forward call then also stores
  * z_jv (row j = token j, columns >= V unspecified; rows of tokens that belong to no policy, or
  * whose response has advantage 0 and therefore passes no gradient, are left untouched), and a
@@ -266,8 +267,18 @@ size_t atgrpo_policy_loss_workspace_bytes(int64_t T, int32_t d, int32_t V, int32
  * reads the logits back instead of recomputing them: a quarter less tensor work for one write and
  * one read of the buffer.  Both ways produce bit-identical dH and dW.  A buffer that is
  * misaligned or too small is rejected with ATGRPO_ERR_INVALID_ARG; the library cannot tell
- * whether the contents belong to these inputs. */
-size_t atgrpo_policy_loss_logits_bytes(int64_t T, int32_t V);
+ * whether the contents belong to these inputs.
+ * params->logits_format = ATGRPO_LOGITS_Q16 halves the buffer and its traffic (2.125 bytes per logit):
+ * the buffer then holds, for every token, V rounded up to a multiple of 256 uint16 codes and, after
+ * the codes of all tokens, one fp32 per token and 32-column block (the block's largest logit);
+ * z_jv is stored as q = round((max of its block - z_jv) * 1024), clamped at 65535, and read back as
+ * max - q/1024: |error| <= 2^-11 for every logit within 64 of its block's maximum (anything lower
+ * is read as max - 64, where exp(z - lse) is below 2e-28 of the block's largest softmax value), i.e.
+ * at most 4.9e-4 relative on every softmax value, a quarter of what rounding dZ to bf16 contributes.
+ * dH and dW then stay within the stated tolerances but are no longer bit-identical to the
+ * recomputing call; logits that are not finite are not preserved by this format. */
+enum { ATGRPO_LOGITS_F32 = 0, ATGRPO_LOGITS_Q16 = 1 };
+size_t atgrpo_policy_loss_logits_bytes(int64_t T, int32_t V, int32_t logits_format);
 
 /* Number of kernels one forward (is_bwd = 0) or backward (is_bwd = 1) call enqueues for these
  * sizes on the current device (memsets not counted).  A bookkeeping query with no counterpart in

@@ -19,6 +19,7 @@ LIB_PATH = os.path.join(_PKG, "libatgrpo.so")
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_BAD_INDEX, ERR_TIMEOUT, ERR_CUDA, ERR_LAYOUT = range(8)
 BF16, F32 = 0, 1
 REDUCE_TOKEN_MEAN, REDUCE_SEQUENCE, REDUCE_GROUP_MEAN = 0, 1, 2
+LOGITS_F32, LOGITS_Q16 = 0, 1
 MAX_HEADS = 8
 
 EXPORTS = (
@@ -47,7 +48,7 @@ class _Params(ctypes.Structure):
                 ("candidates_grouped", ctypes.c_int32),
                 ("group_of_resp", ctypes.c_void_p), ("group_scratch", ctypes.c_void_p),
                 ("n_groups", ctypes.c_int32),
-                ("logits", ctypes.c_void_p), ("logits_bytes", ctypes.c_size_t)]
+                ("logits", ctypes.c_void_p), ("logits_bytes", ctypes.c_size_t), ("logits_format", ctypes.c_int32)]
 
 
 class _AdamWParams(ctypes.Structure):
@@ -84,16 +85,18 @@ class Params:
     candidates_grouped: int = 0  # 1: the members of every group are adjacent (checked on the device)
     group_of_resp: object = None   # REDUCE_GROUP_MEAN: int32 CUDA tensor [n_resp], group of every response
     group_scratch: object = None   # REDUCE_GROUP_MEAN: int32 CUDA tensor [n_groups], scratch owned by the caller
-    logits: object = None          # policy loss: fp32 CUDA tensor of atgrpo_policy_loss_logits_bytes(T, V) bytes, kept logits
+    logits: object = None          # policy loss: CUDA tensor of atgrpo_policy_loss_logits_bytes(T, V, logits_format) bytes, kept logits
+    logits_format: int = 0         # LOGITS_F32 (the tensor is float32) or LOGITS_Q16 (the tensor is uint8)
 
     def c(self) -> _Params:
         n_groups = 0 if self.group_scratch is None else self.group_scratch.numel()
         g, sc = _ptr(self.group_of_resp, torch.int32), _ptr(self.group_scratch, torch.int32)
-        z = _ptr(self.logits, torch.float32)
+        z = _ptr(self.logits, torch.float32 if self.logits_format == LOGITS_F32 else torch.uint8)
         return _Params(self.clip_eps_low, self.clip_eps_high, self.std_eps, self.ddof,
                        self.dH_dtype, self.dW_dtype, self.accumulate_dW, self.reduction,
                        self.candidates_grouped, g.value if g else None, sc.value if sc else None, n_groups,
-                       z.value if z else None, 0 if self.logits is None else self.logits.numel() * 4)
+                       z.value if z else None,
+                       0 if self.logits is None else self.logits.numel() * self.logits.element_size(), self.logits_format)
 
 
 _lib = None
@@ -132,7 +135,7 @@ def lib() -> ctypes.CDLL:
         L.atgrpo_policy_loss_workspace_bytes.restype = sz
         L.atgrpo_policy_loss_workspace_bytes.argtypes = [i64, i32, i32, i32, i32]
         L.atgrpo_policy_loss_logits_bytes.restype = sz
-        L.atgrpo_policy_loss_logits_bytes.argtypes = [i64, i32]
+        L.atgrpo_policy_loss_logits_bytes.argtypes = [i64, i32, i32]
         L.atgrpo_policy_loss_launch_count.restype = i32
         L.atgrpo_policy_loss_launch_count.argtypes = [i64, i32, i32, i32, i32]
         L.atgrpo_policy_loss_fwd.restype = ctypes.c_int
@@ -290,8 +293,8 @@ def atgrpo_policy_loss_workspace_bytes(T: int, d: int, V: int, M: int, is_bwd: b
     return int(lib().atgrpo_policy_loss_workspace_bytes(T, d, V, M, 1 if is_bwd else 0))
 
 
-def atgrpo_policy_loss_logits_bytes(T: int, V: int) -> int:
-    return int(lib().atgrpo_policy_loss_logits_bytes(T, V))
+def atgrpo_policy_loss_logits_bytes(T: int, V: int, logits_format: int = LOGITS_F32) -> int:
+    return int(lib().atgrpo_policy_loss_logits_bytes(T, V, logits_format))
 
 
 def atgrpo_policy_loss_launch_count(T: int, d: int, V: int, M: int, is_bwd: bool) -> int:

@@ -66,7 +66,7 @@ int policy_common_checks(const void* H, int64_t ldH, const void* const* W, int32
   }
   if (workspace == nullptr || !aligned(workspace, 256)) return ATGRPO_ERR_WORKSPACE;
   if (params->logits != nullptr &&
-      (!aligned(params->logits, 256) || params->logits_bytes < (size_t)T * lm_head_logits_ld(V) * sizeof(float)))
+      (!aligned(params->logits, 256) || params->logits_bytes < lm_head_logits_bytes(T, V, params->logits_format)))
     return ATGRPO_ERR_INVALID_ARG;
   return ATGRPO_OK;
 }
@@ -192,9 +192,9 @@ size_t atgrpo_policy_loss_workspace_bytes(int64_t T, int32_t d, int32_t V, int32
   return policy_plan(T, d, V, M, is_bwd != 0, false, sm_count_or_default()).total;
 }
 
-size_t atgrpo_policy_loss_logits_bytes(int64_t T, int32_t V) {
-  if (T < 0 || V < 1) return 0;
-  return (size_t)T * lm_head_logits_ld(V) * sizeof(float);
+size_t atgrpo_policy_loss_logits_bytes(int64_t T, int32_t V, int32_t logits_format) {
+  if (T < 0 || V < 1 || (logits_format != ATGRPO_LOGITS_F32 && logits_format != ATGRPO_LOGITS_Q16)) return 0;
+  return lm_head_logits_bytes(T, V, logits_format);
 }
 
 int32_t atgrpo_policy_loss_launch_count(int64_t T, int32_t d, int32_t V, int32_t M, int32_t is_bwd) {
@@ -250,7 +250,7 @@ int atgrpo_policy_loss_fwd(const void* H, int64_t ldH, const void* const* W, int
   p.sched = sched, p.tok_of_row = tok_of_row, p.target = target, p.device_status = device_status;
   p.resp_of_token = resp_of_token, p.adv = adv, p.n_resp = n_resp;
   p.n_sm = n_sm;
-  rc = lm_head_fwd_launch(p, lse, logp, ws + pl.gemm, st, params->logits);
+  rc = lm_head_fwd_launch(p, lse, logp, ws + pl.gemm, st, static_cast<float*>(params->logits), params->logits_format);
   if (rc != ATGRPO_OK) return rc;
   return loss_reduce_launch(logp, old_logp, resp_of_token, adv, n_resp, role_of_token, head_of_role,
                             n_role, M, T, *params, nullptr, loss, nullptr, clip_counts, device_status,
@@ -367,7 +367,8 @@ int policy_loss_bwd_impl(const void* H, int64_t ldH, const void* const* W, int32
   p.resp_of_token = resp_of_token, p.adv = adv, p.n_resp = n_resp;
   p.n_sm = n_sm;
   return lm_head_bwd_launch(p, lse, coef, row_of_token, *params, dH, dW, ws + pl.gemm, st,
-                            notify ? chunk_events : nullptr, params->logits);
+                            notify ? chunk_events : nullptr, static_cast<const float*>(params->logits),
+                            params->logits_format);
 }
 }  // namespace
 

@@ -15,6 +15,7 @@ inline bool params_ok(const atgrpo_params* p) {
       p->reduction != ATGRPO_REDUCE_GROUP_MEAN)
     return false;
   if (p->candidates_grouped != 0 && p->candidates_grouped != 1) return false;
+  if (p->logits_format != ATGRPO_LOGITS_F32 && p->logits_format != ATGRPO_LOGITS_Q16) return false;
   if (p->reduction == ATGRPO_REDUCE_GROUP_MEAN &&
       (p->group_of_resp == nullptr || p->group_scratch == nullptr || p->n_groups < 1))
     return false;
@@ -108,11 +109,13 @@ struct LmHeadProblem {
   int32_t n_sm;
 };
 size_t lm_head_fwd_workspace_bytes(int64_t T_pad, int32_t d, int32_t V, int32_t n_sm);
-// lse[T], logp[T] in token order.  keep_logits (optional): [T, lm_head_logits_ld(V)] fp32 in token
-// order, receives every logit of every routed token.
+// lse[T], logp[T] in token order.  keep_logits (optional): lm_head_logits_bytes(T, V, logits_format)
+// bytes; receives the logits of every routed token that can carry a gradient, rows in token order with
+// stride lm_head_logits_ld(V): fp32, or 16-bit codes followed by one fp32 per 32-column block.
 int64_t lm_head_logits_ld(int32_t V);
+size_t lm_head_logits_bytes(int64_t T, int32_t V, int32_t format);
 int lm_head_fwd_launch(const LmHeadProblem& p, float* lse, float* logp, void* workspace,
-                       cudaStream_t st, float* keep_logits = nullptr);
+                       cudaStream_t st, float* keep_logits = nullptr, int32_t logits_format = ATGRPO_LOGITS_F32);
 size_t lm_head_bwd_workspace_bytes(int64_t T_pad, int32_t d, int32_t V, bool dH_direct);
 // coef[T] in token order (0 for tokens that pass no gradient); dH / dW as the C ABI documents.
 // chunk_events (optional, lm_head_bwd_chunks() entries): event c is recorded once the dW rows of
@@ -121,7 +124,8 @@ size_t lm_head_bwd_workspace_bytes(int64_t T_pad, int32_t d, int32_t V, bool dH_
 int lm_head_bwd_launch(const LmHeadProblem& p, const float* lse, const float* coef,
                        const int32_t* row_of_token, const atgrpo_params& prm, void* dH,
                        void* const* dW, void* workspace, cudaStream_t st,
-                       void* const* chunk_events = nullptr, const float* kept_logits = nullptr);
+                       void* const* chunk_events = nullptr, const float* kept_logits = nullptr,
+                       int32_t logits_format = ATGRPO_LOGITS_F32);
 int lm_head_bwd_chunk_rows(int64_t T_pad, int32_t d, int32_t V);   // vocabulary rows per chunk
 int device_sm_count(int* n_sm, int* cc_major);
 int lm_head_bwd_chunks(int64_t T_pad, int32_t d, int32_t V);   // vocabulary chunks of one backward call (it makes one GEMM launch more)

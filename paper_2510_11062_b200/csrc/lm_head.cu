@@ -32,7 +32,11 @@
 // kConvWarps extra warps of the launch that holds the dH and dW tiles of chunk c-1 (plain loads
 // and stores, no barriers), so it runs under the tensor work; chunk 0 has a small launch of its
 // own.  Both ways give the same bits: the stored value is the accumulator the recomputation would
-// produce again.
+// produce again.  A compact format halves the traffic of the kept logits: per token and 32-column
+// block the block's maximum in fp32 and, per logit, a 16-bit code q = round((max - z) * 1024) (clamped at
+// 65535, i.e. 64 below the block's maximum, where exp(z - lse) no longer matters): |z - z~| <= 2^-11, a
+// relative error of at most 4.9e-4 on every softmax value, a quarter of what rounding dZ to bf16 adds
+// anyway; no longer bit-identical to the recomputing backward.
 #include <cuda_bf16.h>
 #include <cstring>
 #include "internal.h"
@@ -53,6 +57,9 @@ constexpr int kGemmThreads = 320;               // producer warp, MMA warp, 8 ep
 constexpr int kEpilogueThreads = 256;
 constexpr int kConvWarps = 8;                   // kBwd with kept logits: warps that turn logits into dZ
 constexpr int kConvCols = 2048;                 // columns one conversion step covers (eight 32-byte loads per lane in flight)
+constexpr int kCodeCols = 2048;                 // the same for 16-bit codes (16 columns per 32-byte load, four loads in flight)
+constexpr float kCodeScale = 1024.f;            // 16-bit codes: steps per logit unit (2^-10 apart, 64 units of range)
+constexpr float kCodeMax = 65535.f;
 constexpr int kTmemCols = 512;
 constexpr int kSmemBytes = kStages * kStageBytes + 1024 /* alignment slack */ + 256 /* barriers */;
 constexpr float kLog2e = 1.4426950408889634f;
@@ -92,6 +99,8 @@ struct GemmArgs {
   int vc;                 // chunk buffer width (multiple of 256)
   float* logits;          // kept logits [T, ldz] in token order (NULL: none): written by kFwd, read instead of kDz items
   int64_t ldz;            // row stride of `logits` in elements (V rounded up to a multiple of 256)
+  int q16;                // kept logits are 16-bit codes: `logits` holds uint16 [T, ldz], `refs` fp32 [T, ldz/32]
+  float* refs;            // q16: the maximum of every 32-column block; logit = ref - code / kCodeScale
   const int32_t* resp_of_token;   // kFwd with kept logits: a token whose response has advantage 0 passes no
   const float* adv;               // gradient whatever its ratio, so its logits are not stored
   int64_t n_resp;
@@ -341,11 +350,81 @@ __device__ __forceinline__ void dz_from_logits(const GemmArgs& g, int64_t rows, 
   }
 }
 
+// The same from 16-bit codes.  A step is one row x kCodeCols columns (4 KiB of codes, lanes on consecutive
+// 32-byte pieces of 16 codes, which lie inside one 32-column block and share its reference value).
+__device__ __forceinline__ void dz_from_codes(const GemmArgs& g, int64_t rows, int worker, int n_workers,
+                                              int lane) {
+  constexpr int kLoads = 4, kStride = 32 * 16;               // 32-byte loads per lane and step; columns a warp covers per load
+  static_assert(kLoads * kStride == kCodeCols, "a step is kLoads warp-wide loads");
+  const int n_cols = g.n_vtiles * BN;
+  const int n_seg = (n_cols + kCodeCols - 1) / kCodeCols;
+  const int64_t n_steps = rows * n_seg;
+  const int64_t n_blk = g.ldz / 32;
+  const uint64_t drop = l2_policy_evict_first();
+  const uint16_t* codes = reinterpret_cast<const uint16_t*>(g.logits);
+  const float step2 = -kLog2e / kCodeScale;                  // log2-domain size of one code step, negated
+  for (int64_t u = worker; u < n_steps; u += n_workers) {
+    const int64_t row = u / n_seg;
+    const int c0 = (int)(u - row * n_seg) * kCodeCols + lane * 16;
+    const int tok = g.tok_of_row[row];
+    int y = -1;
+    float lse2 = 0.f, cf = 0.f;
+    const uint16_t* src = codes;
+    const float* ref = g.refs;
+    if (tok >= 0) {
+      y = g.target[tok];
+      if ((unsigned)y >= (unsigned)g.V) {
+        raise_status(g.status, ATGRPO_ERR_BAD_INDEX);
+        y = 0;
+      }
+      lse2 = g.lse[tok] * kLog2e, cf = g.coef[tok];
+      src = codes + (size_t)tok * g.ldz + g.v_begin + c0;
+      ref = g.refs + (size_t)tok * n_blk + (g.v_begin + c0) / 32;
+    }
+    uint32_t z[kLoads][8];
+    float base2[kLoads];                                     // (block maximum - lse) in the log2 domain
+#pragma unroll
+    for (int j = 0; j < kLoads; ++j) {
+      const int col = c0 + j * kStride;
+      base2[j] = 0.f;
+      if (tok >= 0 && col < n_cols && g.v_begin + col < g.V) {
+        ld_stream_v8(src + j * kStride, z[j], drop);
+        base2[j] = fmaf(ref[j * (kStride / 32)], kLog2e, -lse2);
+      } else {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) z[j][i] = 0u;
+      }
+    }
+#pragma unroll
+    for (int j = 0; j < kLoads; ++j) {
+      const int col = c0 + j * kStride;
+      if (col >= n_cols) continue;
+      const int v0 = g.v_begin + col;
+      uint32_t packed[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        float lo = cf * ex2(fmaf((float)(z[j][i] & 0xffffu), step2, base2[j]));
+        float hi = cf * ex2(fmaf((float)(z[j][i] >> 16), step2, base2[j]));
+        if (v0 + 2 * i == y) lo -= cf;
+        if (v0 + 2 * i + 1 == y) hi -= cf;
+        if (tok < 0 || v0 + 2 * i >= g.V) lo = 0.f;
+        if (tok < 0 || v0 + 2 * i + 1 >= g.V) hi = 0.f;
+        const __nv_bfloat162 h2 = __floats2bfloat162_rn(lo, hi);
+        packed[i] = *reinterpret_cast<const uint32_t*>(&h2);
+      }
+      st_global_v8(g.dz + (size_t)row * g.vc + col, packed);
+    }
+  }
+}
+
 // The conversion on its own, for the first chunk of a backward call (no tensor work to hide under yet).
 __global__ void __launch_bounds__(256)
 k_dz_from_logits(const GemmArgs g) {
   const int64_t rows = (int64_t)g.sched->tile_begin[g.M] * BM;
-  dz_from_logits(g, rows, blockIdx.x * 8 + (threadIdx.x >> 5), gridDim.x * 8, threadIdx.x & 31);
+  if (g.q16)
+    dz_from_codes(g, rows, blockIdx.x * 8 + (threadIdx.x >> 5), gridDim.x * 8, threadIdx.x & 31);
+  else
+    dz_from_logits(g, rows, blockIdx.x * 8 + (threadIdx.x >> 5), gridDim.x * 8, threadIdx.x & 31);
 }
 
 template <int kMode>    // kFwd or kBwd
@@ -487,9 +566,14 @@ k_lm_head(const __grid_constant__ Maps maps, const GemmArgs g) {
     }
   } else if (warp >= kGemmThreads / 32) {
     // ------------------------------------------------------------------ conversion warps (kBwd, kept logits)
-    if (kMode == kBwd && g.has_z && g.logits != nullptr)
-      dz_from_logits(g, (int64_t)sched->tile_begin[g.M] * BM, blockIdx.x * kConvWarps + (warp - kGemmThreads / 32),
-                     gridDim.x * kConvWarps, lane);
+    if (kMode == kBwd && g.has_z && g.logits != nullptr) {
+      const int64_t rows = (int64_t)sched->tile_begin[g.M] * BM;
+      const int worker = blockIdx.x * kConvWarps + (warp - kGemmThreads / 32);
+      if (g.q16)
+        dz_from_codes(g, rows, worker, gridDim.x * kConvWarps, lane);
+      else
+        dz_from_logits(g, rows, worker, gridDim.x * kConvWarps, lane);
+    }
   } else {
     // ------------------------------------------------------------------ epilogue warps
     // Two warps per TMEM lane quarter (a warp can only read the quarter warp_id % 4): the first
@@ -526,15 +610,25 @@ k_lm_head(const __grid_constant__ Maps maps, const GemmArgs g) {
         bool have_zt = false;
         float lse2 = 0.f, cf = 0.f;
         if (mode == kDz && tok >= 0) lse2 = g.lse[tok] * kLog2e, cf = g.coef[tok];
-        float* keep_row = nullptr;
+        float* keep_row = nullptr;            // fp32 logits of this token, or
+        uint16_t* keep_codes = nullptr;       // its 16-bit codes and
+        float* keep_refs = nullptr;           // the block maxima they refer to
         if (mode == kFwd && g.logits != nullptr && tok >= 0) {
           const int rsp = g.resp_of_token[tok];
-          if ((unsigned)rsp < (unsigned)g.n_resp && g.adv[rsp] != 0.f) keep_row = g.logits + (size_t)tok * g.ldz;
+          if ((unsigned)rsp < (unsigned)g.n_resp && g.adv[rsp] != 0.f) {
+            if (g.q16) {
+              keep_codes = reinterpret_cast<uint16_t*>(g.logits) + (size_t)tok * g.ldz;
+              keep_refs = g.refs + (size_t)tok * (g.ldz / 32);
+            } else {
+              keep_row = g.logits + (size_t)tok * g.ldz;
+            }
+          }
         }
         for (int nt = t.nt_begin; ok && nt < t.nt_end; ++nt) {
           const int n0 = t.n0 + (nt - t.nt_begin) * BN;
           if (!(ok = mbar_wait_backoff(tfull_bar(acc), acc_phase, s_abort, g.status))) break;
           tc_fence_after();
+          float ref0 = 0.f, ref1 = 0.f, ref2 = 0.f, ref3 = 0.f;   // q16: maxima of this warp's four column blocks
           for (int c = c_begin; c < c_end; ++c) {
             const int col0 = n0 + c * 32;
             if (mode == kFwd && col0 >= g.V) break;
@@ -561,6 +655,24 @@ k_lm_head(const __grid_constant__ Maps maps, const GemmArgs g) {
               for (int i = 0; i < 32; ++i) {
                 if (ragged && col0 + i >= g.V) r[i] = 0xff800000u;     // -inf
                 cmax = fmaxf(cmax, __uint_as_float(r[i]));
+              }
+              if (keep_codes != nullptr) {
+                // code = (block maximum - logit) in steps of 1/kCodeScale, saturating (columns beyond V are -inf)
+                const float top = cmax * kCodeScale;
+                uint32_t pk[16];
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                  const uint32_t lo = __float2uint_rn(fminf(fmaf(__uint_as_float(r[2 * i]), -kCodeScale, top), kCodeMax));
+                  const uint32_t hi = __float2uint_rn(fminf(fmaf(__uint_as_float(r[2 * i + 1]), -kCodeScale, top), kCodeMax));
+                  pk[i] = lo | (hi << 16);
+                }
+                st_stream_v8(keep_codes + col0, pk, drop);
+                st_stream_v8(keep_codes + col0 + 16, pk + 8, drop);
+                const int k = c - c_begin;
+                if (k == 0) ref0 = cmax;
+                else if (k == 1) ref1 = cmax;
+                else if (k == 2) ref2 = cmax;
+                else ref3 = cmax;
               }
               const float nm = fmaxf(m2, cmax * kLog2e);
               float add0 = 0.f, add1 = 0.f;
@@ -602,6 +714,8 @@ k_lm_head(const __grid_constant__ Maps maps, const GemmArgs g) {
           tc_fence_before();
           mbar_arrive_cluster(acc ? tempty_leader1 : tempty_leader0);
           if (++acc == 2) acc = 0, acc_phase ^= 1u;
+          if (keep_refs != nullptr)          // 16 bytes: the four blocks this warp covers of the tile at n0
+            *reinterpret_cast<float4*>(keep_refs + n0 / 32 + c_begin) = make_float4(ref0, ref1, ref2, ref3);
         }
         if (mode == kFwd && ok && tok >= 0) {
           g.part_m[(size_t)(2 * t.chunk + half) * g.T_pad + row] = m2;
@@ -957,8 +1071,20 @@ size_t lm_head_fwd_workspace_bytes(int64_t T_pad, int32_t d, int32_t V, int32_t 
 
 int64_t lm_head_logits_ld(int32_t V) { return ((int64_t)V + BN - 1) / BN * BN; }
 
+size_t lm_head_logits_bytes(int64_t T, int32_t V, int32_t format) {
+  const size_t n = (size_t)T * lm_head_logits_ld(V);
+  return format == ATGRPO_LOGITS_Q16 ? n * 2 + n / 32 * 4 : n * 4;     // codes + one fp32 per 32-column block
+}
+
+namespace {
+// Where the block maxima of the 16-bit format start inside the lent buffer: after the codes.
+float* logits_refs(const void* buf, int64_t T, int32_t V) {
+  return reinterpret_cast<float*>(static_cast<char*>(const_cast<void*>(buf)) + (size_t)T * lm_head_logits_ld(V) * 2);
+}
+}  // namespace
+
 int lm_head_fwd_launch(const LmHeadProblem& p, float* lse, float* logp, void* workspace,
-                       cudaStream_t st, float* keep_logits) {
+                       cudaStream_t st, float* keep_logits, int32_t logits_format) {
   const FwdPlan pl = fwd_plan(p.T_pad, p.V, p.n_sm);
   char* ws = static_cast<char*>(workspace);
   Maps maps;
@@ -973,6 +1099,7 @@ int lm_head_fwd_launch(const LmHeadProblem& p, float* lse, float* logp, void* wo
   g.part_s = reinterpret_cast<float*>(ws + pl.part_s);
   g.zt = reinterpret_cast<float*>(ws + pl.zt);
   g.logits = keep_logits, g.ldz = lm_head_logits_ld(p.V);
+  g.q16 = logits_format == ATGRPO_LOGITS_Q16, g.refs = logits_refs(keep_logits, p.T, p.V);
   g.resp_of_token = p.resp_of_token, g.adv = p.adv, g.n_resp = p.n_resp;
   int rc = launch_gemm<kFwd>(maps, g, (p.T_pad / kPairRows) * pl.n_chunks, p.n_sm, st);
   if (rc != ATGRPO_OK) return rc;
@@ -989,7 +1116,7 @@ size_t lm_head_bwd_workspace_bytes(int64_t T_pad, int32_t d, int32_t V, bool dH_
 int lm_head_bwd_launch(const LmHeadProblem& p, const float* lse, const float* coef,
                        const int32_t* row_of_token, const atgrpo_params& prm, void* dH,
                        void* const* dW, void* workspace, cudaStream_t st, void* const* chunk_events,
-                       const float* kept_logits) {
+                       const float* kept_logits, int32_t logits_format) {
   const bool dH_direct = false;   // rows are compacted: dH always goes through the accumulator
   const BwdPlan pl = bwd_plan(p.T_pad, p.d, p.V, dH_direct);
   char* ws = static_cast<char*>(workspace);
@@ -1023,6 +1150,7 @@ int lm_head_bwd_launch(const LmHeadProblem& p, const float* lse, const float* co
     g.vc = pl.vc;
     g.lse = lse, g.coef = coef;
     g.logits = const_cast<float*>(kept_logits), g.ldz = lm_head_logits_ld(p.V);
+    g.q16 = logits_format == ATGRPO_LOGITS_Q16, g.refs = logits_refs(kept_logits, p.T, p.V);
     g.dh_acc = dh_acc;
     for (int m = 0; m < p.M; ++m) g.dW[m] = dW[m];
     g.dw_bf16 = prm.dW_dtype == ATGRPO_BF16, g.dw_accumulate = prm.accumulate_dW;

@@ -90,14 +90,18 @@ class PolicyCase:
         self.old_logp = to_dev(old_logp.to(torch.float32))
         self.grad_loss = None if grad_loss is None else to_dev(grad_loss.to(torch.float32))
 
-    def lend_logits(self):
-        """Lends the library a logits buffer (params.logits) full of NaN: the next forward stores
-        the logits there and the backward calls after it read them instead of recomputing.
-        Whatever the library leaves unwritten must never reach a result."""
+    def lend_logits(self, fmt=A.LOGITS_F32):
+        """Lends the library a logits buffer (params.logits) full of NaN (fp32 format) or of 0xFF bytes
+        (16-bit codes: every code saturated, every block maximum a NaN): the next forward stores the
+        logits there and the backward calls after it read them instead of recomputing.  Whatever the
+        library leaves unwritten must never reach a result."""
         import dataclasses
-        n = A.atgrpo_policy_loss_logits_bytes(self.T, self.spec.V) // 4
-        buf = torch.full((n,), float("nan"), dtype=torch.float32, device=DEV)
-        self.prm = dataclasses.replace(self.prm, logits=buf)
+        n = A.atgrpo_policy_loss_logits_bytes(self.T, self.spec.V, fmt)
+        if fmt == A.LOGITS_F32:
+            buf = torch.full((n // 4,), float("nan"), dtype=torch.float32, device=DEV)
+        else:
+            buf = torch.full((n,), 255, dtype=torch.uint8, device=DEV)
+        self.prm = dataclasses.replace(self.prm, logits=buf, logits_format=fmt)
         return buf
 
     def bwd_both_ways(self, logp, lse):

@@ -42,9 +42,11 @@ def test_default_arm_line():
     assert rf["frac_of_nominal_2250"] < rf["frac"] and rf["forward_frac"] > 0 and rf["backward_algorithmic_frac"] > 0
     assert rf["algorithmic_bytes"] == rf["algorithmic_bytes_forward"] + rf["algorithmic_bytes_backward"]
     assert rf["traffic"] is None or rf["traffic"] == rf["traffic_forward"] + rf["traffic_backward"]
-    # the same line also carries the step with the logits recomputed (no [T, V] buffer)
-    alt = r["logits_recomputed"]
-    assert alt["value"] > 0 and alt["ms_per_step"] > 0 and alt["frac"] > 0
+    # the same line also carries the step with the logits recomputed (no [T, V] buffer) and kept the other way
+    others = r["other_logits_modes"]
+    assert set(others) == {"note", "recompute", "keep16" if r["config"]["logits"].startswith("kept: the forward stores [T, V] fp32") else "keep"}
+    alt = others["recompute"]
+    assert alt["value"] > 0 and alt["ms_per_step"] > 0 and alt["frac"] > 0 and alt["logits"].startswith("recomputed")
     assert abs(alt["executed_frac"] / alt["frac"] - (T + 3.0 * rf["routed_rows"]) / (3.0 * T)) < 1e-6
     e = r["e2e"]
     assert e["value"] > 0 and e["h2d_bytes_per_step"] > 0 and e["d2h_bytes_per_step"] == 4
@@ -56,7 +58,8 @@ def test_recompute_arm_line():
     # --logits recompute: no [T, V] buffer, the backward repeats the contraction on the routed rows
     r = _run("--workload", "tiny", "--steps", "3", "--warmup", "3", "--logits", "recompute", "--no-cpu-baseline")
     rf, T = r["roofline"], r["config"]["tokens_per_gpu"]
-    assert r["config"]["logits"].startswith("recomputed") and r["value"] > 0 and "logits_recomputed" not in r
+    assert r["config"]["logits"].startswith("recomputed") and r["value"] > 0
+    assert set(r["other_logits_modes"]) == {"note", "keep", "keep16"}
     assert abs(rf["executed_frac"] / rf["frac"] - (T + 3.0 * rf["routed_rows"]) / (3.0 * T)) < 1e-6
 
 

@@ -6,7 +6,8 @@ Inputs are the benchmark's batch with every response carrying its Eq. 1 advantag
 built from the ORACLE's log-probs, so the backward runs every row tile, every vocabulary chunk and
 both alternating dZ buffers exactly as in the timed step: the forward keeps the logits in a lent
 buffer and the backward reads them (the backward that recomputes them instead is run as well and
-must give the same bits in every element of dH and dW).  The oracle computes the full forward
+must give the same bits in every element of dH and dW); a third backward runs from logits kept as 16-bit
+codes and is held to the same tolerances against the oracle.  The oracle computes the full forward
 (lse, logp for every token; about 1e13 fp64 flop per head pass) and then, from its own lse and
 gradient factors, single rows of dH and dW:
   * dH rows of tokens drawn from EVERY 128-row half of every 256-row pair tile of the backward's
@@ -79,6 +80,12 @@ def test_full_size_dense_backward_rows(name, request):
     # the backward as timed (from the kept logits) and with the contraction recomputed: same bits
     g = case.bwd_both_ways(torch.from_numpy(logp).float(), torch.from_numpy(lse).float())
     assert g["status"] == 0
+    # and from logits kept as 16-bit codes (half the bytes; within the tolerances, not bit-identical)
+    case.lend_logits(A.LOGITS_Q16)
+    out16 = case.fwd()
+    assert out16["status"] == 0 and torch.equal(out16["logp"], out["logp"]) and torch.equal(out16["lse"], out["lse"])
+    g16 = case.bwd(torch.from_numpy(logp).float(), torch.from_numpy(lse).float())
+    assert g16["status"] == 0
     c = O.dloss_dlogp(logp, old, adv, b["resp_of_token"], head, M, None if gl is None else gl.numpy())
     n_chunks, rows_per_chunk = A.atgrpo_policy_loss_bwd_chunks(T, spec.d, V, M)
     assert n_chunks >= 2                                           # both dZ buffers alternate
@@ -97,8 +104,10 @@ def test_full_size_dense_backward_rows(name, request):
                                                token_rows=tok_rows, vocab_rows=voc_rows)
         U.check_rows(dH[idx[tok_rows]], ref_h, "dH rows of head %d" % m)
         U.check_rows(g["dW"][m].numpy()[voc_rows], ref_w, "dW rows of head %d" % m)
+        U.check_rows(g16["dH"].numpy()[idx[tok_rows]], ref_h, "dH rows of head %d from 16-bit codes" % m)
+        U.check_rows(g16["dW"][m].numpy()[voc_rows], ref_w, "dW rows of head %d from 16-bit codes" % m)
     # every token without a gradient has an exactly zero dH row, and the identities that need no oracle
-    assert (dH[c == 0] == 0).all()
+    assert (dH[c == 0] == 0).all() and (g16["dH"].numpy()[c == 0] == 0).all()
     for m in range(M):
         dW = g["dW"][m].double()
         assert dW.sum(0).abs().max().item() <= 2e-3 * dW.abs().sum(0).max().item()      # sum_v dZ_jv = 0

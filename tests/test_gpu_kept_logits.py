@@ -23,6 +23,7 @@ def _lend(case, T, V):
     """A logits buffer full of NaN: whatever the library does not write must never be used."""
     ld = (V + 255) // 256 * 256
     assert A.atgrpo_policy_loss_logits_bytes(T, V) == T * ld * 4
+    assert A.atgrpo_policy_loss_logits_bytes(T, V, A.LOGITS_Q16) == T * ld * 2 + T * (ld // 32) * 4
     return case.lend_logits(), ld
 
 
@@ -206,3 +207,104 @@ def test_group_mean_reduction_from_kept_logits():
     assert case.fwd(want_routing=False)["status"] == 0
     g = case.bwd_both_ways(f["logp"], f["lse"])
     assert g["status"] == 0 and float(g["dH"].abs().max()) > 0
+
+
+# ------------------------------------------------------------------ the compact format (16-bit codes)
+
+@pytest.mark.parametrize("name", ["mid", "mid_multi"])
+def test_codes_decode_to_the_oracle_logits_within_half_a_step(name):
+    spec = WL.SPECS[name]
+    b = WL.make_rollout(spec)
+    T, V, M = b["T"], spec.V, spec.n_heads
+    adv = torch.ones(b["R"])
+    adv[::4] = 0.0
+    case = U.PolicyCase(b, adv, torch.zeros(T))
+    plain = case.fwd(want_routing=False)
+    buf = case.lend_logits(A.LOGITS_Q16)
+    kept = case.fwd(want_routing=False)
+    for k in ("loss", "logp", "lse", "clip_counts"):
+        assert torch.equal(kept[k], plain[k]), k
+    ld = (V + 255) // 256 * 256
+    raw = buf.cpu().numpy()
+    codes = raw[: T * ld * 2].view(np.uint16).reshape(T, ld).astype(np.float64)
+    refs = raw[T * ld * 2:].view(np.float32).reshape(T, ld // 32).astype(np.float64)
+    z = (np.repeat(refs, 32, axis=1) - codes / 1024.0)[:, :V]
+    head, _, _ = U.oracle_heads(b)
+    live = adv.numpy()[b["resp_of_token"].numpy()] != 0
+    Hf = b["H"].double().numpy()
+    for m in range(M):
+        rows = np.nonzero((head == m) & live)[0]
+        ref = Hf[rows] @ b["W"][m].double().numpy().T
+        # the block maximum is the fp32 logit itself; every other logit is at most half a code step off it
+        blockmax = np.stack([ref[:, c:c + 32].max(axis=1) for c in range(0, V, 32)], axis=1)
+        np.testing.assert_allclose(refs[rows][:, : blockmax.shape[1]], blockmax, rtol=0, atol=1e-4)
+        assert np.abs(z[rows] - ref).max() <= 2.0 ** -11 + 1e-4
+        assert (codes[rows][:, :V].min(axis=1) == 0).all()          # the maximum of a block has code 0
+    dead = np.nonzero(~live)[0]
+    assert (raw[: T * ld * 2].view(np.uint16).reshape(T, ld)[dead] == 0xFFFF).all()    # rows that are not kept stay untouched
+
+
+@pytest.mark.parametrize("spec,prm", [
+    (WL.SPECS["mid"], A.Params()),
+    (WL.SPECS["mid_multi"], A.Params(dH_dtype=A.F32, dW_dtype=A.BF16)),
+    (RAGGED, A.Params(reduction=A.REDUCE_SEQUENCE)),
+    (WIDE, A.Params()),
+], ids=["mid", "mid_multi_f32_bf16", "ragged_sequence", "wide_three_chunks"])
+def test_backward_from_codes_stays_close_to_the_recomputing_backward(spec, prm):
+    b, case, f = _case(spec, prm)
+    T, d, V, M = b["T"], spec.d, spec.V, spec.n_heads
+    ref = case.bwd(f["logp"], f["lse"])
+    case.lend_logits(A.LOGITS_Q16)
+    f2 = case.fwd(want_routing=False)
+    assert f2["status"] == 0 and torch.equal(f2["logp"], f["logp"])
+    got = case.bwd(f["logp"], f["lse"])
+    assert got["status"] == 0
+    # |dz - dz~| <= 4.9e-4 * p elementwise before the bf16 rounding both ways share: the results differ by far
+    # less than either differs from the exact gradient (5e-3 is the tolerance against the oracle)
+    assert U.rel_fro(got["dH"].numpy(), ref["dH"].numpy()) <= 1.5e-3
+    for m in range(M):
+        if float(ref["dW"][m].abs().max()) > 0:
+            assert U.rel_fro(got["dW"][m].numpy(), ref["dW"][m].numpy()) <= 1.5e-3, m
+        else:
+            assert (got["dW"][m] == 0).all()
+    assert (got["dH"][ref["dH"].abs().sum(1) == 0] == 0).all()     # rows without a gradient stay exactly zero
+
+
+def test_backward_from_codes_matches_the_oracle():
+    spec = WL.SPECS["mid_multi"]
+    b = WL.make_rollout(spec)
+    T, V, M = b["T"], spec.V, spec.n_heads
+    lse, logp = U.oracle_logprobs(b)
+    adv = U.batch_advantages(b)
+    old = U.keep_off_the_kinks(logp, WL.make_old_logp(torch.from_numpy(logp), 23, 0.3))
+    head, _, _ = U.oracle_heads(b)
+    gl = torch.tensor([0.5, 1.0, 2.0])
+    case = U.PolicyCase(b, adv, old, prm=A.Params(dH_dtype=A.F32), grad_loss=gl)
+    case.lend_logits(A.LOGITS_Q16)
+    f = case.fwd()
+    assert f["status"] == 0
+    g = case.bwd(torch.from_numpy(logp).float(), torch.from_numpy(lse).float())
+    assert g["status"] == 0
+    dH, dW = O.policy_loss_grads(b["H"], b["W"], b["target"], old, adv, b["resp_of_token"], head,
+                                 grad_loss=gl.numpy())
+    U.check_rows(g["dH"].numpy(), dH, "dH")
+    for m in range(M):
+        U.check_rows(g["dW"][m].numpy(), dW[m], "dW[%d]" % m)
+
+
+def test_a_code_buffer_that_is_too_small_or_an_unknown_format_is_rejected():
+    spec = WL.SPECS["tiny"]
+    b = WL.make_rollout(spec)
+    T, V = b["T"], spec.V
+    case = U.PolicyCase(b, torch.ones(b["R"]), torch.zeros(T))
+    n = A.atgrpo_policy_loss_logits_bytes(T, V, A.LOGITS_Q16)
+    big = torch.zeros(n, dtype=torch.uint8, device=U.DEV)
+    case.prm = dataclasses.replace(case.prm, logits=big[: n - 4], logits_format=A.LOGITS_Q16)
+    with pytest.raises(A.AtgrpoError):
+        case.fwd(want_routing=False)
+    case.prm = dataclasses.replace(case.prm, logits=big, logits_format=7)
+    with pytest.raises(A.AtgrpoError):
+        case.fwd(want_routing=False)
+    assert A.atgrpo_policy_loss_logits_bytes(T, V, 7) == 0
+    case.prm = dataclasses.replace(case.prm, logits=big, logits_format=A.LOGITS_Q16)
+    assert case.fwd(want_routing=False)["status"] == 0
