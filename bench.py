@@ -160,6 +160,13 @@ class ClockSampler:
         except Exception:
             self.proc = None
 
+    def mark(self):
+        """The timed region starts here: samples written so far belong to the warm-up (same load)."""
+        try:
+            self.skip = os.path.getsize(self.tmp.name)
+        except OSError:
+            self.skip = 0
+
     def stop(self):
         out = dict(sm_mhz=None, sm_max_mhz=None, reasons=[])
         if self.proc is None:
@@ -171,9 +178,14 @@ class ClockSampler:
             self.proc.kill()
         self.tmp.flush()
         self.tmp.seek(0)
+        text = self.tmp.read()
+        skip = getattr(self, "skip", 0)
+        window = "timed region"
+        if len(text[skip:].splitlines()) < 3:          # a short region: take the warm-up steps' samples as well
+            skip, window = 0, "warm-up and timed region (same load)"
         sm, smax, power, reasons = [], [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for ln in self.tmp.read().splitlines():
+        for ln in text[skip:].splitlines():
             f = [x.strip() for x in ln.split(",")]
             if len(f) < 8:
                 continue
@@ -188,7 +200,7 @@ class ClockSampler:
         os.unlink(self.tmp.name)
         if sm:
             out = dict(sm_mhz=statistics.median(sm), sm_max_mhz=max(smax), power_w_max=max(power),
-                       samples=len(sm), reasons=sorted(reasons))
+                       samples=len(sm), window=window, reasons=sorted(reasons))
         return out
 
 
@@ -386,6 +398,7 @@ def run_ours(args):
         r.backward(comm)
 
     ev = lambda: torch.cuda.Event(enable_timing=True)
+    sampler = ClockSampler(local) if rank == 0 else None      # started before the warm-up: nvidia-smi takes a moment to start
     for _ in range(max(args.warmup, 3)):
         step()
     torch.cuda.synchronize()
@@ -393,9 +406,10 @@ def run_ours(args):
         torch.distributed.barrier()
 
     # ---- timed region: device-resident inputs
-    sampler = ClockSampler(local) if rank == 0 else None
     marks = [[ev() for _ in range(4)] for _ in range(args.steps)]
     torch.cuda.synchronize()
+    if sampler:
+        sampler.mark()
     t_start, t_end = ev(), ev()
     t_start.record()
     for k in range(args.steps):

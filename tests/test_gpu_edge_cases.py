@@ -46,6 +46,19 @@ def _check(b, sigma=0.3, prm=None, tol_fro=5e-3):
     assert g2["status"] == 0 and torch.equal(g2["dH"], g["dH"])
     for m in range(M):
         assert torch.equal(g2["dW"][m], g["dW"][m]), m
+    # and with the logits kept as 16-bit codes: the oracle's tolerances again
+    case.lend_logits(A.LOGITS_Q16)
+    out3 = case.fwd()
+    assert out3["status"] == 0 and torch.equal(out3["logp"], out["logp"]) and torch.equal(out3["lse"], out["lse"])
+    g3 = case.bwd(torch.from_numpy(logp).float(), torch.from_numpy(lse).float())
+    assert g3["status"] == 0
+    if np.linalg.norm(dH) > 0:
+        assert U.rel_fro(g3["dH"].numpy(), dH) <= tol_fro
+    for m in range(M):
+        if np.linalg.norm(dW[m]) > 0:
+            assert U.rel_fro(g3["dW"][m].numpy(), dW[m]) <= tol_fro
+        else:
+            assert (g3["dW"][m] == 0).all()
     return out, g
 
 
