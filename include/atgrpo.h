@@ -255,17 +255,18 @@ int atgrpo_clipped_loss(
  * ------------------------------------------------------------------------------------------ */
 size_t atgrpo_policy_loss_workspace_bytes(int64_t T, int32_t d, int32_t V, int32_t M, int32_t is_bwd);
 
-/* Kept logits (optional).  The backward call needs the softmax of every routed token again.  By
- * default it repeats the contraction z = H W_m^T chunk by chunk (2*T*V*d flop more, no memory).
- * A caller with HBM to spare can instead lend params->logits, a buffer of
- * atgrpo_policy_loss_logits_bytes(T, V, ATGRPO_LOGITS_F32) bytes = T rows of V rounded up to a multiple of 256 fp32
- * values (2.45 G logits = 9.8 GB at T = 16157, V = 151936): the forward call then also stores
+/* Kept logits (optional; a memory / compute trade the paper says nothing about).  The gradient of
+ * Eq. 2 needs the softmax pi_theta(v | .) of every token that passes a gradient, i.e. its logits
+ * again.  By default the backward call repeats the contraction z = H W_m^T chunk by chunk
+ * (2*T*V*d flop more, no memory).  A caller with HBM to spare can instead lend params->logits, a
+ * buffer of atgrpo_policy_loss_logits_bytes(T, V, ATGRPO_LOGITS_F32) bytes = T rows of V rounded
+ * up to a multiple of 256 fp32 values (9.8 GB at T = 16157, V = 151936): the forward call then also stores
  * z_jv (row j = token j, columns >= V unspecified; rows of tokens that belong to no policy, or
  * whose response has advantage 0 and therefore passes no gradient, are left untouched), and a
  * backward call that is given the same buffer -- after a forward call
  * with the same H, W, target, adv and routing arguments, nothing having written to it in between --
  * reads the logits back instead of recomputing them: a quarter less tensor work for one write and
- * one read of the buffer.  Both ways produce bit-identical dH and dW.  A buffer that is
+ * one read of the buffer.  With fp32 logits both ways produce bit-identical dH and dW.  A buffer that is
  * misaligned or too small is rejected with ATGRPO_ERR_INVALID_ARG; the library cannot tell
  * whether the contents belong to these inputs.
  * params->logits_format = ATGRPO_LOGITS_Q16 halves the buffer and its traffic (2.125 bytes per logit):
