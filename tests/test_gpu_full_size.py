@@ -90,6 +90,15 @@ def test_full_size_sparse_advantages(name):
     assert (dH[rest] == 0).all()
     for m in range(M):
         assert U.rel_fro(g["dW"][m].numpy(), dW[m]) <= 5e-3, m
+    if name in ("qwen3_8b", "long_resp"):
+        # the same from logits kept as 16-bit codes (d = 4096 / the longest batch): the oracle's tolerances again
+        case.lend_logits(A.LOGITS_Q16)
+        assert case.fwd()["status"] == 0
+        g16 = case.bwd(logp_in, lse_in)
+        assert g16["status"] == 0
+        assert U.rel_fro(g16["dH"].numpy()[act], dH_act) <= 5e-3 and (g16["dH"].numpy()[rest] == 0).all()
+        for m in range(M):
+            assert U.rel_fro(g16["dW"][m].numpy(), dW[m]) <= 5e-3, m
 
 
 @pytest.mark.parametrize("dw_dtype", [A.F32, A.BF16])
