@@ -59,7 +59,6 @@ constexpr int kConvWarps = 8;                   // kBwd with kept logits: warps 
 constexpr int kConvCols = 2048;                 // columns one conversion step covers (eight 32-byte loads per lane in flight)
 constexpr int kCodeCols = 2048;                 // the same for 16-bit codes (16 columns per 32-byte load, four loads in flight)
 constexpr float kCodeScale = 1024.f;            // 16-bit codes: steps per logit unit (2^-10 apart, 64 units of range)
-constexpr float kCodeMax = 65535.f;
 constexpr int kTmemCols = 512;
 constexpr int kSmemBytes = kStages * kStageBytes + 1024 /* alignment slack */ + 256 /* barriers */;
 constexpr float kLog2e = 1.4426950408889634f;
@@ -155,6 +154,20 @@ __device__ __forceinline__ void ld_stream_v8(const void* p, uint32_t* v, uint64_
                : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
                : "l"(p), "l"(policy)
                : "memory");
+}
+
+// 16-bit codes.  A float-to-integer cvt clamps to the range of its destination type (+inf, the code of a
+// column beyond the vocabulary, becomes 65535).
+__device__ __forceinline__ uint32_t pack_codes(float lo, float hi) {
+  uint32_t r;
+  asm("{\n\t.reg .b16 l, h;\n\tcvt.rni.u16.f32 l, %1;\n\tcvt.rni.u16.f32 h, %2;\n\tmov.b32 %0, {l, h};\n\t}"
+      : "=r"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+
+__device__ __forceinline__ void unpack_codes(uint32_t v, float& lo, float& hi) {
+  asm("{\n\t.reg .b16 l, h;\n\tmov.b32 {l, h}, %2;\n\tcvt.rn.f32.u16 %0, l;\n\tcvt.rn.f32.u16 %1, h;\n\t}"
+      : "=f"(lo), "=f"(hi) : "r"(v));
 }
 
 struct Tile {
@@ -299,11 +312,14 @@ __device__ __forceinline__ void dz_from_logits(const GemmArgs& g, int64_t rows, 
                                                int lane) {
   const int n_cols = g.n_vtiles * BN;                       // columns of the chunk buffer this chunk fills
   const int n_seg = (n_cols + kConvCols - 1) / kConvCols;
-  const int64_t n_steps = rows * n_seg;
   const uint64_t drop = l2_policy_evict_first();
-  for (int64_t u = worker; u < n_steps; u += n_workers) {
-    const int64_t row = u / n_seg;
-    const int c0 = (int)(u - row * n_seg) * kConvCols + lane * 8;   // this lane's first column in the buffer
+  // step u = row * n_seg + seg for u = worker, worker + n_workers, ...: (row, seg) advanced without dividing
+  const int d_row = n_workers / n_seg, d_seg = n_workers % n_seg;
+  int64_t row = worker / n_seg;
+  for (int seg = worker % n_seg; row < rows; row += d_row, seg += d_seg) {
+    if (seg >= n_seg) seg -= n_seg, ++row;
+    if (row >= rows) break;
+    const int c0 = seg * kConvCols + lane * 8;              // this lane's first column in the buffer
     const int tok = g.tok_of_row[row];
     int y = -1;
     float lse2 = 0.f, cf = 0.f;
@@ -336,10 +352,15 @@ __device__ __forceinline__ void dz_from_logits(const GemmArgs& g, int64_t rows, 
       const int v0 = g.v_begin + col;                        // vocabulary row of z[j][0]
       float gz[8];
 #pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        gz[i] = cf * ex2(fmaf(__uint_as_float(z[j][i]), kLog2e, -lse2));
-        if (v0 + i == y) gz[i] -= cf;
-        if (tok < 0 || v0 + i >= g.V) gz[i] = 0.f;
+      for (int i = 0; i < 8; ++i) gz[i] = cf * ex2(fmaf(__uint_as_float(z[j][i]), kLog2e, -lse2));
+      // (a padding row has z = 0, lse = 0 and cf = 0: exact zeros.)  Only the piece that holds the target
+      // column or reaches beyond the vocabulary needs more
+      if ((unsigned)(y - v0) < 8u || v0 + 8 > g.V) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          if (v0 + i == y) gz[i] -= cf;
+          if (v0 + i >= g.V) gz[i] = 0.f;
+        }
       }
       uint4 w;
       __nv_bfloat162* wh = reinterpret_cast<__nv_bfloat162*>(&w);
@@ -358,14 +379,16 @@ __device__ __forceinline__ void dz_from_codes(const GemmArgs& g, int64_t rows, i
   static_assert(kLoads * kStride == kCodeCols, "a step is kLoads warp-wide loads");
   const int n_cols = g.n_vtiles * BN;
   const int n_seg = (n_cols + kCodeCols - 1) / kCodeCols;
-  const int64_t n_steps = rows * n_seg;
   const int64_t n_blk = g.ldz / 32;
   const uint64_t drop = l2_policy_evict_first();
   const uint16_t* codes = reinterpret_cast<const uint16_t*>(g.logits);
   const float step2 = -kLog2e / kCodeScale;                  // log2-domain size of one code step, negated
-  for (int64_t u = worker; u < n_steps; u += n_workers) {
-    const int64_t row = u / n_seg;
-    const int c0 = (int)(u - row * n_seg) * kCodeCols + lane * 16;
+  const int d_row = n_workers / n_seg, d_seg = n_workers % n_seg;
+  int64_t row = worker / n_seg;
+  for (int seg = worker % n_seg; row < rows; row += d_row, seg += d_seg) {
+    if (seg >= n_seg) seg -= n_seg, ++row;
+    if (row >= rows) break;
+    const int c0 = seg * kCodeCols + lane * 16;
     const int tok = g.tok_of_row[row];
     int y = -1;
     float lse2 = 0.f, cf = 0.f;
@@ -400,15 +423,20 @@ __device__ __forceinline__ void dz_from_codes(const GemmArgs& g, int64_t rows, i
       const int col = c0 + j * kStride;
       if (col >= n_cols) continue;
       const int v0 = g.v_begin + col;
+      const bool edge = (unsigned)(y - v0) < 16u || v0 + 16 > g.V;   // this piece holds the target column or leaves the vocabulary
       uint32_t packed[8];
 #pragma unroll
       for (int i = 0; i < 8; ++i) {
-        float lo = cf * ex2(fmaf((float)(z[j][i] & 0xffffu), step2, base2[j]));
-        float hi = cf * ex2(fmaf((float)(z[j][i] >> 16), step2, base2[j]));
-        if (v0 + 2 * i == y) lo -= cf;
-        if (v0 + 2 * i + 1 == y) hi -= cf;
-        if (tok < 0 || v0 + 2 * i >= g.V) lo = 0.f;
-        if (tok < 0 || v0 + 2 * i + 1 >= g.V) hi = 0.f;
+        float qlo, qhi;
+        unpack_codes(z[j][i], qlo, qhi);
+        float lo = cf * ex2(fmaf(qlo, step2, base2[j]));
+        float hi = cf * ex2(fmaf(qhi, step2, base2[j]));
+        if (edge) {
+          if (v0 + 2 * i == y) lo -= cf;
+          if (v0 + 2 * i + 1 == y) hi -= cf;
+          if (v0 + 2 * i >= g.V) lo = 0.f;
+          if (v0 + 2 * i + 1 >= g.V) hi = 0.f;
+        }
         const __nv_bfloat162 h2 = __floats2bfloat162_rn(lo, hi);
         packed[i] = *reinterpret_cast<const uint32_t*>(&h2);
       }
@@ -661,11 +689,9 @@ k_lm_head(const __grid_constant__ Maps maps, const GemmArgs g) {
                 const float top = cmax * kCodeScale;
                 uint32_t pk[16];
 #pragma unroll
-                for (int i = 0; i < 16; ++i) {
-                  const uint32_t lo = __float2uint_rn(fminf(fmaf(__uint_as_float(r[2 * i]), -kCodeScale, top), kCodeMax));
-                  const uint32_t hi = __float2uint_rn(fminf(fmaf(__uint_as_float(r[2 * i + 1]), -kCodeScale, top), kCodeMax));
-                  pk[i] = lo | (hi << 16);
-                }
+                for (int i = 0; i < 16; ++i)
+                  pk[i] = pack_codes(fmaf(__uint_as_float(r[2 * i]), -kCodeScale, top),
+                                     fmaf(__uint_as_float(r[2 * i + 1]), -kCodeScale, top));
                 st_stream_v8(keep_codes + col0, pk, drop);
                 st_stream_v8(keep_codes + col0 + 16, pk + 8, drop);
                 const int k = c - c_begin;
