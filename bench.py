@@ -468,7 +468,7 @@ def run_ours(args):
     # ---- the same step in the other ways of obtaining the logits in the backward, each timed the same
     # way right after (3 warm-up steps, the same number of steps), so that one line carries all of them
     alts = {}
-    if world == 1:
+    if world == 1 and not args.main_only:
         main_prm = r.prm
         for mode in LOGITS_MODES:
             if mode == args.logits:
@@ -884,6 +884,8 @@ def main():
                          "backward reads them (same bits as recomputing); keep16: the same with 16-bit codes "
                          "(half the bytes, |logit error| <= 2^-11); recompute: the backward repeats the "
                          "contraction (no extra memory)")
+    ap.add_argument("--main-only", action="store_true",
+                    help="time only the --logits mode asked for, not the other ones after it (profiling runs)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--launcher-check", action="store_true",
                     help="start the ranks, join a gloo group, print a line with value null; no GPU work")

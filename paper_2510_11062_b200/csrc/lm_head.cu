@@ -864,13 +864,22 @@ k_lse_combine(const Schedule* sched, int M, const int32_t* tok_of_row, int64_t T
   const int grp = threadIdx.y;
   float mx = -INFINITY, s = 0.f;
   if (p < rows) {
-    for (int c = grp; c < n_parts; c += 8) {
-      const float ps = part_s[(size_t)c * T_pad + p];
-      if (ps > 0.f) {                                   // a part without valid columns holds (-inf, 0)
-        const float pm = part_m[(size_t)c * T_pad + p];
-        const float nm = fmaxf(mx, pm);
-        s = s * exp2f(mx - nm) + ps * exp2f(pm - nm);
-        mx = nm;
+    // four parts per round: their eight loads are issued together, then merged in ascending part order
+    for (int c0 = grp; c0 < n_parts; c0 += 32) {
+      float ps[4], pm[4];
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const int c = c0 + 8 * k;
+        ps[k] = c < n_parts ? part_s[(size_t)c * T_pad + p] : 0.f;
+        pm[k] = c < n_parts ? part_m[(size_t)c * T_pad + p] : 0.f;
+      }
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        if (ps[k] > 0.f) {                              // a part without valid columns holds (-inf, 0)
+          const float nm = fmaxf(mx, pm[k]);
+          s = s * exp2f(mx - nm) + ps[k] * exp2f(pm[k] - nm);
+          mx = nm;
+        }
       }
     }
   }
