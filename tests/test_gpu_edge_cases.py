@@ -211,3 +211,13 @@ def test_a_bounded_wait_that_runs_out_reports_timeout_and_leaves_the_context_usa
     assert waited.cpu().tolist() == [1, 1]
     assert A.atgrpo_selftest_bounded_wait(10**9, st, waited) == A.ERR_INVALID_ARG     # limits are capped
     _check(WL.make_rollout(WL.SPECS["tiny"]))
+
+
+@pytest.mark.parametrize("scale", [6.0, 16.0])
+def test_peaked_distributions_with_logits_tens_of_units_apart(scale):
+    # hidden states scaled up: logits of std 6 / 16 (extremes beyond +-25 / +-70), softmax concentrated on a few
+    # entries, most probabilities underflowing; all three ways of obtaining the logits in the backward
+    spec = WL.RolloutSpec("peaked", 4, 2, 2, 4, (10, 10), (40, 40), 256, 5000 + 37, 2, 611, 1)
+    b = WL.make_rollout(spec)
+    b["H"] = (b["H"].float() * scale).to(torch.bfloat16)
+    _check(b, sigma=0.3)
