@@ -179,9 +179,10 @@ class ClockSampler:
         self.tmp.flush()
         self.tmp.seek(0)
         text = self.tmp.read()
-        skip = getattr(self, "skip", 0)
-        window = "timed region"
-        if len(text[skip:].splitlines()) < 3:          # a short region: take the warm-up steps' samples as well
+        skip = getattr(self, "skip", None)
+        window = "timed region" if skip is not None else "warm-up and timed calls"
+        skip = skip or 0
+        if skip and len(text[skip:].splitlines()) < 3:  # a short region: take the warm-up steps' samples as well
             skip, window = 0, "warm-up and timed region (same load)"
         sm, smax, power, reasons = [], [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
@@ -653,10 +654,11 @@ def run_update_step(args):
                             A.AdamWParams(step=step_no[0]))
 
     ev = lambda: torch.cuda.Event(enable_timing=True)
+    sampler = ClockSampler(local)              # started before the warm-up: nvidia-smi takes a moment to start
     for _ in range(max(args.warmup, 3)):
         step()
     torch.cuda.synchronize()
-    sampler = ClockSampler(local)
+    sampler.mark()
     marks = [[ev() for _ in range(3)] for _ in range(args.steps)]
     t0, t1 = ev(), ev()
     t0.record()
