@@ -148,3 +148,50 @@ def test_backward_is_bitwise_repeatable():
     assert torch.equal(a["dH"], c["dH"])
     for x, y in zip(a["dW"], c["dW"]):
         assert torch.equal(x, y)
+
+
+def test_two_calls_on_two_streams_with_their_own_workspaces():
+    # "calls may run concurrently on different streams if they use different workspaces and outputs":
+    # two different batches, forward + backward each, enqueued on two streams without any ordering between
+    # them, must give what each gives alone (one of them with kept logits)
+    dev = U.DEV
+    cases = []
+    for name, keep in (("mid", True), ("mid_multi", False)):
+        b, lse, logp, adv, old = _case(name, 0.3)
+        c = U.PolicyCase(b, adv, old)
+        if keep:
+            c.lend_logits()
+        alone_f = c.fwd(want_routing=False)
+        alone_b = c.bwd(alone_f["logp"], alone_f["lse"])
+        cases.append((b, c, alone_f, alone_b))
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    outs = []
+    torch.cuda.synchronize()
+    for rep in range(3):
+        outs.clear()
+        for (b, c, f, _), st in zip(cases, streams):
+            T, M, d, V = b["T"], c.M, c.spec.d, c.spec.V
+            with torch.cuda.stream(st):
+                o = dict(loss=torch.zeros(M, device=dev), logp=torch.zeros(T, device=dev), lse=torch.zeros(T, device=dev),
+                         dH=torch.zeros(T, d, dtype=torch.bfloat16, device=dev),
+                         dW=[torch.zeros(V, d, device=dev) for _ in range(M)], status=A.new_status(dev),
+                         ws_f=A.workspace(A.atgrpo_policy_loss_workspace_bytes(T, d, V, M, False), dev),
+                         ws_b=A.workspace(A.atgrpo_policy_loss_workspace_bytes(T, d, V, M, True), dev))
+                outs.append(o)
+        for (b, c, f, _), st, o in zip(cases, streams, outs):
+            with torch.cuda.stream(st):
+                A.atgrpo_policy_loss_fwd(c.H, c.W, c.target, c.role_of_token, c.head_of_role, c.resp_of_token, c.adv,
+                                         c.old_logp, c.prm, o["loss"], o["logp"], o["lse"], device_status=o["status"],
+                                         workspace=o["ws_f"])
+        for (b, c, f, _), st, o in zip(cases, streams, outs):
+            with torch.cuda.stream(st):
+                A.atgrpo_policy_loss_bwd(c.H, c.W, c.target, c.role_of_token, c.head_of_role, c.resp_of_token, c.adv,
+                                         c.old_logp, o["logp"], o["lse"], None, c.prm, o["dH"], o["dW"],
+                                         device_status=o["status"], workspace=o["ws_b"])
+        torch.cuda.synchronize()
+        for (b, c, f, g), o in zip(cases, outs):
+            assert int(o["status"].item()) == 0
+            assert torch.equal(o["logp"].cpu(), f["logp"]) and torch.equal(o["loss"].cpu(), f["loss"])
+            assert torch.equal(o["dH"].float().cpu(), g["dH"])
+            for m in range(c.M):
+                assert torch.equal(o["dW"][m].cpu(), g["dW"][m])
